@@ -1,0 +1,145 @@
+/* stb.h - C ABI of the N:M structured-binary linear layer y = W^ x on NVIDIA B200 (sm_100a).
+ *
+ * The layer follows STBLLM (arXiv 2408.01803): of every M = 8 consecutive input columns of
+ * an output row exactly N weights are kept (Section 3.3); a kept weight is +-1 times an
+ * fp16 scale (Eq. 1); within every block of 128 input columns the kept weights of a row are
+ * split into a dense, an intermediate and a sparse region with one scale each (Section 3.4,
+ * "Non-Salient Part"; Algorithm 2, Trisection) and the kept weights of the block's salient
+ * columns carry a second, residual +-1 term with its own scale (Eq. 4; Algorithm 2,
+ * Res_Approx).  In fp32 a kept weight is  s * a_region,  a kept salient weight is
+ * fl32(s1 * a_sal1 + s2 * a_sal2), a dropped weight is 0.
+ *
+ * All entry points are asynchronous on the CUDA stream they are given (a cudaStream_t passed
+ * as void*; NULL = the default stream) unless stated otherwise.  Every data pointer is a
+ * DEVICE pointer owned by the caller unless its comment says HOST.  The library allocates no
+ * device memory and keeps no mutable global state.  Argument errors are returned
+ * synchronously and launch nothing; conditions only the device can see (a corrupt logical
+ * layer, a bounded wait that ran out) are written to the caller's `dev_status` word (device
+ * memory, int32, may be NULL, must be zeroed by the caller) and are read by the caller after
+ * it has synchronised the stream.  Nothing traps, aborts or prints.
+ */
+#ifndef STB_H_
+#define STB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum stb_status {
+  STB_OK = 0,
+  STB_ERR_ARG = 1,          /* null pointer, negative size, bad leading dimension */
+  STB_ERR_SHAPE = 2,        /* n < 1, m < 128 or m not a multiple of 128 */
+  STB_ERR_NM = 3,           /* N outside 1..8 */
+  STB_ERR_SIZE = 4,         /* buffer or workspace too small, batch outside its range */
+  STB_ERR_UNSUPPORTED = 5,  /* dtype or mode this build does not provide */
+  STB_ERR_CORRUPT = 6,      /* device: logical layer or packed header fails validation */
+  STB_ERR_TIMEOUT = 7,      /* device: a bounded wait on an mbarrier ran out */
+  STB_ERR_CUDA = 8          /* a CUDA runtime call failed (launch error) */
+} stb_status;
+
+typedef enum stb_dtype { STB_F16 = 0, STB_BF16 = 1, STB_F32 = 2 } stb_dtype;
+
+/* Logical (unpacked) layer: the quantizer's output, one field per piece of information of
+ * Sections 3.3-3.4.  n output rows, m input columns, N kept of every 8.
+ *   keep    [n][m/8]      bit c (LSB first) of a byte: column 8g+c of group g is kept;
+ *                         every byte has exactly N bits set               (Section 3.3)
+ *   sign    [n][m/8]      bit k: sign of the k-th kept weight of the group in ascending
+ *                         column order, 1 = +1, 0 = -1; bits >= N are zero       (Eq. 1-2)
+ *   region  [n][m/8]      2 bits per kept weight, same rank order: 0 dense, 1 intermediate,
+ *                         2 sparse (Algorithm 2, Trisection), 3 = the column is salient
+ *   sign2   [n][m/128]    bit t: residual sign (Eq. 4) of the kept weight in the t-th
+ *                         salient column (ascending) of the block; 0 where that weight is
+ *                         dropped; bits >= number of salient columns are zero
+ *   salient [m/128][2]    128-bit mask of the block's salient columns, word 0 = columns
+ *                         0..63; at most 32 bits set                  (Algorithm 2, Salient)
+ *   scale   [n][m/128][5] fp16 bit patterns a_dense, a_inter, a_sparse, a_sal1, a_sal2
+ */
+typedef struct stb_logical {
+  int n, m, N;
+  const uint8_t *keep;
+  const uint8_t *sign;
+  const uint16_t *region;
+  const uint32_t *sign2;
+  const uint64_t *salient;
+  const uint16_t *scale;
+} stb_logical;
+
+/* HOST struct filled by stb_packed_info. */
+typedef struct stb_info {
+  int n, m, N;
+  int status;             /* what the pack kernels found: STB_OK or STB_ERR_CORRUPT */
+  uint64_t used_bytes;    /* header + per-block table + all tiles */
+  uint64_t stream_bytes;  /* tiles only: the bytes one GEMV pass streams from HBM */
+} stb_info;
+
+/* One step of stb_layer_stack: out[batch][n] = layer(in[batch][m]).  HOST struct. */
+typedef struct stb_step {
+  const void *packed;
+  int n, m, N;
+  const void *in;   /* fp16 [batch][ldin]  */
+  void *out;        /* fp32 or fp16 [batch][ldout], see odt */
+  stb_dtype odt;    /* STB_F32 or STB_F16 (fp32 sum rounded to nearest even) */
+  int batch;
+  size_t ldin, ldout;
+} stb_step;
+
+/* Upper bound of the packed size of an n x m layer at N:8 (the packed size depends on the
+ * number of salient columns per block, at most 4 bytes per row and block; this is the size
+ * with all of them).  *bytes is HOST memory.  Synchronous, no CUDA call. */
+int stb_pack_size(int n, int m, int N, size_t *bytes);
+
+/* Fused pack / transpose: logical arrays -> the streaming layout read by stb_gemv and
+ * stb_gemm (the counterpart of the paper's matrix compression and value compression steps,
+ * Appendix C).  The packed buffer must be 256-byte aligned and hold stb_pack_size bytes.
+ * Validates on the device that every keep byte has N bits, that sign / region / sign2 carry
+ * no bits beyond their fields, that region 3 marks exactly the kept weights of salient
+ * columns and that no block has more than 32 salient columns; a violation stores
+ * STB_ERR_CORRUPT in *dev_status and in the packed header (the packed data is then not to be
+ * used).  Two small launches on `stream`. */
+int stb_pack(const stb_logical *L, void *packed, size_t packed_bytes, int *dev_status,
+             void *stream);
+
+/* Reads the packed header back (SYNCHRONOUS: waits for `stream`, copies 64 bytes to the
+ * host).  Not for the hot path. */
+int stb_packed_info(const void *packed, stb_info *info, void *stream);
+
+/* Parity hook: decode the packed layer to a dense row-major matrix W[n][ldw].
+ * dt = STB_F32: exactly the fp32 definition at the top of this file.
+ * dt = STB_F16 / STB_BF16: that fp32 value rounded to nearest even. */
+int stb_dequant(const void *packed, int n, int m, int N, void *W, stb_dtype dt, size_t ldw,
+                void *stream);
+
+/* Decode GEMV, batch 1..16:  y[t][i] = sum_j W^[i][j] * x[t][j],  fp32 accumulation.
+ * x: fp16 [batch][ldx] (ldx >= m, ldx a multiple of 8, x 16-byte aligned); y: [batch][ldy]
+ * (ldy >= n) in fp32 (ydt = STB_F32) or fp16 (STB_F16: the fp32 sum rounded to nearest even,
+ * for chaining layers).  The memory-bound case of the paper's Appendix C.2 (decoding stage,
+ * N = batch). */
+int stb_gemv(const void *packed, int n, int m, int N, const void *x, int batch, size_t ldx,
+             void *y, stb_dtype ydt, size_t ldy, int *dev_status, void *stream);
+
+/* Bytes of workspace stb_gemm needs for T tokens (0 if none).  HOST result. */
+int stb_gemm_workspace(int n, int m, int N, int T, size_t *bytes);
+
+/* Prefill GEMM:  Y[t][i] = sum_j W^[i][j] * X[t][j]  on the tensor cores (tcgen05, fp32
+ * accumulation in tensor memory); W^ is decoded tile by tile to bf16 (RN-even).
+ * X: bf16 [T][ldx]; Y: fp32 or bf16 [T][ldy] (ydt).  The compute-bound case of Appendix C.2
+ * (prefilling stage, N = sequence length x batch).  ws / ws_bytes: caller-owned workspace of
+ * stb_gemm_workspace bytes (may be NULL when that is 0). */
+int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size_t ldx, void *Y,
+             stb_dtype ydt, size_t ldy, void *ws, size_t ws_bytes, int *dev_status,
+             void *stream);
+
+/* Runs `count` GEMV steps in order on one stream; every step carries its own N (layer-wise
+ * N:M assignment, Section 3.3).  steps is a HOST array.  Launches only. */
+int stb_layer_stack(const stb_step *steps, int count, int *dev_status, void *stream);
+
+/* Static string for a status code. */
+const char *stb_status_str(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STB_H_ */

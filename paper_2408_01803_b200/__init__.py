@@ -1,0 +1,208 @@
+"""Python binding of libstb.so: the N:M structured-binary linear layer on B200 (sm_100a).
+
+Argument marshalling only: every step of the path (pack, dequant, GEMV, GEMM, layer stack)
+runs in the CUDA kernels behind the C ABI declared in include/stb.h.  torch is used for
+device memory and streams.  There is no CPU fallback: if the shared library is missing the
+import of this package raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libstb.so")
+
+STB_OK, STB_ERR_ARG, STB_ERR_SHAPE, STB_ERR_NM, STB_ERR_SIZE = 0, 1, 2, 3, 4
+STB_ERR_UNSUPPORTED, STB_ERR_CORRUPT, STB_ERR_TIMEOUT, STB_ERR_CUDA = 5, 6, 7, 8
+STB_F16, STB_BF16, STB_F32 = 0, 1, 2
+
+EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv",
+           "stb_gemm_workspace", "stb_gemm", "stb_layer_stack", "stb_status_str"]
+
+
+class StbError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_str(status), status))
+
+
+class _Logical(C.Structure):
+    _fields_ = [("n", C.c_int), ("m", C.c_int), ("N", C.c_int),
+                ("keep", C.c_void_p), ("sign", C.c_void_p), ("region", C.c_void_p),
+                ("sign2", C.c_void_p), ("salient", C.c_void_p), ("scale", C.c_void_p)]
+
+
+class _Info(C.Structure):
+    _fields_ = [("n", C.c_int), ("m", C.c_int), ("N", C.c_int), ("status", C.c_int),
+                ("used_bytes", C.c_uint64), ("stream_bytes", C.c_uint64)]
+
+
+class _Step(C.Structure):
+    _fields_ = [("packed", C.c_void_p), ("n", C.c_int), ("m", C.c_int), ("N", C.c_int),
+                ("inp", C.c_void_p), ("out", C.c_void_p), ("odt", C.c_int), ("batch", C.c_int),
+                ("ldin", C.c_size_t), ("ldout", C.c_size_t)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("libstb.so is not built (%s): run `python -m paper_2408_01803_b200.build`; "
+                          "there is no CPU fallback" % LIB_PATH)
+    lib = C.CDLL(LIB_PATH)
+    v, i, z, p = C.c_void_p, C.c_int, C.c_size_t, C.POINTER
+    lib.stb_pack_size.argtypes = [i, i, i, p(z)]
+    lib.stb_pack.argtypes = [p(_Logical), v, z, v, v]
+    lib.stb_packed_info.argtypes = [v, p(_Info), v]
+    lib.stb_dequant.argtypes = [v, i, i, i, v, i, z, v]
+    lib.stb_gemv.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
+    lib.stb_gemm_workspace.argtypes = [i, i, i, i, p(z)]
+    lib.stb_gemm.argtypes = [v, i, i, i, v, i, z, v, i, z, v, z, v, v]
+    lib.stb_layer_stack.argtypes = [p(_Step), i, v, v]
+    lib.stb_status_str.argtypes = [i]
+    lib.stb_status_str.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "stb_status_str":
+            getattr(lib, name).restype = i
+    return lib
+
+
+_lib = _load()
+
+
+def status_str(status: int) -> str:
+    return _lib.stb_status_str(int(status)).decode()
+
+
+def _check(rc: int, where: str):
+    if rc != STB_OK:
+        raise StbError(rc, where)
+
+
+def _stream(stream=None):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+def pack_size(n: int, m: int, N: int) -> int:
+    out = C.c_size_t()
+    _check(_lib.stb_pack_size(n, m, N, C.byref(out)), "stb_pack_size")
+    return out.value
+
+
+@dataclass
+class PackedLayer:
+    """A packed layer: the device buffer and the three integers every call needs."""
+    n: int
+    m: int
+    N: int
+    buf: "object"        # torch.uint8 CUDA tensor
+    dev_status: "object"  # torch.int32[1] CUDA tensor
+
+    def info(self, stream=None) -> dict:
+        inf = _Info()
+        _check(_lib.stb_packed_info(_ptr(self.buf), C.byref(inf), _stream(stream)), "stb_packed_info")
+        return {"n": inf.n, "m": inf.m, "N": inf.N, "status": inf.status,
+                "used_bytes": inf.used_bytes, "stream_bytes": inf.stream_bytes}
+
+
+def pack(n, m, N, keep, sign, region, sign2, salient, scale, stream=None, buf=None) -> PackedLayer:
+    """stb_pack: logical CUDA tensors (uint8/uint8/int16-as-u16/int32-as-u32/int64-as-u64/
+    int16-as-fp16-bits, C-contiguous) -> PackedLayer."""
+    import torch
+    dev = keep.device
+    for t in (keep, sign, region, sign2, salient, scale):
+        assert t.is_cuda and t.is_contiguous()
+    if buf is None:
+        buf = torch.empty(pack_size(n, m, N), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    L = _Logical(n, m, N, keep.data_ptr(), sign.data_ptr(), region.data_ptr(), sign2.data_ptr(),
+                 salient.data_ptr(), scale.data_ptr())
+    _check(_lib.stb_pack(C.byref(L), _ptr(buf), buf.numel(), _ptr(status), _stream(stream)), "stb_pack")
+    return PackedLayer(n, m, N, buf, status)
+
+
+def pack_numpy(d: dict, device="cuda", stream=None) -> PackedLayer:
+    """Convenience: upload a logical layer given as numpy arrays (the dict of
+    stb_inputs.logical_layer or the fields of an oracle.Logical) and pack it."""
+    import numpy as np
+    import torch
+    def up(a, view):
+        return torch.from_numpy(np.ascontiguousarray(a).view(view)).to(device)
+    return pack(int(d["n"]), int(d["m"]), int(d["N"]), up(d["keep"], np.uint8), up(d["sign"], np.uint8),
+                up(d["region"], np.int16), up(d["sign2"], np.int32), up(d["salient"], np.int64),
+                up(d["scale"], np.int16), stream=stream)
+
+
+def dequant(layer: PackedLayer, dtype=None, out=None, stream=None):
+    import torch
+    dtype = dtype or torch.float32
+    dt = {torch.float32: STB_F32, torch.float16: STB_F16, torch.bfloat16: STB_BF16}[dtype]
+    if out is None:
+        out = torch.empty((layer.n, layer.m), dtype=dtype, device=layer.buf.device)
+    assert out.dtype == dtype and out.stride(1) == 1
+    _check(_lib.stb_dequant(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(out), dt, out.stride(0),
+                            _stream(stream)), "stb_dequant")
+    return out
+
+
+def gemv(layer: PackedLayer, x, out=None, out_dtype=None, stream=None):
+    """stb_gemv: x fp16 [batch][m] (or [m]) -> y [batch][n] fp32 (or fp16)."""
+    import torch
+    x2 = x if x.dim() == 2 else x.unsqueeze(0)
+    assert x2.dtype == torch.float16 and x2.is_cuda and x2.stride(1) == 1
+    batch = x2.shape[0]
+    if out is None:
+        out = torch.empty((batch, layer.n), dtype=out_dtype or torch.float32, device=x.device)
+    ydt = {torch.float32: STB_F32, torch.float16: STB_F16}[out.dtype]
+    _check(_lib.stb_gemv(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(x2), batch, x2.stride(0),
+                         _ptr(out), ydt, out.stride(0), _ptr(layer.dev_status), _stream(stream)), "stb_gemv")
+    return out if x.dim() == 2 else out[0]
+
+
+def gemm_workspace(n, m, N, T) -> int:
+    out = C.c_size_t()
+    _check(_lib.stb_gemm_workspace(n, m, N, T, C.byref(out)), "stb_gemm_workspace")
+    return out.value
+
+
+def gemm(layer: PackedLayer, X, out=None, out_dtype=None, ws=None, stream=None):
+    """stb_gemm: X bf16 [T][m] -> Y [T][n] fp32 (or bf16)."""
+    import torch
+    assert X.dtype == torch.bfloat16 and X.is_cuda and X.dim() == 2 and X.stride(1) == 1
+    T = X.shape[0]
+    if out is None:
+        out = torch.empty((T, layer.n), dtype=out_dtype or torch.float32, device=X.device)
+    ydt = {torch.float32: STB_F32, torch.bfloat16: STB_BF16}[out.dtype]
+    need = gemm_workspace(layer.n, layer.m, layer.N, T)
+    if need and (ws is None or ws.numel() * ws.element_size() < need):
+        ws = torch.empty(need, dtype=torch.uint8, device=X.device)
+    _check(_lib.stb_gemm(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(X), T, X.stride(0), _ptr(out),
+                         ydt, out.stride(0), _ptr(ws), (ws.numel() * ws.element_size()) if ws is not None else 0,
+                         _ptr(layer.dev_status), _stream(stream)), "stb_gemm")
+    return out
+
+
+def make_steps(steps):
+    """Marshal a list of (layer, x, out) into the C array stb_layer_stack takes."""
+    import torch
+    arr = (_Step * len(steps))()
+    for k, (layer, x, out) in enumerate(steps):
+        x2 = x if x.dim() == 2 else x.unsqueeze(0)
+        o2 = out if out.dim() == 2 else out.unsqueeze(0)
+        assert x2.dtype == torch.float16 and x2.stride(1) == 1 and o2.stride(1) == 1
+        odt = {torch.float32: STB_F32, torch.float16: STB_F16}[o2.dtype]
+        arr[k] = _Step(layer.buf.data_ptr(), layer.n, layer.m, layer.N, x2.data_ptr(), o2.data_ptr(), odt,
+                       x2.shape[0], x2.stride(0), o2.stride(0))
+    return arr
+
+
+def layer_stack(steps, dev_status=None, stream=None, marshalled=None):
+    """stb_layer_stack over a list of (PackedLayer, x, out) triples (or a pre-marshalled array)."""
+    arr = marshalled if marshalled is not None else make_steps(steps)
+    _check(_lib.stb_layer_stack(arr, len(arr), _ptr(dev_status), _stream(stream)), "stb_layer_stack")

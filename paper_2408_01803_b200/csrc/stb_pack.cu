@@ -1,0 +1,263 @@
+// stb_pack: fused pack / transpose of a logical N:8 structured-binary layer into the
+// tile-major streaming layout (stb_layout.cuh), plus the small host-side entry points that
+// need no kernel of their own.  Counterpart of the paper's "matrix compression" and "value
+// compression" steps (Appendix C), generalised to an 8-bit keep mask, N sign bits and 2N region
+// bits per group, five scales per row-block and the residual sign bits of salient columns.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/stb.h"
+#include "stb_layout.cuh"
+
+namespace stb {
+
+// ---------------------------------------------------------------------------------------
+// Header + per-block table.  One CTA; thread 0 does the (short) prefix sum over blocks.
+__global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ salient,
+                              uint8_t* __restrict__ packed, int* dev_status) {
+  const int nblk = m / kBlock;
+  Header* hdr = reinterpret_cast<Header*>(packed);
+  BlockInfo* bi = reinterpret_cast<BlockInfo*>(packed + sizeof(Header));
+  __shared__ int bad;
+  if (threadIdx.x == 0) bad = 0;
+  __syncthreads();
+  for (int b = threadIdx.x; b < nblk; b += blockDim.x) {
+    uint64_t lo = salient[2 * b], hi = salient[2 * b + 1];
+    int ns = __popcll(lo) + __popcll(hi);
+    if (ns > kMaxSalient) { bad = 1; ns = kMaxSalient; }
+    bi[b].salient[0] = lo;
+    bi[b].salient[1] = hi;
+    bi[b].nsal = (uint32_t)ns;
+    bi[b].res_bytes = (uint32_t)((ns + 7) / 8);
+    bi[b].tile_bytes = tile_bytes(N, (ns + 7) / 8);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t off = 0, mx = 0;
+    for (int b = 0; b < nblk; ++b) {
+      bi[b].tile_off = off;
+      off += bi[b].tile_bytes;
+      mx = bi[b].tile_bytes > mx ? bi[b].tile_bytes : mx;
+    }
+    const int ntile = (n + kTileRows - 1) / kTileRows;
+    hdr->magic = kMagic;
+    hdr->version = 1;
+    hdr->n = n; hdr->m = m; hdr->N = N;
+    hdr->nblk = nblk;
+    hdr->ntile = ntile;
+    hdr->tiles_offset = tiles_offset(nblk);
+    hdr->rt_stride = off;
+    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + (uint64_t)off * (uint64_t)ntile;
+    hdr->status = bad ? (uint32_t)STB_ERR_CORRUPT : 0u;
+    hdr->max_tile_bytes = mx;
+    hdr->pad[0] = hdr->pad[1] = 0;
+    if (bad && dev_status) *dev_status = STB_ERR_CORRUPT;
+  }
+}
+
+template <int NW>
+__device__ __forceinline__ void store_planes(uint8_t* tile, uint32_t base, const uint32_t* w,
+                                             int lane) {
+  constexpr int Q4 = NW / 4;
+#pragma unroll
+  for (int q = 0; q < Q4; ++q)
+    *reinterpret_cast<uint4*>(tile + base + q * 512 + lane * 16) =
+        make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+  uint32_t o = base + Q4 * 512;
+  if (NW & 2) {
+    *reinterpret_cast<uint2*>(tile + o + lane * 8) = make_uint2(w[4 * Q4], w[4 * Q4 + 1]);
+    o += 256;
+  }
+  if (NW & 1) *reinterpret_cast<uint32_t*>(tile + o + lane * 4) = w[NW - 1];
+}
+
+// One warp per tile (32 rows x one block); lane = row.  Adjacent warps take adjacent blocks
+// of the same rows, so the 16- and 32-byte pieces each lane reads share sectors with its
+// neighbours in L2.
+template <int N>
+__global__ void __launch_bounds__(256)
+pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
+  const int nblk = L.m / kBlock, ngrp = L.m / kGroup;
+  const int ntile = (L.n + kTileRows - 1) / kTileRows;
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (warp >= (long long)ntile * nblk) return;
+  const int rt = (int)(warp / nblk), b = (int)(warp % nblk);
+  const int row = rt * kTileRows + lane;
+  const bool valid = row < L.n;
+
+  Header* hdr = reinterpret_cast<Header*>(packed);
+  const BlockInfo* bi = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header)) + b;
+  const uint64_t sal_lo = bi->salient[0], sal_hi = bi->salient[1];
+  const int nsal = (int)bi->nsal, rb = (int)bi->res_bytes;
+  uint8_t* tile = packed + tiles_offset(nblk) + (size_t)rt * (size_t)hdr->rt_stride + bi->tile_off;
+
+  uint32_t keepw[4] = {0, 0, 0, 0}, signw[4] = {0, 0, 0, 0}, regw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  uint32_t s2 = 0;
+  uint16_t sc[5] = {0, 0, 0, 0, 0};
+  if (valid) {
+    const size_t gofs = (size_t)row * ngrp + (size_t)b * 16;
+    uint4 k4 = *reinterpret_cast<const uint4*>(L.keep + gofs);
+    uint4 s4 = *reinterpret_cast<const uint4*>(L.sign + gofs);
+    const uint4* rp = reinterpret_cast<const uint4*>(L.region + gofs);
+    uint4 r0 = rp[0], r1 = rp[1];
+    keepw[0] = k4.x; keepw[1] = k4.y; keepw[2] = k4.z; keepw[3] = k4.w;
+    signw[0] = s4.x; signw[1] = s4.y; signw[2] = s4.z; signw[3] = s4.w;
+    regw[0] = r0.x; regw[1] = r0.y; regw[2] = r0.z; regw[3] = r0.w;
+    regw[4] = r1.x; regw[5] = r1.y; regw[6] = r1.z; regw[7] = r1.w;
+    s2 = L.sign2[(size_t)row * nblk + b];
+    const uint16_t* sp = L.scale + ((size_t)row * nblk + b) * 5;
+#pragma unroll
+    for (int q = 0; q < 5; ++q) sc[q] = sp[q];
+  }
+
+  bool bad = false;
+  uint32_t R[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // region words (N used)
+  uint32_t S[4] = {0, 0, 0, 0};               // sign words ((N+1)/2 used, last is the half for odd N)
+#pragma unroll
+  for (int g = 0; g < 16; ++g) {
+    const uint32_t kb = (keepw[g >> 2] >> (8 * (g & 3))) & 0xFFu;
+    const uint32_t sb = (signw[g >> 2] >> (8 * (g & 3))) & 0xFFu;
+    const uint32_t rg = (regw[g >> 1] >> (16 * (g & 1))) & 0xFFFFu;
+    const uint32_t salb = (uint32_t)(((g < 8 ? sal_lo : sal_hi) >> (8 * (g & 7))) & 0xFFull);
+    if (valid) {
+      if (__popc(kb) != N) bad = true;
+      if (N < 8 && ((sb >> N) != 0 || (rg >> (2 * N)) != 0)) bad = true;
+    }
+    uint32_t c3 = 0;
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+      const int w = g * N + k;
+      const uint32_t code = (rg >> (2 * k)) & 3u;
+      const uint32_t neg = ((sb >> k) & 1u) ^ 1u;
+      R[w >> 4] |= code << code_bit(w);
+      S[w >> 5] |= (valid ? neg : 0u) << sign_bit(w);
+      c3 |= (code == 3u ? 1u : 0u) << k;
+    }
+    // region 3 must mark exactly the kept weights of salient columns
+    uint32_t expect = 0, t = kb & salb;
+    while (t) {
+      const int c = __ffs(t) - 1;
+      t &= t - 1;
+      expect |= 1u << __popc(kb & ((1u << c) - 1u));
+    }
+    if (valid && c3 != expect) bad = true;
+  }
+  // residual sign bits: none beyond S_b, none on a dropped weight
+  if (valid) {
+    if (nsal < 32 && (s2 >> nsal) != 0) bad = true;
+    int t = 0;
+#pragma unroll 1
+    for (int half = 0; half < 2; ++half) {
+      uint64_t mk = half ? sal_hi : sal_lo;
+      while (mk) {
+        const int c = __ffsll((long long)mk) - 1 + 64 * half;
+        mk &= mk - 1;
+        const uint32_t kbit = (keepw[c >> 5] >> (c & 31)) & 1u;
+        if (!kbit && ((s2 >> t) & 1u)) bad = true;
+        ++t;
+      }
+    }
+  }
+
+  // ---- write the tile, plane by plane (coalesced vector stores) ----
+  *reinterpret_cast<uint4*>(tile + lane * 16) = make_uint4(keepw[0], keepw[1], keepw[2], keepw[3]);
+  store_planes<N>(tile, off_region(N), R, lane);
+  store_planes<N / 2>(tile, off_sign(N), S, lane);
+  if (N & 1) {
+    const uint32_t h = S[N / 2];
+    const uint32_t up = __shfl_down_sync(0xFFFFFFFFu, half_to_upper(h), 16);
+    if (lane < 16) *reinterpret_cast<uint32_t*>(tile + sign_half_off(N, lane)) = h | up;
+  }
+  const uint32_t A = (sc[0] & 0xFFu) | ((sc[1] & 0xFFu) << 8) | ((sc[2] & 0xFFu) << 16) | ((uint32_t)(sc[3] & 0xFFu) << 24);
+  const uint32_t B = (sc[0] >> 8) | ((uint32_t)(sc[1] >> 8) << 8) | ((uint32_t)(sc[2] >> 8) << 16) | ((uint32_t)(sc[3] >> 8) << 24);
+  *reinterpret_cast<uint2*>(tile + off_scale(N) + lane * 8) = make_uint2(A, B);
+  *reinterpret_cast<uint16_t*>(tile + off_sal2(N) + lane * 2) = sc[4];
+  for (int p = 0; p < rb; ++p) tile[off_resid(N) + p * 32 + lane] = (uint8_t)(s2 >> (8 * p));
+
+  if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) {
+    hdr->status = (uint32_t)STB_ERR_CORRUPT;
+    if (dev_status) *dev_status = STB_ERR_CORRUPT;
+  }
+}
+
+template <int N>
+static cudaError_t launch_pack(const stb_logical& L, uint8_t* packed, int* dev_status,
+                               cudaStream_t s) {
+  const long long tiles = (long long)((L.n + kTileRows - 1) / kTileRows) * (L.m / kBlock);
+  const unsigned grid = (unsigned)((tiles + 7) / 8);
+  pack_kernel<N><<<grid, 256, 0, s>>>(L, packed, dev_status);
+  return cudaGetLastError();
+}
+
+}  // namespace stb
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+extern "C" int stb_pack_size(int n, int m, int N, size_t* bytes) {
+  if (!bytes) return STB_ERR_ARG;
+  if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
+  if (N < 1 || N > 8) return STB_ERR_NM;
+  const size_t nblk = (size_t)m / stb::kBlock, ntile = ((size_t)n + 31) / 32;
+  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * (size_t)stb::tile_bytes(N, 4);
+  return STB_OK;
+}
+
+extern "C" int stb_pack(const stb_logical* L, void* packed, size_t packed_bytes, int* dev_status,
+                        void* stream) {
+  if (!L || !packed) return STB_ERR_ARG;
+  size_t need = 0;
+  int rc = stb_pack_size(L->n, L->m, L->N, &need);
+  if (rc != STB_OK) return rc;
+  if (!L->keep || !L->sign || !L->region || !L->sign2 || !L->salient || !L->scale) return STB_ERR_ARG;
+  if (!aligned16(L->keep) || !aligned16(L->sign) || !aligned16(L->region) || !aligned16(L->salient) ||
+      (reinterpret_cast<uintptr_t>(L->sign2) & 3u) || (reinterpret_cast<uintptr_t>(L->scale) & 1u) ||
+      (reinterpret_cast<uintptr_t>(packed) & 255u))
+    return STB_ERR_ARG;
+  if (packed_bytes < need) return STB_ERR_SIZE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* out = static_cast<uint8_t*>(packed);
+  stb::header_kernel<<<1, 256, 0, s>>>(L->n, L->m, L->N, L->salient, out, dev_status);
+  if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
+  cudaError_t e = cudaSuccess;
+  switch (L->N) {
+    case 1: e = stb::launch_pack<1>(*L, out, dev_status, s); break;
+    case 2: e = stb::launch_pack<2>(*L, out, dev_status, s); break;
+    case 3: e = stb::launch_pack<3>(*L, out, dev_status, s); break;
+    case 4: e = stb::launch_pack<4>(*L, out, dev_status, s); break;
+    case 5: e = stb::launch_pack<5>(*L, out, dev_status, s); break;
+    case 6: e = stb::launch_pack<6>(*L, out, dev_status, s); break;
+    case 7: e = stb::launch_pack<7>(*L, out, dev_status, s); break;
+    case 8: e = stb::launch_pack<8>(*L, out, dev_status, s); break;
+  }
+  return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
+}
+
+extern "C" int stb_packed_info(const void* packed, stb_info* info, void* stream) {
+  if (!packed || !info) return STB_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  stb::Header h;
+  if (cudaMemcpyAsync(&h, packed, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return STB_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return STB_ERR_CUDA;
+  if (h.magic != stb::kMagic) return STB_ERR_CORRUPT;
+  info->n = h.n; info->m = h.m; info->N = h.N;
+  info->status = (int)h.status;
+  info->used_bytes = h.used_bytes;
+  info->stream_bytes = h.rt_stride * (uint64_t)h.ntile;
+  return STB_OK;
+}
+
+extern "C" const char* stb_status_str(int status) {
+  switch (status) {
+    case STB_OK: return "ok";
+    case STB_ERR_ARG: return "bad argument";
+    case STB_ERR_SHAPE: return "bad shape (need n >= 1, m a positive multiple of 128)";
+    case STB_ERR_NM: return "N outside 1..8";
+    case STB_ERR_SIZE: return "buffer too small or batch out of range";
+    case STB_ERR_UNSUPPORTED: return "unsupported dtype or mode";
+    case STB_ERR_CORRUPT: return "logical layer or packed header failed validation";
+    case STB_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case STB_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}

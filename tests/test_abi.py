@@ -1,0 +1,67 @@
+"""The C-ABI library loads on a machine without a GPU, exports every symbol that include/stb.h
+declares, and rejects bad arguments on the host before any CUDA call."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def stb():
+    from paper_2408_01803_b200 import build
+    build.build()
+    import paper_2408_01803_b200 as stb
+    return stb
+
+
+def test_every_declared_symbol_is_exported(stb):
+    hdr = open(os.path.join(ROOT, "include", "stb.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(stb_[a-z_0-9]+)\s*\(", hdr))
+    assert {"stb_pack", "stb_gemv", "stb_gemm", "stb_layer_stack", "stb_pack_size", "stb_dequant"} <= names
+    lib = C.CDLL(stb.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert names == set(stb.EXPORTS)
+
+
+def test_pack_size_formula_and_errors(stb):
+    # 50 / 56 / 62 bytes per row-block at 4:8 / 5:8 / 6:8 plus at most 4 residual bytes
+    for N, per in ((4, 50), (5, 56), (6, 62)):
+        n, m = 4096, 4096
+        hdr = (64 + 32 * (m // 128) + 255) // 256 * 256
+        assert stb.pack_size(n, m, N) == hdr + (n // 32) * (m // 128) * 32 * (per + 4)
+    assert stb.pack_size(33, 128, 4) == 256 + 2 * 32 * 54      # ragged rows pad to a tile of 32
+    for args, code in (((0, 128, 4), stb.STB_ERR_SHAPE), ((8, 100, 4), stb.STB_ERR_SHAPE),
+                       ((8, 0, 4), stb.STB_ERR_SHAPE), ((8, 128, 0), stb.STB_ERR_NM), ((8, 128, 9), stb.STB_ERR_NM)):
+        with pytest.raises(stb.StbError) as e:
+            stb.pack_size(*args)
+        assert e.value.status == code
+
+
+def test_host_side_argument_checks_launch_nothing(stb):
+    lib = stb._lib
+    null = C.c_void_p(0)
+    one = C.c_void_p(256)          # never dereferenced: every call below fails validation first
+    assert lib.stb_pack(None, one, 1 << 20, null, null) == stb.STB_ERR_ARG
+    L = stb._Logical(32, 128, 4, 256, 256, 256, 256, 256, 256)
+    assert lib.stb_pack(C.byref(L), null, 1 << 20, null, null) == stb.STB_ERR_ARG
+    assert lib.stb_pack(C.byref(L), one, 16, null, null) == stb.STB_ERR_SIZE
+    L.N = 9
+    assert lib.stb_pack(C.byref(L), one, 1 << 20, null, null) == stb.STB_ERR_NM
+    L.N = 4; L.m = 130
+    assert lib.stb_pack(C.byref(L), one, 1 << 20, null, null) == stb.STB_ERR_SHAPE
+    L.m = 128; L.keep = 257
+    assert lib.stb_pack(C.byref(L), one, 1 << 20, null, null) == stb.STB_ERR_ARG      # misaligned
+    assert lib.stb_gemv(null, 32, 128, 4, one, 1, 128, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_ARG
+    assert lib.stb_gemv(one, 32, 128, 4, one, 0, 128, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_SIZE
+    assert lib.stb_gemv(one, 32, 128, 4, one, 17, 128, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_SIZE
+    assert lib.stb_gemv(one, 32, 128, 4, one, 1, 64, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_ARG
+    assert lib.stb_gemv(one, 32, 128, 4, one, 1, 128, one, stb.STB_BF16, 32, null, null) == stb.STB_ERR_UNSUPPORTED
+    assert lib.stb_dequant(one, 32, 128, 4, one, 7, 128, null) == stb.STB_ERR_UNSUPPORTED
+    assert lib.stb_dequant(one, 32, 128, 4, one, stb.STB_F32, 64, null) == stb.STB_ERR_ARG
+    assert lib.stb_layer_stack(None, 1, null, null) == stb.STB_ERR_ARG
+    assert stb.status_str(stb.STB_ERR_TIMEOUT).startswith("a bounded")

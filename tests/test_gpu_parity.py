@@ -1,0 +1,170 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+  * stb_pack + stb_dequant: fp32 decode bit-exact against the oracle's decode (-0 == +0).
+  * stb_gemv: max|y_gpu - y_ref| <= 5e-3 * max|y_ref| against the float64
+    dequantise-then-matmul of the oracle.
+"""
+import numpy as np
+import pytest
+
+import oracle
+import stb_inputs as si
+
+pytestmark = pytest.mark.gpu
+TOL = 5e-3
+
+
+@pytest.fixture(scope="module")
+def stb():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2408_01803_b200 as stb
+    return stb
+
+
+def _fields(L):
+    return {"n": L.n, "m": L.m, "N": L.N, "keep": L.keep, "sign": L.sign, "region": L.region,
+            "sign2": L.sign2, "salient": L.salient, "scale": L.scale}
+
+
+def _quantized(n, m, N, seed):
+    W = si.dense_weight(n, m, seed).astype(np.float64)
+    L, _, _ = oracle.quantize(W, si.calib_norms(m, seed), N)
+    return L
+
+
+def _check_gemv(stb, layer, What, m, batch, seed, out_dtype=None):
+    import torch
+    x = si.activations(batch, m, seed)
+    y_ref = oracle.matmul(What, x.astype(np.float64))
+    xd = torch.from_numpy(x).cuda()
+    y = stb.gemv(layer, xd, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    assert int(layer.dev_status.item()) == 0
+    err = np.abs(y.double().cpu().numpy() - y_ref).max()
+    tol = TOL * np.abs(y_ref).max()
+    if out_dtype is not None:
+        tol += 2.0 ** -11 * np.abs(y_ref).max()      # one fp16 rounding of the result
+    assert err <= tol, (err, tol)
+    return err / np.abs(y_ref).max()
+
+
+@pytest.mark.parametrize("N", [1, 2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("n,m", [(40, 256), (100, 384)])
+def test_quantized_layer_dequant_bit_exact_and_gemv(stb, N, n, m):
+    import torch
+    L = _quantized(n, m, N, 1000 + 10 * N + n)
+    What = oracle.decode(L)
+    layer = stb.pack_numpy(_fields(L))
+    info = layer.info()
+    assert info["status"] == 0 and (info["n"], info["m"], info["N"]) == (n, m, N)
+    assert int(layer.dev_status.item()) == 0
+    got = stb.dequant(layer).cpu().numpy()
+    assert np.array_equal(got, What)                       # bit-exact values (-0 == +0)
+    for dt in (torch.float16, torch.bfloat16):
+        g16 = stb.dequant(layer, dtype=dt).float().cpu().numpy()
+        want = torch.from_numpy(What).to(dt).float().numpy()
+        assert np.array_equal(g16, want)
+    for batch in (1, 3, 4, 7, 16):
+        _check_gemv(stb, layer, What, m, batch, 7 + batch)
+    _check_gemv(stb, layer, What, m, 2, 99, out_dtype=torch.float16)
+
+
+@pytest.mark.parametrize("N,n,m", [(4, 4096, 4096), (6, 11008, 4096), (6, 4096, 11008), (5, 5120, 5120),
+                                   (5, 5120, 13824)])
+def test_full_size_layers_sampled_rows(stb, N, n, m):
+    """Full workload shapes with directly drawn logical layers: sampled output rows against the
+    oracle's decode-and-multiply, plus sampled rows of the dequantised matrix bit for bit."""
+    import torch
+    d = si.logical_layer(n, m, N, si.seed_for(2, N))
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    info = layer.info()
+    assert info["status"] == 0
+    nres = sum(-(-bin(int(a) | (int(b) << 64)).count("1") // 8) for a, b in d["salient"])
+    per = {4: 50, 5: 56, 6: 62}[N]
+    assert info["stream_bytes"] == (n // 32) * 32 * (per * (m // 128) + nres)
+    g = np.random.default_rng(N)
+    rows = np.sort(g.choice(n, size=192, replace=False)).astype(np.int32)
+    rows[:4] = [0, 1, n - 2, n - 1]
+    rows = np.unique(rows)
+    for batch in (1, 4, 16):
+        x = si.activations(batch, m, si.seed_for(2, 8 + batch))
+        y_ref = oracle.layer_rows(L, rows, x.astype(np.float64))
+        y = stb.gemv(layer, torch.from_numpy(x).cuda())
+        torch.cuda.synchronize()
+        assert int(layer.dev_status.item()) == 0
+        yg = y.double().cpu().numpy()[:, rows]
+        assert np.abs(yg - y_ref).max() <= TOL * np.abs(y_ref).max()
+    Wg = stb.dequant(layer)
+    sub = oracle.Logical(len(rows), m, N, d["keep"][rows].copy(), d["sign"][rows].copy(), d["region"][rows].copy(),
+                         d["sign2"][rows].copy(), d["salient"], d["scale"][rows].copy())
+    assert np.array_equal(Wg[torch.from_numpy(rows.astype(np.int64)).cuda()].cpu().numpy(), oracle.decode(sub))
+
+
+def test_pack_flags_corrupt_layers(stb):
+    import torch
+    base = si.logical_layer(64, 256, 4, 5)
+    def status_of(d):
+        layer = stb.pack_numpy(d)
+        torch.cuda.synchronize()
+        return int(layer.dev_status.item()), layer.info()["status"]
+    assert status_of(base) == (0, 0)
+    d = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in base.items()}
+    d["keep"][3, 5] = 0b00000111                      # three bits instead of four
+    assert status_of(d) == (stb.STB_ERR_CORRUPT, stb.STB_ERR_CORRUPT)
+    d = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in base.items()}
+    d["sign"][0, 0] |= 0x10                           # sign bit beyond N
+    assert status_of(d)[0] == stb.STB_ERR_CORRUPT
+    d = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in base.items()}
+    d["salient"][1, 0] = np.uint64(0xFFFFFFFFFF)      # 40 salient columns in one block
+    assert status_of(d)[0] == stb.STB_ERR_CORRUPT
+    d = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in base.items()}
+    d["salient"][:] = 0                               # region 3 without a salient column
+    assert status_of(d)[0] == stb.STB_ERR_CORRUPT
+    # a layer packed for one shape must not be run as another: the kernel refuses and reports
+    layer = stb.pack_numpy(base)
+    wrong = stb.PackedLayer(64, 256, 5, layer.buf, layer.dev_status)
+    y = torch.zeros(1, 64, device="cuda")
+    stb.gemv(wrong, torch.zeros(1, 256, dtype=torch.float16, device="cuda"), out=y)
+    torch.cuda.synchronize()
+    assert int(layer.dev_status.item()) == stb.STB_ERR_CORRUPT
+
+
+def test_degenerate_layers(stb):
+    """No salient column at all, all weights kept (N = 8), a single tile with one row."""
+    import torch
+    d = si.logical_layer(1, 128, 8, 3, max_salient=0)
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    assert np.array_equal(stb.dequant(layer).cpu().numpy(), oracle.decode(L))
+    _check_gemv(stb, layer, oracle.decode(L), 128, 1, 4)
+    d = si.logical_layer(33, 128, 3, 4, max_salient=0)
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    assert layer.info()["stream_bytes"] == 2 * 32 * (16 + 6 + 12 + 10)
+    assert np.array_equal(stb.dequant(layer).cpu().numpy(), oracle.decode(L))
+    _check_gemv(stb, layer, oracle.decode(L), 128, 16, 5)
+
+
+def test_layer_stack_chains_layers_with_per_layer_N(stb):
+    import torch
+    shapes = [(256, 384, 4), (128, 256, 6), (96, 128, 5)]          # (n, m, N): m of a layer = n of the previous
+    layers, Ws = [], []
+    for k, (n, m, N) in enumerate(shapes):
+        d = si.logical_layer(n, m, N, 60 + k)
+        layers.append(stb.pack_numpy(d)); Ws.append(oracle.decode(oracle.Logical(**d)))
+    x0 = si.activations(2, 384, 61)
+    bufs = [torch.from_numpy(x0).cuda(), torch.empty(2, 256, dtype=torch.float16, device="cuda"),
+            torch.empty(2, 128, dtype=torch.float16, device="cuda"), torch.empty(2, 96, dtype=torch.float32, device="cuda")]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stb.layer_stack([(layers[k], bufs[k], bufs[k + 1]) for k in range(3)], dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    # parity per layer: the oracle is fed the same (GPU-produced, fp16-rounded) input
+    for k in range(3):
+        xin = bufs[k].double().cpu().numpy()
+        y_ref = oracle.matmul(Ws[k], xin)
+        got = bufs[k + 1].double().cpu().numpy()
+        tol = TOL * np.abs(y_ref).max() + (2.0 ** -11 * np.abs(y_ref).max() if k < 2 else 0)
+        assert np.abs(got - y_ref).max() <= tol
