@@ -2,8 +2,10 @@
 
 Argument marshalling only: every step of the path (pack, dequant, GEMV, GEMM, layer stack)
 runs in the CUDA kernels behind the C ABI declared in include/stb.h.  torch is used for
-device memory and streams.  There is no CPU fallback: if the shared library is missing the
-import of this package raises.
+device memory and streams.  There is no CPU fallback: the shared library is loaded on the
+first call of any function here, and a missing library raises ImportError at that point
+(`python -m paper_2408_01803_b200.build` compiles it; importing the package alone must work
+without it so that the build module can be reached).
 """
 from __future__ import annotations
 
@@ -67,7 +69,17 @@ def _load():
     return lib
 
 
-_lib = _load()
+class _LazyLib:
+    """Loads libstb.so on first attribute access; raises ImportError if it is not built."""
+    _real = None
+
+    def __getattr__(self, name):
+        if _LazyLib._real is None:
+            _LazyLib._real = _load()
+        return getattr(_LazyLib._real, name)
+
+
+_lib = _LazyLib()
 
 
 def status_str(status: int) -> str:
