@@ -1,0 +1,449 @@
+#!/usr/bin/env python
+"""Benchmark of the N:M structured-binary linear layer on B200.
+
+One step = one decode pass (batch 1) over the three MLP linears of a LLaMA-2-7B decoder layer at
+6:8: gate 11008x4096 and up 11008x4096 read the same fp16 input, down 4096x11008 reads gate's
+fp16 output; the three GEMVs are queued by stb_layer_stack on one stream.  The headline value is
+the effective HBM bandwidth: bytes of packed weights streamed per second.  Weights are resident
+in HBM; every step reads another copy of the packed layers so that no byte comes from L2.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]          CUDA path, one JSON line
+  python bench.py --impl reference ...                         the CPU oracle on the host cores
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent
+replica of the same workload: the layer is not sharded, there is no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import stb_inputs as si
+
+METRIC = "gemv_packed_weight_bandwidth"
+UNIT = "GB/s"
+WORKLOAD = "llama2-7b-mlp gate/up 11008x4096 + down 4096x11008, 6:8, block 128, batch-1 decode GEMV"
+MLP = [("gate", 11008, 4096), ("up", 11008, 4096), ("down", 4096, 11008)]
+MLP_N = 6
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def mlp_logical(k: int) -> dict:
+    name, n, m = MLP[k]
+    return si.logical_layer(n, m, MLP_N, si.seed_for(2, k))
+
+
+# ------------------------------------------------------------------------------------------
+# clocks: NVML polled from a thread while the timed region runs (read-only queries)
+class ClockSampler:
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+               0x10: "sync_boost"}
+
+    def __init__(self, torch_device_index: int):
+        self.samples, self.h, self.nv, self._stop, self._thr = [], None, None, threading.Event(), None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # noqa: BLE001
+            self.err = repr(e)
+
+    def sample(self):
+        if self.h is None:
+            return
+        nv = self.nv
+        try:
+            mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            try:
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+            except Exception:
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            self.samples.append((time.perf_counter(), mhz, mask))
+        except Exception:
+            pass
+
+    def start(self, period=0.01):
+        def loop():
+            while not self._stop.is_set():
+                self.sample()
+                time.sleep(period)
+        self._thr = threading.Thread(target=loop, daemon=True)
+        self._thr.start()
+
+    def stop(self, t0, t1):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+        if self.h is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable: " + getattr(self, "err", "")}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples[-1:]
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        reasons = sorted(v for k, v in self.REASONS.items() if mask & k)
+        return {"sm_mhz": float(np.median([s[1] for s in inside])) if inside else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(inside)}
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_pass(Ls, xs, rows, threads=0):
+    """One decode pass of the oracle over the listed output rows of each layer (fp32 decode from
+    the logical arrays + float64 multiply-accumulate).  Returns seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    for L, x, r in zip(Ls, xs, rows):
+        oracle.layer_rows(L, r, x, nthreads=threads)
+    return time.perf_counter() - t0
+
+
+def stream_bytes_of(d: dict) -> int:
+    """Bytes one GEMV pass streams for a logical layer: 16 + 6N + 10 bytes per row and block plus
+    one residual byte per row and block for every started group of 8 salient columns; rows are
+    padded to tiles of 32."""
+    n, m, N = d["n"], d["m"], d["N"]
+    nres = sum(-(-bin(int(a) | (int(b) << 64)).count("1") // 8) for a, b in d["salient"])
+    return -(-n // 32) * 32 * ((26 + 6 * N) * (m // 128) + nres)
+
+
+def reference_arm(args):
+    """The CPU oracle, as it stands, on the host cores: same workload, metric and unit.  Each step
+    is a bounded sample of output rows so that the run ends within minutes."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    ds = [mlp_logical(k) for k in range(3)]
+    Ls = [oracle.Logical(**d) for d in ds]
+    x0 = si.activations(1, 4096, si.seed_for(2, 8)).astype(np.float64)
+    x1 = si.activations(1, 11008, si.seed_for(2, 9)).astype(np.float64)     # stands in for gate's output
+    xs = [x0, x0, x1]
+    cores = oracle.hardware_threads()
+    # calibrate the row rate on a small sample, then size a step for ~60 s over all steps
+    probe = [np.arange(0, d["n"], 16, dtype=np.int32) for d in ds]
+    tp = oracle_pass(Ls, xs, probe)
+    frac_probe = 1.0 / 16
+    budget = 60.0 / max(1, args.steps + args.warmup)
+    frac = min(1.0, frac_probe * budget / max(tp, 1e-6))
+    stride = max(1, int(np.ceil(1.0 / frac)))
+    rows = [np.arange(0, d["n"], stride, dtype=np.int32) for d in ds]
+    bytes_step = sum(stream_bytes_of(d) * len(r) / (-(-d["n"] // 32) * 32) for d, r in zip(ds, rows))
+    for _ in range(args.warmup):
+        oracle_pass(Ls, xs, rows)
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_pass(Ls, xs, rows)
+    val = bytes_step * args.steps / t / 1e9
+    sample = "every %d-th output row of gate, up and down per step (%d rows, %.2f MB of packed weights)" % (
+        stride, sum(len(r) for r in rows), bytes_step / 1e6)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch": 1, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ------------------------------------------------------------------------------------------
+class Workload:
+    """The MLP layers packed on the device, `copies` times each at distinct addresses."""
+
+    def __init__(self, stb, torch, copies):
+        self.stb, self.torch = stb, torch
+        self.logical = [mlp_logical(k) for k in range(3)]
+        self.layers = []          # [copy][k]
+        first = [stb.pack_numpy(d) for d in self.logical]
+        torch.cuda.synchronize()
+        for lay in first:
+            assert int(lay.dev_status.item()) == 0
+        self.infos = [lay.info() for lay in first]
+        for c in range(copies):
+            if c == 0:
+                self.layers.append(first)
+            else:
+                self.layers.append([stb.PackedLayer(l.n, l.m, l.N, l.buf[: self.infos[k]["used_bytes"]].clone(),
+                                                    l.dev_status) for k, l in enumerate(first)])
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.x_np = si.activations(1, 4096, si.seed_for(2, 8))
+        self.x = torch.from_numpy(self.x_np).cuda()
+        self.h_gate = torch.zeros(1, 11008, dtype=torch.float16, device="cuda")
+        self.h_up = torch.zeros(1, 11008, dtype=torch.float16, device="cuda")
+        self.y = torch.zeros(1, 4096, dtype=torch.float32, device="cuda")
+        self.steps = [stb.make_steps([(ls[0], self.x, self.h_gate), (ls[1], self.x, self.h_up),
+                                      (ls[2], self.h_gate, self.y)]) for ls in self.layers]
+        self.bytes_step = sum(i["stream_bytes"] for i in self.infos)
+
+    def step(self, c):
+        self.stb.layer_stack(None, dev_status=self.status, marshalled=self.steps[c % len(self.steps)])
+
+
+def capture(torch, fns):
+    """One CUDA graph that runs every callable of `fns` once, in order."""
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        fns[0]()                           # warm: module load, attribute set-up happen outside capture
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g):
+        for f in fns:
+            f()
+    return g
+
+
+def time_graph(torch, g, calls_per_replay, min_calls=2000, warm=3):
+    """Average microseconds per call of a captured sequence, CUDA events on the replay stream."""
+    reps = max(3, -(-min_calls // calls_per_replay))
+    for _ in range(warm):
+        g.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return 1e3 * e0.elapsed_time(e1) / (reps * calls_per_replay)
+
+
+def gemv_table(stb, torch, wl, pk):
+    """Isolated per-layer GEMV timings, cold L2 (rotating over distinct packed copies), for the
+    decode batches of the workload; plus the other decode shapes and a dense bf16 cuBLAS GEMV
+    (torch.matmul) of the same shape as context."""
+    out = []
+
+    def one(name, copies, n, m, N, sbytes, batches):
+        for b in batches:
+            x = torch.from_numpy(si.activations(b, m, si.seed_for(2, 10 + b))).cuda()
+            y = torch.empty(b, n, dtype=torch.float32, device="cuda")
+            fns = [(lambda lay=lay: stb.gemv(lay, x, out=y)) for lay in copies]
+            g = capture(torch, fns)
+            us = time_graph(torch, g, len(fns))
+            out.append({"layer": name, "n": n, "m": m, "N": N, "batch": b, "us_per_layer": round(us, 3),
+                        "packed_MB": round(sbytes / 1e6, 3), "GBps": round(sbytes / us / 1e3, 1),
+                        "frac_of_measured_hbm": round(sbytes / us / 1e3 / pk["hbm_gbs"], 4)})
+            del g
+
+    ncopy = len(wl.layers)
+    one("gate/up 11008x4096", [wl.layers[c][k] for c in range(ncopy) for k in (0, 1)], 11008, 4096, MLP_N,
+        wl.infos[0]["stream_bytes"], (1, 4, 8, 16))
+    one("down 4096x11008", [wl.layers[c][2] for c in range(ncopy)], 4096, 11008, MLP_N,
+        wl.infos[2]["stream_bytes"], (1, 4, 8, 16))
+    # other decode shapes of the workload list (batch 1): 7B attention at 4:8, 13B block at 5:8
+    for name, n, m, N, item in (("7B q_proj 4096x4096", 4096, 4096, 4, 0), ("13B q 5120x5120", 5120, 5120, 5, 1),
+                                ("13B gate 13824x5120", 13824, 5120, 5, 2), ("13B down 5120x13824", 5120, 13824, 5, 3)):
+        d = si.logical_layer(n, m, N, si.seed_for(3, item))
+        lay = stb.pack_numpy(d)
+        used = lay.info()["used_bytes"]
+        sb = lay.info()["stream_bytes"]
+        k = max(4, min(48, -(-3 * L2_BYTES // sb)))
+        copies = [lay] + [stb.PackedLayer(n, m, N, lay.buf[:used].clone(), lay.dev_status) for _ in range(k - 1)]
+        one(name, copies, n, m, N, sb, (1,))
+        del copies, lay
+        torch.cuda.empty_cache()
+    # dense bf16 context
+    ctx = []
+    for name, n, m in (("gate/up 11008x4096", 11008, 4096), ("down 4096x11008", 4096, 11008)):
+        k = max(2, -(-3 * L2_BYTES // (2 * n * m)))
+        Ws = [torch.randn(n, m, device="cuda", dtype=torch.bfloat16) for _ in range(k)]
+        x = torch.randn(m, 1, device="cuda", dtype=torch.bfloat16)
+        y = torch.empty(n, 1, device="cuda", dtype=torch.bfloat16)
+        g = capture(torch, [(lambda W=W: torch.matmul(W, x, out=y)) for W in Ws])
+        us = time_graph(torch, g, k, min_calls=400)
+        ctx.append({"layer": name, "kind": "dense bf16 torch.matmul (cuBLAS), batch 1", "us_per_layer": round(us, 3),
+                    "dense_MB": round(2 * n * m / 1e6, 2), "GBps": round(2 * n * m / us / 1e3, 1)})
+        del g, Ws
+        torch.cuda.empty_cache()
+    return out, ctx
+
+
+def cuda_arm(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2408_01803_b200 import build
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if rank == 0 or not os.path.exists(os.path.join(ROOT, "paper_2408_01803_b200", "libstb.so")):
+        build.build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    import paper_2408_01803_b200 as stb
+    pk = peaks()
+
+    copies = 12          # 12 x 65.5 MB per rotation: more than 6 x L2
+    wl = Workload(stb, torch, copies)
+    K, W = args.steps, args.warmup
+
+    # graph of `copies` consecutive steps (every step another copy of the weights) + remainder
+    g_full = capture(torch, [(lambda c=c: wl.step(c)) for c in range(copies)])
+    rem = K % copies
+    g_rem = capture(torch, [(lambda c=c: wl.step(c)) for c in range(rem)]) if rem else None
+    for i in range(max(W, 3)):
+        wl.step(i)
+    g_full.replay()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(K // copies):
+        g_full.replay()
+    if g_rem is not None:
+        g_rem.replay()
+    e1.record()
+    sampler.sample()
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    if world > 1:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1)
+    assert int(wl.status.item()) == 0, "device status %d" % int(wl.status.item())
+    if world > 1:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    launches = 3 * K
+    value = world * wl.bytes_step * K / (ms * 1e-3) / 1e9
+    launch_us = 1e3 * ms / launches
+    per_launch_bytes = wl.bytes_step / 3.0
+    achieved = per_launch_bytes / launch_us / 1e3
+
+    # end to end: x from pinned host memory, y back to the host, every step
+    xh = torch.from_numpy(wl.x_np.copy()).pin_memory()
+    yh = torch.empty(1, 4096, dtype=torch.float32).pin_memory()
+    Ke = min(K, 5000)
+    for i in range(5):
+        stb.layer_stack_host(wl.steps[i % copies], xh, yh, dev_status=wl.status)
+        torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    w0 = time.perf_counter()
+    for i in range(Ke):
+        stb.layer_stack_host(wl.steps[i % copies], xh, yh, dev_status=wl.status)
+        torch.cuda.current_stream().synchronize()
+    w1 = time.perf_counter()
+    e2e_s = w1 - w0
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_val = world * wl.bytes_step * Ke / e2e_s / 1e9
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch": 1, "layers_per_step": 3, "packed_bytes_per_step": wl.bytes_step,
+                   "us_per_layer": round(launch_us, 3),
+                   "l2": "cold: %d distinct packed copies of each layer (%.0f MB per rotation, L2 is 126 MB)" % (
+                       copies, copies * wl.bytes_step / 1e6),
+                   "launch": "stb_layer_stack captured in a CUDA graph, %d steps per replay" % copies,
+                   "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": xh.numel() * 2, "d2h_bytes_per_step": yh.numel() * 4,
+                "steps": Ke, "us_per_step": round(1e6 * e2e_s / Ke, 2),
+                "call": "stb_layer_stack_host: pinned host x -> device, 3 GEMVs, y -> pinned host, stream sync per step"},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": None,
+                     "kernel": "stb::gemv_fast_kernel<6>", "peak_source": pk["_source"],
+                     "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
+                     "note": "launch_us = timed region / launches (includes the gaps between launches)"},
+    }
+    if world == 1 and not args.no_extras:
+        tab, ctx = gemv_table(stb, torch, wl, pk)
+        line["gemv_layers"] = tab
+        line["dense_context"] = ctx
+        line["paper_context"] = ("paper's own kernel (2:4 1-bit GEMM, RTX 4090): up to 17.85x over ABQ-LLM 2-bit, "
+                                 "263.45 TFLOPS = 79.74% of that GPU's sparse tensor-core peak at sequence length 8192")
+    if world == 1 and not args.no_cpu:
+        import oracle
+        oracle.build()
+        Ls = [oracle.Logical(**d) for d in wl.logical]
+        x0 = wl.x_np.astype(np.float64)
+        x1 = wl.h_gate.double().cpu().numpy()
+        xs = [x0, x0, x1]
+        rows = [np.arange(d["n"], dtype=np.int32) for d in wl.logical]
+        t, reps = 0.0, 0
+        while t < 10.0 and reps < 50:
+            t += oracle_pass(Ls, xs, rows)
+            reps += 1
+        line["cpu_baseline"] = {"value": wl.bytes_step * reps / t / 1e9, "unit": UNIT, "cores": oracle.hardware_threads(),
+                                "kind": "oracle", "sample": "all output rows of gate, up and down, batch 1, %d passes (%.1f s)" % (reps, t),
+                                "us_per_layer": round(1e6 * t / reps / 3, 1)}
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None, help="default: 60000 (cuda), 20 (reference)")
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-layer table and the dense context")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = args.steps or 20
+        reference_arm(args)
+    else:
+        args.steps = args.steps or 60000
+        cuda_arm(args)
+
+
+if __name__ == "__main__":
+    main()

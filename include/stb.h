@@ -136,6 +136,14 @@ int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size
  * N:M assignment, Section 3.3).  steps is a HOST array.  Launches only. */
 int stb_layer_stack(const stb_step *steps, int count, int *dev_status, void *stream);
 
+/* stb_layer_stack for a caller whose activations live in HOST memory: copies in_bytes from
+ * in_host (HOST, pinned for the copy to be asynchronous) into steps[0].in, runs the steps,
+ * then copies out_bytes from steps[count-1].out to out_host (HOST).  The device buffers named
+ * in the steps stay caller-owned staging; everything is queued on `stream` and the caller
+ * synchronises it before reading out_host.  Same per-layer N rule (Section 3.3). */
+int stb_layer_stack_host(const stb_step *steps, int count, const void *in_host, size_t in_bytes,
+                         void *out_host, size_t out_bytes, int *dev_status, void *stream);
+
 /* Static string for a status code. */
 const char *stb_status_str(int status);
 

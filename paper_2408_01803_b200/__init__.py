@@ -21,7 +21,7 @@ STB_ERR_UNSUPPORTED, STB_ERR_CORRUPT, STB_ERR_TIMEOUT, STB_ERR_CUDA = 5, 6, 7, 8
 STB_F16, STB_BF16, STB_F32 = 0, 1, 2
 
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv",
-           "stb_gemm_workspace", "stb_gemm", "stb_layer_stack", "stb_status_str"]
+           "stb_gemm_workspace", "stb_gemm", "stb_layer_stack", "stb_layer_stack_host", "stb_status_str"]
 
 
 class StbError(RuntimeError):
@@ -61,6 +61,7 @@ def _load():
     lib.stb_gemm_workspace.argtypes = [i, i, i, i, p(z)]
     lib.stb_gemm.argtypes = [v, i, i, i, v, i, z, v, i, z, v, z, v, v]
     lib.stb_layer_stack.argtypes = [p(_Step), i, v, v]
+    lib.stb_layer_stack_host.argtypes = [p(_Step), i, v, z, v, z, v, v]
     lib.stb_status_str.argtypes = [i]
     lib.stb_status_str.restype = C.c_char_p
     for name in EXPORTS:
@@ -218,3 +219,12 @@ def layer_stack(steps, dev_status=None, stream=None, marshalled=None):
     """stb_layer_stack over a list of (PackedLayer, x, out) triples (or a pre-marshalled array)."""
     arr = marshalled if marshalled is not None else make_steps(steps)
     _check(_lib.stb_layer_stack(arr, len(arr), _ptr(dev_status), _stream(stream)), "stb_layer_stack")
+
+
+def layer_stack_host(marshalled, x_host, y_host, dev_status=None, stream=None):
+    """stb_layer_stack_host: x_host / y_host are pinned CPU tensors; the first step's input and
+    the last step's output (device tensors named in `marshalled`) are the staging buffers."""
+    _check(_lib.stb_layer_stack_host(marshalled, len(marshalled), C.c_void_p(x_host.data_ptr()),
+                                     x_host.numel() * x_host.element_size(), C.c_void_p(y_host.data_ptr()),
+                                     y_host.numel() * y_host.element_size(), _ptr(dev_status), _stream(stream)),
+           "stb_layer_stack_host")

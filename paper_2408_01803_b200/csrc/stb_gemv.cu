@@ -292,3 +292,16 @@ extern "C" int stb_layer_stack(const stb_step* steps, int count, int* dev_status
   }
   return STB_OK;
 }
+
+extern "C" int stb_layer_stack_host(const stb_step* steps, int count, const void* in_host, size_t in_bytes,
+                                    void* out_host, size_t out_bytes, int* dev_status, void* stream) {
+  if (!steps || count < 1 || !in_host || !out_host || !steps[0].in || !steps[count - 1].out) return STB_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(const_cast<void*>(steps[0].in), in_host, in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return STB_ERR_CUDA;
+  const int rc = stb_layer_stack(steps, count, dev_status, stream);
+  if (rc != STB_OK) return rc;
+  if (cudaMemcpyAsync(out_host, steps[count - 1].out, out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return STB_ERR_CUDA;
+  return STB_OK;
+}

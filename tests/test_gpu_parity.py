@@ -18,6 +18,8 @@ TOL = 5e-3
 def stb():
     import torch
     assert torch.cuda.is_available()
+    from paper_2408_01803_b200 import build
+    build.build()                      # no-op when libstb.so is newer than its sources
     import paper_2408_01803_b200 as stb
     return stb
 
