@@ -128,11 +128,12 @@ def oracle_pass(Ls, xs, rows, threads=0):
 
 def stream_bytes_of(d: dict) -> int:
     """Bytes one GEMV pass streams for a logical layer: 16 + 6N + 10 bytes per row and block plus
-    one residual byte per row and block for every started group of 8 salient columns; rows are
-    padded to tiles of 32."""
+    two residual bits for each of the 0 / 4 / 8 / 16 / 32 salient-column slots of a block (the
+    smallest count that holds the layer's largest block); rows are padded to tiles of 32."""
     n, m, N = d["n"], d["m"], d["N"]
-    nres = sum(-(-bin(int(a) | (int(b) << 64)).count("1") // 8) for a, b in d["salient"])
-    return -(-n // 32) * 32 * ((26 + 6 * N) * (m // 128) + nres)
+    most = max(bin(int(a) | (int(b) << 64)).count("1") for a, b in d["salient"])
+    spb = 0 if most == 0 else 4 if most <= 4 else 8 if most <= 8 else 16 if most <= 16 else 32
+    return -(-n // 32) * 32 * (26 + 6 * N + spb // 4) * (m // 128)
 
 
 def reference_arm(args):

@@ -1,85 +1,258 @@
-// Plain (position-order) decode of one row-block from the packed layout.  Used by
-// stb_dequant and by the general GEMV kernel (any N, any batch); the fast batch-1 GEMV has
-// its own rank-order decode.
+// Decode of the packed layout (stb_layout.cuh), shared by the CUDA kernels.  Everything here
+// works on 32-bit words and is host + device code: compiled for the host (byte permute
+// emulated) the bit layouts are checked against the plain definition without a GPU.
+//
+//   LaneTile / load_lane_tile   the registers one lane holds of one tile
+//   build_lane_words            logical fields of the lane's 16 slots -> packed words (pack)
+//   plain_slot                  position-order decode of one slot, bit by bit (dequant, general
+//                               GEMV): the plain definition, any N
+//   FastRows / fast_slot        N = 4, 5, 6: byte-permute decode of one slot into 8 half
+//                               precision weights (4 registers), the form the tensor-core paths
+//                               consume.  Works on whatever 16-bit scale bytes it is given
+//                               (fp16 for the GEMV, bf16 for the GEMM).
 #pragma once
-#include <cuda_fp16.h>
 #include <stdint.h>
 
 #include "stb_layout.cuh"
 
 namespace stb {
 
+STB_HD uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
+#if defined(__CUDA_ARCH__)
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(s));
+  return d;
+#else
+  const uint64_t src = ((uint64_t)b << 32) | a;
+  uint32_t d = 0;
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t nib = (s >> (4 * i)) & 0xFu;
+    uint32_t byte = (uint32_t)(src >> (8 * (nib & 7u))) & 0xFFu;
+    if (nib & 8u) byte = (byte & 0x80u) ? 0xFFu : 0x00u;
+    d |= byte << (8 * i);
+  }
+  return d;
+#endif
+}
+
+// ------------------------------------------------------------------------------------------
 template <int N>
-struct RowBlock {
-  uint32_t mask[4];
+struct LaneTile {
+  static constexpr int kFull = sign_full_words(N);
+  uint32_t mask[4];                     // word j = row g + 8 j: byte s = keep byte of group 4 s + t
+  uint32_t R[N];                        // region words (low part, then high part)
+  uint32_t S[kFull > 0 ? kFull : 1];    // full sign words (low part, then high part)
+  uint32_t half;                        // shared half sign word, already in lower-lane form
+  uint32_t A[4], B[4];                  // per row j: low / high bytes of the four main scales
+  uint32_t sal2[2];                     // a_sal2 of rows 0,1 / 2,3 (two fp16 per word)
+};
+
+template <int NW>
+STB_HD void load_planes(const uint8_t* tile, uint32_t base, uint32_t* w, int lane) {
+  constexpr int Q4 = NW / 4;
+#pragma unroll
+  for (int q = 0; q < Q4; ++q) {
+    const uint4 v = *reinterpret_cast<const uint4*>(tile + base + q * 512 + lane * 16);
+    w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+  }
+  uint32_t o = base + Q4 * 512;
+  if (NW & 2) {
+    const uint2 v = *reinterpret_cast<const uint2*>(tile + o + lane * 8);
+    w[4 * Q4] = v.x; w[4 * Q4 + 1] = v.y;
+    o += 256;
+  }
+  if (NW & 1) w[NW - 1] = *reinterpret_cast<const uint32_t*>(tile + o + lane * 4);
+}
+
+// `tile` may point to global or to shared memory (16-byte aligned).
+template <int N>
+STB_HD void load_lane_tile(const uint8_t* tile, int lane, LaneTile<N>& t) {
+  const int g = lane >> 2;
+  const uint4 mk = *reinterpret_cast<const uint4*>(tile + lane * 16);
+  t.mask[0] = mk.x; t.mask[1] = mk.y; t.mask[2] = mk.z; t.mask[3] = mk.w;
+  load_planes<N>(tile, off_region(N), t.R, lane);
+  load_planes<LaneTile<N>::kFull>(tile, off_sign(N), t.S, lane);
+  t.half = 0;
+  if (sign_has_half(N)) {
+    const uint32_t h = *reinterpret_cast<const uint32_t*>(tile + sign_half_off(N, lane));
+    t.half = lane < 16 ? (h & 0x66666666u) : half_from_upper(h & 0x99999999u);
+  }
+  const uint4 s0 = *reinterpret_cast<const uint4*>(tile + scale_off(N, g, 0));
+  const uint4 s1 = *reinterpret_cast<const uint4*>(tile + scale_off(N, g, 2));
+  t.A[0] = s0.x; t.B[0] = s0.y; t.A[1] = s0.z; t.B[1] = s0.w;
+  t.A[2] = s1.x; t.B[2] = s1.y; t.A[3] = s1.z; t.B[3] = s1.w;
+  const uint2 a2 = *reinterpret_cast<const uint2*>(tile + sal2_off(N, g, 0));
+  t.sal2[0] = a2.x; t.sal2[1] = a2.y;
+}
+
+// fp16 bit pattern of main scale q (0..3) / of a_sal2 of row j
+template <int N>
+STB_HD uint32_t scale_bits(const LaneTile<N>& t, int j, int q) {
+  return ((t.A[j] >> (8 * q)) & 0xFFu) | (((t.B[j] >> (8 * q)) & 0xFFu) << 8);
+}
+template <int N>
+STB_HD uint32_t sal2_bits(const LaneTile<N>& t, int j) {
+  return (t.sal2[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+}
+
+// ------------------------------------------------------------------------------------------
+// Pack side: the lane's words from the logical fields of its 16 slots.
+//   keep[u], sign[u] (bit k = 1: k-th kept weight is +1), region[u] (2 bits per kept weight)
+template <int N>
+struct LaneWords {
   uint32_t R[N];
-  uint32_t S[(N + 1) / 2];   // odd N: last entry is the half word in lower-lane form
-  float alpha[5];
-  uint32_t resid;            // residual sign bits of the block's salient columns (1 = +1)
+  uint32_t S[LaneTile<N>::kFull > 0 ? LaneTile<N>::kFull : 1];
+  uint32_t half;      // lower-lane form
 };
 
 template <int N>
-__device__ __forceinline__ void load_rowblock(const uint8_t* __restrict__ tile, int lane, int rb,
-                                              RowBlock<N>& r) {
-  const uint4 mk = *reinterpret_cast<const uint4*>(tile + lane * 16);
-  r.mask[0] = mk.x; r.mask[1] = mk.y; r.mask[2] = mk.z; r.mask[3] = mk.w;
+STB_HD void build_lane_words(const uint32_t (&sign)[16], const uint32_t (&region)[16], bool valid,
+                             LaneWords<N>& w) {
 #pragma unroll
-  for (int i = 0; i < N; ++i)
-    r.R[i] = *reinterpret_cast<const uint32_t*>(tile + region_word_off(N, i, lane));
+  for (int i = 0; i < N; ++i) w.R[i] = 0;
 #pragma unroll
-  for (int i = 0; i < N / 2; ++i)
-    r.S[i] = *reinterpret_cast<const uint32_t*>(tile + sign_word_off(N, i, lane));
-  if (N & 1) {
-    uint32_t h = *reinterpret_cast<const uint32_t*>(tile + sign_half_off(N, lane));
-    r.S[N / 2] = lane < 16 ? (h & 0x66666666u) : half_from_upper(h);
-  }
-  const uint2 ab = *reinterpret_cast<const uint2*>(tile + off_scale(N) + lane * 8);
+  for (int i = 0; i < (LaneTile<N>::kFull > 0 ? LaneTile<N>::kFull : 1); ++i) w.S[i] = 0;
+  w.half = 0;
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const uint16_t hb = (uint16_t)(((ab.x >> (8 * q)) & 0xFFu) | (((ab.y >> (8 * q)) & 0xFFu) << 8));
-    r.alpha[q] = __half2float(__ushort_as_half(hb));
-  }
-  r.alpha[4] = __half2float(__ushort_as_half(
-      *reinterpret_cast<const uint16_t*>(tile + off_sal2(N) + lane * 2)));
-  r.resid = 0;
-  for (int p = 0; p < rb; ++p) r.resid |= (uint32_t)tile[off_resid(N) + p * 32 + lane] << (8 * p);
-}
-
-// Decode group g (8 columns) of the row-block into fp32, position order.
-// salb: the block's salient bits of this group; tbase: number of salient columns of the block
-// before this group.
-template <int N>
-__device__ __forceinline__ void decode_group(const RowBlock<N>& r, int g, uint32_t salb, int tbase,
-                                             float out[8]) {
-  const uint32_t kb = (r.mask[g >> 2] >> (8 * (g & 3))) & 0xFFu;
-  // the group's weights w = g*N .. g*N+N-1 touch at most two region words and two sign
-  // words; pick between them with compile-time indices (g is an unrolled loop counter)
-  const int iw0 = (g * N) >> 4, iw1 = (iw0 + 1 < N) ? iw0 + 1 : N - 1;
-  constexpr int NS = (N + 1) / 2;
-  const int sw0 = (g * N) >> 5, sw1 = (sw0 + 1 < NS) ? sw0 + 1 : NS - 1;
+  for (int u = 0; u < 16; ++u) {
 #pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    float v = 0.0f;
-    if ((kb >> c) & 1u) {
-      const int w = g * N + __popc(kb & ((1u << c) - 1u));
-      const uint32_t rw = ((w >> 4) == iw0) ? r.R[iw0] : r.R[iw1];
-      const uint32_t sw = ((w >> 5) == sw0) ? r.S[sw0] : r.S[sw1];
-      const uint32_t code = (rw >> code_bit(w)) & 3u;
-      const uint32_t neg = (sw >> sign_bit(w)) & 1u;
-      const float s1 = neg ? -1.0f : 1.0f;
-      if (code == 3u) {
-        const int t = tbase + __popc(salb & ((1u << c) - 1u));
-        const float s2 = ((r.resid >> t) & 1u) ? 1.0f : -1.0f;
-        v = __fadd_rn(s1 * r.alpha[3], s2 * r.alpha[4]);
-      } else {
-        v = s1 * (code == 0u ? r.alpha[0] : (code == 1u ? r.alpha[1] : r.alpha[2]));
-      }
+    for (int k = 0; k < N; ++k) {
+      const uint32_t code = valid ? (region[u] >> (2 * k)) & 3u : 0u;
+      const uint32_t neg = valid ? ((sign[u] >> k) & 1u) ^ 1u : 0u;
+      const BitPos rp = region_pos(N, u, k), sp = sign_pos(N, u, k);
+      w.R[rp.word] |= code << rp.bit;
+      if (sp.half) w.half |= neg << sp.bit;
+      else w.S[sp.word] |= neg << sp.bit;
     }
-    out[c] = v;
   }
 }
 
-__device__ __forceinline__ bool header_matches(const Header* h, int n, int m, int N) {
+// ------------------------------------------------------------------------------------------
+// Plain decode of slot u = 4 j + s into (code, negative) per column, then to values by the
+// caller.  out_code[c] = 0..3 region code, 4 = dropped; out_neg[c] = 1 for a negative weight.
+template <int N>
+STB_HD void plain_slot(const LaneTile<N>& t, int u, uint32_t (&out_code)[8], uint32_t (&out_neg)[8]) {
+  const int j = u >> 2, s = u & 3;
+  const uint32_t kb = (t.mask[j] >> (8 * s)) & 0xFFu;
+  int k = 0;
+  for (int c = 0; c < 8; ++c) {
+    out_code[c] = 4u; out_neg[c] = 0u;
+    if (!((kb >> c) & 1u) || k >= N) continue;
+    const BitPos rp = region_pos(N, u, k), sp = sign_pos(N, u, k);
+    uint32_t rw = 0, sw = 0;
+    for (int i = 0; i < N; ++i) rw = (i == rp.word) ? t.R[i] : rw;
+    if (sp.half) sw = t.half;
+    else
+      for (int i = 0; i < LaneTile<N>::kFull; ++i) sw = (i == sp.word) ? t.S[i] : sw;
+    out_code[c] = (rw >> rp.bit) & 3u;
+    out_neg[c] = (sw >> sp.bit) & 1u;
+    ++k;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Fast decode, N = 4, 5, 6.
+//
+// Scale side: the codes are stored so that masking a region word gives byte-permute selectors
+// (one nibble per kept weight) into the four scale bytes of the row; the sign bit is OR-ed into
+// bit 2 of the nibble and picks the byte of +scale or -scale.  One permute per byte plane gives
+// the low / high bytes of four kept weights in rank order: ranks 0..3 of a slot from the low
+// part, ranks 4.. from the high part (N = 6: ranks 4,5 of two slots per permute; N = 5: rank 4
+// of the four slots of a row).
+// Position side: a 256-entry table maps the keep byte to a selector (one nibble per column:
+// the rank of the column among the kept ones, or 7 = a zero byte) that spreads the rank-ordered
+// bytes to the 8 column positions; two more permutes per pair of registers re-interleave low
+// and high bytes into 16-bit values.
+template <int N>
+struct FastRows {
+  static_assert(N >= 4 && N <= 6, "fast decode covers N = 4, 5, 6");
+  uint32_t A[4], Bp[4], Bn[4];
+  uint32_t e[4], o[4];
+  uint32_t eh[2], oh[2];
+
+  // A_, B_: low / high bytes of the four main scales per row, in the 16-bit format wanted
+  STB_HD void init(const LaneTile<N>& t, const uint32_t (&A_)[4], const uint32_t (&B_)[4]) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      A[j] = A_[j]; Bp[j] = B_[j]; Bn[j] = B_[j] ^ 0x80808080u;
+      const uint32_t sw = t.S[j >> 1];
+      const uint32_t se = (j & 1) ? (sw >> 1) : sw;
+      const uint32_t so = (j & 1) ? (sw << 2) : (sw << 1);
+      e[j] = (t.R[j] & 0x33333333u) | (se & 0x44444444u);
+      o[j] = ((t.R[j] >> 2) & 0x33333333u) | (so & 0x44444444u);
+    }
+    eh[0] = eh[1] = oh[0] = oh[1] = 0;
+    if (N == 6) {
+      const uint32_t sw = t.S[2];
+      eh[0] = (t.R[4] & 0x33333333u) | (sw & 0x44444444u);
+      oh[0] = ((t.R[4] >> 2) & 0x33333333u) | ((sw << 1) & 0x44444444u);
+      eh[1] = (t.R[5] & 0x33333333u) | ((sw >> 1) & 0x44444444u);
+      oh[1] = ((t.R[5] >> 2) & 0x33333333u) | ((sw << 2) & 0x44444444u);
+    } else if (N == 5) {
+      eh[0] = (t.R[4] & 0x33333333u) | (t.half & 0x44444444u);
+      oh[0] = ((t.R[4] >> 2) & 0x33333333u) | ((t.half << 1) & 0x44444444u);
+    }
+  }
+
+  // rank-ordered bytes of ranks 4.. : N = 6 one call per (row j, step pair sp), N = 5 one call
+  // per row j (sp ignored)
+  STB_HD void high(int j, int sp, uint32_t& XL, uint32_t& XH) const {
+    uint32_t sel;
+    if (N == 6) sel = ((j & 1) ? oh[j >> 1] : eh[j >> 1]) >> (16 * sp);
+    else sel = ((j & 2) ? oh[0] : eh[0]) >> (16 * (j & 1));
+    XL = prmt(A[j], A[j], sel);
+    XH = prmt(Bp[j], Bn[j], sel);
+  }
+
+  // Slot (j, s) -> f[0..3]: columns (0,1), (2,3), (4,5), (6,7) as 16-bit pairs (low half =
+  // lower column).  P = position selector of the slot's keep byte.
+  STB_HD void slot(int j, int s, uint32_t P, uint32_t XL, uint32_t XH, uint32_t (&f)[4]) const {
+    const uint32_t sel = ((s & 2) ? o[j] : e[j]) >> (16 * (s & 1));
+    const uint32_t lo0 = prmt(A[j], A[j], sel), hi0 = prmt(Bp[j], Bn[j], sel);
+    uint32_t lo1 = 0, hi1 = 0;
+    if (N == 6) {
+      lo1 = (s & 1) ? (XL >> 16) : (XL & 0xFFFFu);
+      hi1 = (s & 1) ? (XH >> 16) : (XH & 0xFFFFu);
+    } else if (N == 5) {
+      lo1 = prmt(XL, 0u, 0x4440u + (uint32_t)s);
+      hi1 = prmt(XH, 0u, 0x4440u + (uint32_t)s);
+    }
+    const uint32_t P1 = P >> 16;
+    const uint32_t pl0 = prmt(lo0, lo1, P), pl1 = prmt(lo0, lo1, P1);
+    const uint32_t ph0 = prmt(hi0, hi1, P), ph1 = prmt(hi0, hi1, P1);
+    f[0] = prmt(pl0, ph0, 0x5140u);
+    f[1] = prmt(pl0, ph0, 0x7362u);
+    f[2] = prmt(pl1, ph1, 0x5140u);
+    f[3] = prmt(pl1, ph1, 0x7362u);
+  }
+};
+
+// position selector of a keep byte: nibble c = rank of column c among the kept columns, 7 for a
+// dropped column (byte 7 of the rank-ordered bytes is zero for N <= 7)
+STB_HD uint32_t position_selector(uint32_t keep_byte) {
+  uint32_t p = 0, r = 0;
+  for (int c = 0; c < 8; ++c) {
+    if ((keep_byte >> c) & 1u) { p |= (r & 7u) << (4 * c); ++r; }
+    else p |= 7u << (4 * c);
+  }
+  return p;
+}
+STB_HD uint32_t keep_byte_of(const uint32_t (&mask)[4], int j, int s) {
+  return prmt(mask[j], 0u, 0x4440u + (uint32_t)s);
+}
+
+// Residual selectors of one resid word (rows r_0..r_3 of the lane, 4 slots): row j's four
+// nibbles (0 = +a_sal2, 1 = none, 2 = -a_sal2) index the bytes of
+//   L2 = (lo, 0, lo, 0)   H2 = (hi, 0, hi ^ 0x80, 0)      (lo / hi byte of a_sal2 of the row)
+STB_HD uint32_t resid_selector(uint32_t word, int j) {
+  const uint32_t v = (j & 2) ? ((word >> 2) & 0x33333333u) : (word & 0x33333333u);
+  return (v >> (16 * (j & 1))) & 0xFFFFu;
+}
+STB_HD uint32_t resid_code(uint32_t word, int j, int q4) {
+  return (word >> code_bit(4 * j + q4)) & 3u;
+}
+
+STB_HD bool header_matches(const Header* h, int n, int m, int N) {
   return h->magic == kMagic && h->n == n && h->m == m && h->N == N && h->status == 0u;
 }
 

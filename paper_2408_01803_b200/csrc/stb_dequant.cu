@@ -16,7 +16,7 @@ template <> __device__ __forceinline__ float cvt_out<float>(float v) { return v;
 template <> __device__ __forceinline__ __half cvt_out<__half>(float v) { return __float2half_rn(v); }
 template <> __device__ __forceinline__ __nv_bfloat16 cvt_out<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
-// One warp per tile, lane = row.
+// One warp per tile; lane = (g, t) decodes its 16 (row, group) slots, 8 columns each.
 template <int N, typename T>
 __global__ void __launch_bounds__(256)
 dequant_kernel(const uint8_t* __restrict__ packed, int n, int m, T* __restrict__ W, size_t ldw) {
@@ -24,27 +24,47 @@ dequant_kernel(const uint8_t* __restrict__ packed, int n, int m, T* __restrict__
   if (!header_matches(hdr, n, m, N)) return;
   const int nblk = m / kBlock;
   const int ntile = (n + kTileRows - 1) / kTileRows;
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (warp >= (long long)ntile * nblk) return;
   const int rt = (int)(warp / nblk), b = (int)(warp % nblk);
   const BlockInfo* bi = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header)) + b;
-  const uint8_t* tile = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride + bi->tile_off;
-  RowBlock<N> r;
-  load_rowblock<N>(tile, lane, (int)bi->res_bytes, r);
-  const int row = rt * kTileRows + lane;
-  if (row >= n) return;
+  const uint8_t* tile = packed + hdr->tiles_offset + ((size_t)rt * nblk + b) * (size_t)hdr->tile_bytes;
+  const int spb = (int)hdr->spb;
+  LaneTile<N> lt;
+  load_lane_tile<N>(tile, lane, lt);
   const uint64_t sal[2] = {bi->salient[0], bi->salient[1]};
-  T* dst = W + (size_t)row * ldw + (size_t)b * kBlock;
-  int tbase = 0;
-#pragma unroll
-  for (int g = 0; g < 16; ++g) {
-    const uint32_t salb = (uint32_t)((sal[g >> 3] >> (8 * (g & 7))) & 0xFFull);
-    float v[8];
-    decode_group<N>(r, g, salb, tbase, v);
-    tbase += __popc(salb);
-#pragma unroll
-    for (int c = 0; c < 8; ++c) dst[g * 8 + c] = cvt_out<T>(v[c]);
+  for (int u = 0; u < 16; ++u) {
+    const int j = u >> 2, s = u & 3;
+    const int row = rt * kTileRows + g + 8 * j;
+    const int grp = 4 * s + t;                                   // group of the block
+    uint32_t code[8], neg[8];
+    plain_slot<N>(lt, u, code, neg);
+    if (row >= n) continue;
+    const uint32_t salb = (uint32_t)((sal[grp >> 3] >> (8 * (grp & 7))) & 0xFFull);
+    // number of salient columns of the block before this group
+    int qbase = grp >= 8 ? __popcll(sal[0]) : 0;
+    qbase += __popcll(sal[grp >> 3] & ((1ull << (8 * (grp & 7))) - 1ull));
+    float alpha[5];
+    for (int q = 0; q < 4; ++q) alpha[q] = __half2float(__ushort_as_half((unsigned short)scale_bits<N>(lt, j, q)));
+    alpha[4] = __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(lt, j)));
+    T* dst = W + (size_t)row * ldw + (size_t)b * kBlock + grp * 8;
+    for (int c = 0; c < 8; ++c) {
+      float v = 0.0f;
+      if (code[c] < 4u) {
+        const float s1 = neg[c] ? -1.0f : 1.0f;
+        if (code[c] == 3u) {
+          const int q = qbase + __popc(salb & ((1u << c) - 1u));
+          const uint32_t word = q < spb ? *reinterpret_cast<const uint32_t*>(tile + resid_word_off(N, spb, g, q >> 2)) : 0x55555555u;
+          const uint32_t rc = resid_code(word, j, q & 3);
+          const float s2 = rc == 0u ? 1.0f : -1.0f;
+          v = __fadd_rn(s1 * alpha[3], s2 * alpha[4]);
+        } else {
+          v = s1 * alpha[code[c]];
+        }
+      }
+      dst[c] = cvt_out<T>(v);
+    }
   }
 }
 

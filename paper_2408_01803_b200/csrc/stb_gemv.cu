@@ -1,36 +1,60 @@
 // stb_gemv: decode GEMV  y[t][i] = sum_j W^[i][j] x[t][j],  batch 1..16, fp32 accumulation.
 // The memory-bound decoding stage of Appendix C.2: every packed byte is read once.
+#include <cooperative_groups.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
-
-#include "../../include/stb.h"
-#include <cooperative_groups.h>
 #include <stdlib.h>
 
+#include "../../include/stb.h"
 #include "stb_decode.cuh"
-#include "stb_gemv_fast.cuh"
 #include "stb_layout.cuh"
+#include "stb_ptx.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace stb {
 
-// -----------------------------------------------------------------------------------------
-// Fast batch-1 kernel, N = 4, 5, 6.  Grid: one thread-block cluster of `ksplit` CTAs per row
-// tile (32 rows); CTA k of the cluster takes the k-th slice of the 128-column blocks, its 8
-// warps take the blocks of the slice round-robin, lane = row.  The packed tiles go straight
-// from HBM into registers (one coalesced vector load per field plane, next tile prefetched
-// while the current one is decoded); x is staged once per CTA in shared memory, byte-planar.
-// Partial sums: 8 warps through shared memory, then the CTAs of the cluster through
-// distributed shared memory in rank order, so the result does not depend on timing.
-constexpr int kFastWarps = 8;
+// ------------------------------------------------------------------------------------------
+// Tensor-core GEMV, N = 4, 5, 6, batch <= 8 NB.
+//
+// Grid: one thread-block cluster of `ksplit` CTAs per row tile (32 rows); CTA k of the cluster
+// takes the k-th slice of the 128-column blocks and its warps take contiguous runs of that
+// slice.  Each warp streams its tiles from HBM into a private ring in shared memory with 1-D
+// bulk copies (kDepth tiles in flight), reads a tile into registers, decodes it slot by slot
+// into fp16 operand registers (stb_decode.cuh) and multiplies with m16n8k16 tensor-core
+// instructions: A = 16 rows x 16 columns of W^, B = the staged activations (8 batch rows),
+// fp32 accumulators in registers for the whole run.  The residual term of the salient columns
+// goes through the same instruction, with the salient slots of 16 / SPB blocks as its K
+// dimension.  Partial sums: warps through shared memory, CTAs of the cluster through
+// distributed shared memory, both in a fixed order.
+constexpr int kDepth = 4;
+constexpr long long kWaitLimit = 2000000000ll;     // about a second of SM clocks
 
-template <int N>
-__global__ void __launch_bounds__(kFastWarps * 32)
-gemv_fast_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* __restrict__ x,
-                 void* __restrict__ y, int y_f16, int* dev_status, int ksplit, int bpp) {
-  extern __shared__ uint4 smem4[];
+struct GemvSmem {
+  uint32_t bars, xs, xsal, ring, part, total;       // byte offsets
+  uint32_t xstride, tile_stride;
+};
+__host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int batch, int bpp, int ksplit, int NB) {
+  GemvSmem s;
+  s.bars = 1024;
+  s.xs = s.bars + (uint32_t)(warps * kDepth * 8);
+  s.xs = (s.xs + 15u) & ~15u;
+  s.xstride = (uint32_t)bpp * 256u + 64u;
+  s.xsal = s.xs + (uint32_t)batch * s.xstride;
+  s.ring = s.xsal + (uint32_t)batch * (uint32_t)bpp * 64u;
+  s.ring = (s.ring + 127u) & ~127u;
+  s.tile_stride = (tile_bytes(N, kMaxSalient) + 127u) & ~127u;
+  s.part = s.ring + (uint32_t)(warps * kDepth) * s.tile_stride;
+  s.total = s.part + (uint32_t)ksplit * 32u * 8u * (uint32_t)NB * 4u;
+  return s;
+}
+
+template <int N, int NB>
+__global__ void __launch_bounds__(256)
+gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* __restrict__ x, int batch,
+                size_t ldx, void* __restrict__ y, int y_f16, size_t ldy, int* dev_status, int ksplit, int bpp) {
+  extern __shared__ __align__(128) uint8_t smem[];
   const Header* hdr = reinterpret_cast<const Header*>(packed);
   // every CTA of a cluster takes the same branch here (the header is the same for all)
   if (!header_matches(hdr, n, m, N)) {
@@ -38,142 +62,273 @@ gemv_fast_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half*
     return;
   }
   const int nblk = m / kBlock;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warps = (int)(blockDim.x >> 5);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
   const int kpart = (int)(blockIdx.x % (unsigned)ksplit), rt = (int)(blockIdx.x / (unsigned)ksplit);
   const int b0 = kpart * bpp, b1 = min(nblk, b0 + bpp);
+  const int nbp = max(b1 - b0, 0);
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+  const uint32_t tbytes = hdr->tile_bytes;
+  const int spb = (int)hdr->spb;
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
+  const GemvSmem L = gemv_smem(N, warps, batch, bpp, ksplit, NB);
 
-  // shared memory: [selector tables 2 KB][x byte-planar bpp*256 B][x plain fp16 bpp*256 B][partials]
-  uint32_t* tab = reinterpret_cast<uint32_t*>(smem4);
-  uint4* xs = smem4 + 128;
-  __half* xplain = reinterpret_cast<__half*>(xs + (size_t)bpp * 16);
-  float* red = reinterpret_cast<float*>(xplain + (size_t)bpp * kBlock);   // [kFastWarps][32] then [ksplit][32]
+  uint32_t* ptab = reinterpret_cast<uint32_t*>(smem);
+  uint8_t* xs = smem + L.xs;
+  __half* xsal = reinterpret_cast<__half*>(smem + L.xsal);
+  uint8_t* ring = smem + L.ring + (size_t)warp * kDepth * L.tile_stride;
+  const uint32_t bar0 = smem_u32(smem + L.bars) + (uint32_t)warp * kDepth * 8u;
 
-  // first tile of this warp: issue its loads before anything else
-  fast::Tile<N> cur;
-  int b = b0 + warp;
-  if (b < b1) fast::load_tile<N>(rtbase + binfo[b].tile_off, lane, (int)binfo[b].res_bytes, cur);
+  // this warp's run of blocks
+  const int per = (nbp + warps - 1) / warps;
+  const int wb0 = b0 + warp * per, wb1 = min(b1, wb0 + per);
+  const int cnt = max(wb1 - wb0, 0);
 
-  fast::build_tables(tab, N, threadIdx.x, blockDim.x);
-  for (int gidx = threadIdx.x; gidx < (b1 - b0) * 16; gidx += blockDim.x) {
-    const uint4 h = __ldg(reinterpret_cast<const uint4*>(x + (size_t)b0 * kBlock) + gidx);
-    reinterpret_cast<uint4*>(xplain)[gidx] = h;
-    xs[gidx] = make_uint4(fast::prmt(h.x, h.y, 0x6420u), fast::prmt(h.z, h.w, 0x6420u),
-                          fast::prmt(h.x, h.y, 0x7531u), fast::prmt(h.z, h.w, 0x7531u));
+  // start the weight stream before anything else
+  if (lane == 0) {
+    for (int i = 0; i < kDepth; ++i) mbar_init(bar0 + 8u * i, 1);
+    fence_async_smem();
+    for (int i = 0; i < kDepth && i < cnt; ++i) {
+      mbar_expect_tx(bar0 + 8u * i, tbytes);
+      bulk_g2s(smem_u32(ring + (size_t)i * L.tile_stride), rtbase + (size_t)(wb0 + i) * tbytes, tbytes, bar0 + 8u * i);
+    }
   }
-  __syncthreads();
 
-  float acc = 0.0f;
-  while (b < b1) {
-    const BlockInfo* bi = binfo + b;
-    const int bn = b + kFastWarps;
-    fast::Tile<N> nxt;
-    if (bn < b1) fast::load_tile<N>(rtbase + binfo[bn].tile_off, lane, (int)binfo[bn].res_bytes, nxt);
-    acc += fast::rowblock_dot<N>(cur, xs + (size_t)(b - b0) * 16, tab, lane);
-    // residual term of the block's salient columns: a_sal2 * (+-1) * x[col] where kept
-    const int nsal = (int)bi->nsal;
-    if (nsal) {
-      const float a2 = __half2float(__ushort_as_half((unsigned short)cur.sal2));
-      const __half* xb = xplain + (size_t)(b - b0) * kBlock;
-      float r = 0.0f;
-      int t = 0;
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
-        uint64_t mk = bi->salient[half];
-        while (mk) {
-          const int c = __ffsll((long long)mk) - 1 + 64 * half;
+  // stage the activations of this CTA's columns, the salient-column activations and the table
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) ptab[i] = g_pos_table.v[i];
+  for (int bt = 0; bt < batch; ++bt) {
+    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)bt * ldx + (size_t)b0 * kBlock);
+    uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)bt * L.xstride);
+    for (int i = threadIdx.x; i < nbp * 16; i += blockDim.x) dst[i] = __ldg(src + i);
+  }
+  if (spb > 0) {
+    for (int i = threadIdx.x; i < nbp * batch; i += blockDim.x) {
+      const int bl = i % nbp, bt = i / nbp;
+      const BlockInfo* bi = binfo + b0 + bl;
+      __half* dst = xsal + ((size_t)bt * bpp + bl) * spb;
+      const __half* xr = x + (size_t)bt * ldx + (size_t)(b0 + bl) * kBlock;
+      int q = 0;
+      for (int h = 0; h < 2; ++h) {
+        uint64_t mk = bi->salient[h];
+        while (mk && q < spb) {
+          const int c = __ffsll((long long)mk) - 1 + 64 * h;
           mk &= mk - 1;
-          const int wi = c >> 5;
-          const uint32_t mw = wi == 0 ? cur.mask[0] : (wi == 1 ? cur.mask[1] : (wi == 2 ? cur.mask[2] : cur.mask[3]));
-          const float xv = __half2float(xb[c]);
-          const float sv = ((cur.resid >> t) & 1u) ? xv : -xv;
-          r += ((mw >> (c & 31)) & 1u) ? sv : 0.0f;
-          ++t;
+          dst[q++] = xr[c];
         }
       }
-      acc = fmaf(a2, r, acc);
+      for (; q < spb; ++q) dst[q] = __ushort_as_half((unsigned short)0);
     }
-    if (bn < b1) cur = nxt;
-    b = bn;
   }
-
-  red[warp * 32 + lane] = acc;
   __syncthreads();
-  float s = 0.0f;
-  if (warp == 0) {
+
+  float acc[2][NB][4];
 #pragma unroll
-    for (int w = 0; w < kFastWarps; ++w) s += red[w * 32 + lane];
-  }
-  const int row = rt * kTileRows + lane;
-  if (ksplit == 1) {
-    if (warp == 0 && row < n) {
-      if (y_f16) static_cast<__half*>(y)[row] = __float2half_rn(s);
-      else static_cast<float*>(y)[row] = s;
+  for (int a = 0; a < 2; ++a)
+#pragma unroll
+    for (int c = 0; c < NB; ++c)
+#pragma unroll
+      for (int d = 0; d < 4; ++d) acc[a][c][d] = 0.0f;
+
+  // residual bookkeeping: 16 / SPB blocks share one residual instruction (K = 16 salient slots)
+  const int bpr = spb == 0 ? 1 : (spb >= 16 ? 1 : 16 / spb);     // blocks per residual instruction
+  const int wpb = spb >= 16 ? 4 : (spb >> 2);                     // words of a block per instruction
+  uint32_t rword = 0x55555555u, rword2 = 0x55555555u, rsal0 = 0, rsal1 = 0;
+  int rblk = 0;
+  bool failed = false;
+
+  for (int it = 0; it < cnt; ++it) {
+    const int slot = it % kDepth;
+    const uint32_t bar = bar0 + 8u * slot;
+    // all lanes poll; the verdict is made warp-uniform so that nobody is left at a __syncwarp
+    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(it / kDepth) & 1u, kWaitLimit))) { failed = true; break; }
+    const uint8_t* tile = ring + (size_t)slot * L.tile_stride;
+    LaneTile<N> lt;
+    load_lane_tile<N>(tile, lane, lt);
+    const int b = wb0 + it;
+    if (spb > 0) {
+      const int pos = it % bpr;
+      if (bpr == 1 || t / wpb == pos) {
+        const int wq = bpr == 1 ? t : t % wpb;
+        rword = *reinterpret_cast<const uint32_t*>(tile + resid_word_off(N, spb, g, wq));
+        if (spb == 32) rword2 = *reinterpret_cast<const uint32_t*>(tile + resid_word_off(N, spb, g, wq + 4));
+        rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1];
+        rblk = b - b0;
+      }
     }
-    return;
+    __syncwarp();
+    if (lane == 0 && it + kDepth < cnt) {          // refill the slot that was just read
+      fence_async_smem();
+      mbar_expect_tx(bar, tbytes);
+      bulk_g2s(smem_u32(tile), rtbase + (size_t)(b + kDepth) * tbytes, tbytes, bar);
+    }
+
+    FastRows<N> fr;
+    fr.init(lt, lt.A, lt.B);
+    uint32_t XL[4] = {0, 0, 0, 0}, XH[4] = {0, 0, 0, 0};
+    if (N == 5) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) fr.high(j, 0, XL[j], XH[j]);
+    }
+    const uint8_t* xb = xs + (size_t)(b - b0) * 256 + t * 16;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      uint4 xf[NB];
+#pragma unroll
+      for (int c = 0; c < NB; ++c) {
+        xf[c] = make_uint4(0, 0, 0, 0);
+        if (g + 8 * c < batch) xf[c] = *reinterpret_cast<const uint4*>(xb + (size_t)(g + 8 * c) * L.xstride + s * 64);
+      }
+      uint32_t f[4][4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (N == 6 && (s & 1) == 0) fr.high(j, s >> 1, XL[j], XH[j]);
+        const uint32_t P = ptab[keep_byte_of(lt.mask, j, s)];
+        fr.slot(j, s, P, XL[j], XH[j], f[j]);
+      }
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int c = 0; c < NB; ++c) {
+          mma16816(acc[mt][c], f[2 * mt][0], f[2 * mt + 1][0], f[2 * mt][1], f[2 * mt + 1][1], xf[c].x, xf[c].y);
+          mma16816(acc[mt][c], f[2 * mt][2], f[2 * mt + 1][2], f[2 * mt][3], f[2 * mt + 1][3], xf[c].z, xf[c].w);
+        }
+    }
+
+    // residual term: once the salient slots of `bpr` blocks are collected (or at the end)
+    if (spb > 0 && ((it % bpr) == bpr - 1 || it == cnt - 1)) {
+#pragma unroll 1
+      for (int pass = 0; pass < (spb == 32 ? 2 : 1); ++pass) {
+        const uint32_t rw = pass ? rword2 : rword;
+        const int wq = (bpr == 1 ? t : t % wpb) + 4 * pass;
+        uint32_t fa[4][2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t h = (((j & 2) ? rsal1 : rsal0) >> (16 * (j & 1))) & 0xFFFFu;
+          const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
+          const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
+          const uint32_t sel = resid_selector(rw, j);
+          const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
+          fa[j][0] = prmt(lo4, hi4, 0x5140u);
+          fa[j][1] = prmt(lo4, hi4, 0x7362u);
+        }
+#pragma unroll
+        for (int c = 0; c < NB; ++c) {
+          uint2 xr = make_uint2(0, 0);
+          if (g + 8 * c < batch)
+            xr = *reinterpret_cast<const uint2*>(xsal + ((size_t)(g + 8 * c) * bpp + rblk) * spb + wq * 4);
+          mma16816(acc[0][c], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
+          mma16816(acc[1][c], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
+        }
+      }
+      rword = 0x55555555u; rword2 = 0x55555555u;
+    }
   }
-  cg::cluster_group cluster = cg::this_cluster();
-  float* part = red + kFastWarps * 32;                       // [ksplit][32], used on cluster rank 0
-  if (warp == 0) {
-    float* dst = cluster.map_shared_rank(part, 0);
-    dst[kpart * 32 + lane] = s;
+
+  if (failed) {
+    // give the copies still in flight time to land before the shared memory is given up
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000) {}
+    if (lane == 0 && dev_status) *dev_status = STB_ERR_TIMEOUT;
   }
-  cluster.sync();
-  if (kpart == 0 && warp == 0 && row < n) {
-    float tsum = 0.0f;
-    for (int k = 0; k < ksplit; ++k) tsum += part[k * 32 + lane];
-    if (y_f16) static_cast<__half*>(y)[row] = __float2half_rn(tsum);
-    else static_cast<float*>(y)[row] = tsum;
+  __syncthreads();     // every warp is done with its ring: reuse it for the partial sums
+
+  // red[warp][row 0..31][batch 0..8NB-1]
+  constexpr int BW = 8 * NB;
+  float* red = reinterpret_cast<float*>(smem + L.ring);
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int c = 0; c < NB; ++c) {
+      float* r0 = red + ((size_t)warp * 32 + (g + 16 * mt)) * BW + 8 * c + 2 * t;
+      float* r1 = r0 + 8 * BW;
+      r0[0] = acc[mt][c][0]; r0[1] = acc[mt][c][1];
+      r1[0] = acc[mt][c][2]; r1[1] = acc[mt][c][3];
+    }
+  __syncthreads();
+  float* part = reinterpret_cast<float*>(smem + L.part);       // [ksplit][32][BW], used on cluster rank 0
+  for (int i = threadIdx.x; i < 32 * BW; i += blockDim.x) {
+    float sacc = 0.0f;
+    for (int w = 0; w < warps; ++w) sacc += red[(size_t)w * 32 * BW + i];
+    if (ksplit == 1) {
+      const int row = rt * kTileRows + i / BW, bt = i % BW;
+      if (row < n && bt < batch) {
+        if (y_f16) static_cast<__half*>(y)[(size_t)bt * ldy + row] = __float2half_rn(sacc);
+        else static_cast<float*>(y)[(size_t)bt * ldy + row] = sacc;
+      }
+    } else {
+      float* dst = cg::this_cluster().map_shared_rank(part, 0);
+      dst[(size_t)kpart * 32 * BW + i] = sacc;
+    }
+  }
+  if (ksplit == 1) return;
+  cg::this_cluster().sync();
+  if (kpart == 0) {
+    for (int i = threadIdx.x; i < 32 * BW; i += blockDim.x) {
+      const int row = rt * kTileRows + i / BW, bt = i % BW;
+      if (row < n && bt < batch) {
+        float tsum = 0.0f;
+        for (int k = 0; k < ksplit; ++k) tsum += part[(size_t)k * 32 * BW + i];
+        if (y_f16) static_cast<__half*>(y)[(size_t)bt * ldy + row] = __float2half_rn(tsum);
+        else static_cast<float*>(y)[(size_t)bt * ldy + row] = tsum;
+      }
+    }
   }
 }
 
-static int fast_ksplit(int n, int m) {
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = getenv("STB_GEMV_KSPLIT");
-    forced = e ? atoi(e) : 0;
-  }
+static int env_int(const char* name) {
+  const char* e = getenv(name);
+  return e ? atoi(e) : 0;
+}
+
+// Launch shape: ksplit CTAs per row tile and warps per CTA, chosen so that a warp gets a run of
+// a few tiles and the grid has several CTAs per SM (small CTAs spread evenly over the 148 SMs).
+static void gemv_shape(int n, int m, int batch, int& ksplit, int& warps) {
+  static int f_ks = -1, f_w = -1;
+  if (f_ks < 0) { f_ks = env_int("STB_GEMV_KSPLIT"); f_w = env_int("STB_GEMV_WARPS"); }
   const int ntile = (n + kTileRows - 1) / kTileRows, nblk = m / kBlock;
+  warps = (f_w == 2 || f_w == 4 || f_w == 8) ? f_w : 4;
   int ks = 1;
-  if (forced == 1 || forced == 2 || forced == 4 || forced == 8) ks = forced;
+  if (f_ks == 1 || f_ks == 2 || f_ks == 4 || f_ks == 8) ks = f_ks;
   else
-    while (ks < 8 && ntile * ks < 444 && nblk / (2 * ks) >= kFastWarps) ks *= 2;
+    while (ks < 8 && ntile * ks < 592 && nblk / (2 * ks) >= 2 * warps) ks *= 2;
   while (ks > 1 && ks > nblk) ks /= 2;
-  return ks;
+  // the activations of a CTA's slice must fit in shared memory
+  while (ks < 8 && (size_t)batch * ((size_t)((nblk + ks - 1) / ks) * 320 + 64) > 96 * 1024) ks *= 2;
+  ksplit = ks;
 }
 
-template <int N>
-static cudaError_t launch_fast(const uint8_t* packed, int n, int m, const __half* x, void* y, int y_f16,
-                               int* dev_status, cudaStream_t s) {
+template <int N, int NB>
+static cudaError_t launch_mma(const uint8_t* packed, int n, int m, const __half* x, int batch, size_t ldx,
+                              void* y, int y_f16, size_t ldy, int* dev_status, cudaStream_t s) {
   const int ntile = (n + kTileRows - 1) / kTileRows, nblk = m / kBlock;
-  const int ksplit = fast_ksplit(n, m);
+  int ksplit, warps;
+  gemv_shape(n, m, batch, ksplit, warps);
   const int bpp = (nblk + ksplit - 1) / ksplit;
-  const size_t smem = 2048 + (size_t)bpp * 512 + (kFastWarps + 8) * 32 * sizeof(float);
-  static bool attr_done[9] = {false};
-  if (smem > 48 * 1024 && !attr_done[N]) {
-    cudaError_t e = cudaFuncSetAttribute(gemv_fast_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  const GemvSmem L = gemv_smem(N, warps, batch, bpp, ksplit, NB);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(gemv_mma_kernel<N, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done[N] = true;
+    attr_done = true;
   }
-  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  if (L.total > 200 * 1024) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(ntile * ksplit), 1, 1);
-  cfg.blockDim = dim3(kFastWarps * 32, 1, 1);
-  cfg.dynamicSmemBytes = smem;
+  cfg.blockDim = dim3((unsigned)(warps * 32), 1, 1);
+  cfg.dynamicSmemBytes = L.total;
   cfg.stream = s;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)ksplit; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemv_fast_kernel<N>, packed, n, m, x, y, y_f16, dev_status, ksplit, bpp);
+  return cudaLaunchKernelEx(&cfg, gemv_mma_kernel<N, NB>, packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status, ksplit, bpp);
 }
 
-// -----------------------------------------------------------------------------------------
+// ------------------------------------------------------------------------------------------
 // General kernel: any N in 1..8, batch <= BT.  One CTA per row tile (32 rows), 8 warps split
-// the blocks, lane = row; position-order decode, x read through L1 (all lanes of a warp read
-// the same address).  Partial sums of the 8 warps are combined in shared memory in a fixed
-// order, so the result is deterministic.
+// the blocks, lane = (g, t); plain position-order decode and fp32 multiply-adds, x read
+// through L1.  The four lanes that share a row combine with shuffles, the 8 warps through
+// shared memory in a fixed order, so the result is deterministic.
 template <int N, int BT>
 __global__ void __launch_bounds__(256)
 gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* __restrict__ x,
@@ -184,56 +339,98 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
     return;
   }
   const int nblk = m / kBlock;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
   const int rt = blockIdx.x;
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
+  const int spb = (int)hdr->spb;
 
-  float acc[BT];
+  float acc[4][BT];
 #pragma unroll
-  for (int t = 0; t < BT; ++t) acc[t] = 0.0f;
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int bt = 0; bt < BT; ++bt) acc[j][bt] = 0.0f;
 
   for (int b = warp; b < nblk; b += 8) {
-    const BlockInfo* bi = binfo + b;
-    RowBlock<N> r;
-    load_rowblock<N>(rtbase + bi->tile_off, lane, (int)bi->res_bytes, r);
-    const uint64_t sal[2] = {bi->salient[0], bi->salient[1]};
-    int tbase = 0;
+    const uint8_t* tile = rtbase + (size_t)b * hdr->tile_bytes;
+    LaneTile<N> lt;
+    load_lane_tile<N>(tile, lane, lt);
+    const uint64_t sal[2] = {binfo[b].salient[0], binfo[b].salient[1]};
 #pragma unroll
-    for (int g = 0; g < 16; ++g) {
-      const uint32_t salb = (uint32_t)((sal[g >> 3] >> (8 * (g & 7))) & 0xFFull);
-      float v[8];
-      decode_group<N>(r, g, salb, tbase, v);
-      tbase += __popc(salb);
+    for (int j = 0; j < 4; ++j) {
+      float alpha[5];
 #pragma unroll
-      for (int t = 0; t < BT; ++t) {
-        if (t < batch) {
-          const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)t * ldx + (size_t)b * kBlock + g * 8));
-          const __half2* xh = reinterpret_cast<const __half2*>(&xv);
+      for (int q = 0; q < 4; ++q) alpha[q] = __half2float(__ushort_as_half((unsigned short)scale_bits<N>(lt, j, q)));
+      alpha[4] = __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(lt, j)));
+#pragma unroll 1
+      for (int s = 0; s < 4; ++s) {
+        const int grp = 4 * s + t;
+        uint32_t code[8], neg[8];
+        plain_slot<N>(lt, 4 * j + s, code, neg);
+        const uint32_t salb = (uint32_t)((sal[grp >> 3] >> (8 * (grp & 7))) & 0xFFull);
+        int qbase = grp >= 8 ? __popcll(sal[0]) : 0;
+        qbase += __popcll(sal[grp >> 3] & ((1ull << (8 * (grp & 7))) - 1ull));
+        float v[8];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const float2 xf = __half22float2(xh[c]);
-            acc[t] = fmaf(v[2 * c], xf.x, acc[t]);
-            acc[t] = fmaf(v[2 * c + 1], xf.y, acc[t]);
+        for (int c = 0; c < 8; ++c) {
+          float w = 0.0f;
+          if (code[c] < 4u) {
+            const float s1 = neg[c] ? -1.0f : 1.0f;
+            if (code[c] == 3u) {
+              const int q = qbase + __popc(salb & ((1u << c) - 1u));
+              const uint32_t word = q < spb ? *reinterpret_cast<const uint32_t*>(tile + resid_word_off(N, spb, g, q >> 2)) : 0x55555555u;
+              const float s2 = resid_code(word, j, q & 3) == 0u ? 1.0f : -1.0f;
+              w = __fadd_rn(s1 * alpha[3], s2 * alpha[4]);
+            } else {
+              w = s1 * (code[c] == 0u ? alpha[0] : (code[c] == 1u ? alpha[1] : alpha[2]));
+            }
+          }
+          v[c] = w;
+        }
+#pragma unroll
+        for (int bt = 0; bt < BT; ++bt) {
+          if (bt < batch) {
+            const uint4 xv = __ldg(reinterpret_cast<const uint4*>(x + (size_t)bt * ldx + (size_t)b * kBlock + grp * 8));
+            const __half2* xh = reinterpret_cast<const __half2*>(&xv);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const float2 xf = __half22float2(xh[c]);
+              acc[j][bt] = fmaf(v[2 * c], xf.x, acc[j][bt]);
+              acc[j][bt] = fmaf(v[2 * c + 1], xf.y, acc[j][bt]);
+            }
           }
         }
       }
     }
   }
 
-  __shared__ float red[8][BT][32];
+  // the four lanes t of a row
 #pragma unroll
-  for (int t = 0; t < BT; ++t) red[warp][t][lane] = acc[t];
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int bt = 0; bt < BT; ++bt) {
+      float a = acc[j][bt];
+      a += __shfl_xor_sync(0xFFFFFFFFu, a, 1);
+      a += __shfl_xor_sync(0xFFFFFFFFu, a, 2);
+      acc[j][bt] = a;
+    }
+  __shared__ float red[8][BT][32];
+  if (t == 0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int bt = 0; bt < BT; ++bt) red[warp][bt][g + 8 * j] = acc[j][bt];
+  }
   __syncthreads();
   for (int idx = threadIdx.x; idx < BT * 32; idx += blockDim.x) {
-    const int t = idx >> 5, l = idx & 31;
+    const int bt = idx >> 5, l = idx & 31;
     const int row = rt * kTileRows + l;
-    if (t < batch && row < n) {
+    if (bt < batch && row < n) {
       float s = 0.0f;
 #pragma unroll
-      for (int w = 0; w < 8; ++w) s += red[w][t][l];
-      if (y_f16) static_cast<__half*>(y)[(size_t)t * ldy + row] = __float2half_rn(s);
-      else static_cast<float*>(y)[(size_t)t * ldy + row] = s;
+      for (int w = 0; w < 8; ++w) s += red[w][bt][l];
+      if (y_f16) static_cast<__half*>(y)[(size_t)bt * ldy + row] = __float2half_rn(s);
+      else static_cast<float*>(y)[(size_t)bt * ldy + row] = s;
     }
   }
 }
@@ -242,8 +439,8 @@ template <int N>
 static cudaError_t launch_general(const uint8_t* packed, int n, int m, const __half* x, int batch,
                                   size_t ldx, void* y, int y_f16, size_t ldy, int* dev_status, cudaStream_t s) {
   const unsigned grid = (unsigned)((n + kTileRows - 1) / kTileRows);
-  if (batch == 1) gemv_general_kernel<N, 1><<<grid, 256, 0, s>>>(packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status);
-  else if (batch <= 4) gemv_general_kernel<N, 4><<<grid, 256, 0, s>>>(packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status);
+  if (batch <= 2) gemv_general_kernel<N, 2><<<grid, 256, 0, s>>>(packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status);
+  else if (batch <= 8) gemv_general_kernel<N, 8><<<grid, 256, 0, s>>>(packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status);
   else gemv_general_kernel<N, 16><<<grid, 256, 0, s>>>(packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status);
   return cudaGetLastError();
 }
@@ -263,10 +460,17 @@ extern "C" int stb_gemv(const void* packed, int n, int m, int N, const void* x, 
   const uint8_t* p = static_cast<const uint8_t*>(packed);
   const __half* xh = static_cast<const __half*>(x);
   cudaError_t e = cudaSuccess;
-  if (batch == 1 && N >= 4 && N <= 6) {
-    if (N == 4) e = stb::launch_fast<4>(p, n, m, xh, y, y_f16, dev_status, s);
-    else if (N == 5) e = stb::launch_fast<5>(p, n, m, xh, y, y_f16, dev_status, s);
-    else e = stb::launch_fast<6>(p, n, m, xh, y, y_f16, dev_status, s);
+  static const bool force_general = stb::env_int("STB_GEMV_GENERAL") != 0;
+  if (N >= 4 && N <= 6 && !force_general) {
+    if (batch <= 8) {
+      if (N == 4) e = stb::launch_mma<4, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+      else if (N == 5) e = stb::launch_mma<5, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+      else e = stb::launch_mma<6, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+    } else {
+      if (N == 4) e = stb::launch_mma<4, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+      else if (N == 5) e = stb::launch_mma<5, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+      else e = stb::launch_mma<6, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+    }
     return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
   }
   switch (N) {

@@ -1,40 +1,59 @@
 // Packed ("streaming") layout of an N:8 structured-binary layer, shared by the CUDA kernels.
+// Plain C++ (no CUDA types) so that the index arithmetic can also be compiled and checked on
+// the host.
 //
-// The unit of the layout is a TILE: 32 output rows x one 128-column block.  Inside a tile
-// every field is stored lane-major (lane = row within the tile) so that a warp reads each
-// field with one fully coalesced vector load per plane:
+// The unit of the layout is a TILE: 32 output rows x one 128-column block; all tiles of a layer
+// have the same size and follow each other in (row tile, block) order after a header and a
+// per-block table.  Inside a tile the work is split the way a warp-level tensor-core
+// instruction (m16n8k16) splits a 16 x 16 operand: lane = 4 g + t  (g = 0..7, t = 0..3) owns
+//     rows    r_j = g + 8 j      (j = 0..3) of the tile and, of each of them,
+//     groups  G_s = 4 s + t      (s = 0..3) of the block (a group = 8 columns),
+// i.e. 16 (row, group) slots  u = 4 j + s,  as many weights as one row of the block.  With
+// this split the 8 decoded fp16 weights of slot (j, s) are exactly the lane's operand
+// registers of two m16n8k16 instructions (columns 32 s + 8 t + 0..7 of rows g + 8 j).
 //
-//   mask    32 x uint4                      16 keep bytes of the row-block (group g = byte g)
-//   region  N words per lane                16 two-bit codes per word, quad-interleaved (below)
-//   sign    N/2 words per lane (+ a half)   32 sign bits per word, pre-positioned (below)
-//   scale   32 x uint2 + 32 x u16           byte-planar: word A = low bytes of the fp16 scales
-//                                           a_dense,a_inter,a_sparse,a_sal1; word B = their
-//                                           high bytes; then a_sal2 as u16
-//   resid   rb byte planes of 32 bytes      residual sign bits of the block's salient columns,
-//                                           rb = ceil(S_b / 8), S_b = salient columns of block
+// Every field is stored lane-major so that a warp reads it with coalesced vector loads:
 //
-// Tile bytes = 512 + 128 N + 64 N + 320 + 32 rb  (50 / 56 / 62 bytes per row-block at
-// N = 4 / 5 / 6, plus rb).  Tiles of one row tile are contiguous in block order; row tiles
-// follow each other with stride rt_stride.  A header and a per-block table come first.
+//   mask    32 x uint4          byte u of the lane's 16 bytes = keep byte of slot u
+//   region  N words per lane    two-bit region codes, 16 per word, of the lane's 16 N kept
+//                               weights: first the "low" part (ranks k < min(N, 4) of every
+//                               slot, weight number wl = u NL + k), then the "high" part
+//                               (ranks 4..N-1, wh = u NH + k - 4).  Inside a word the codes are
+//                               nibble-interleaved (code_bit) so that (R & 0x33333333) and
+//                               ((R >> 2) & 0x33333333) are byte-permute selectors.
+//   sign    N/2 words per lane  one bit per kept weight (1 = negative), same low / high split
+//                               and weight numbering, pre-positioned (sign_bit) so that one
+//                               shift puts the bits of a selector word on bit 2 of its
+//                               nibbles.  An odd part ends in half a word: lanes l and l + 16
+//                               share word l of a 16-word plane (lower lane bits 2,1 of each
+//                               nibble, upper lane bits 3,0).
+//   scale   32 x uint2          per row: word A = low bytes of the fp16 scales a_dense,
+//                               a_inter, a_sparse, a_sal1; word B = their high bytes.  Rows
+//                               are stored in the order p = 4 (r % 8) + r / 8, so that the
+//                               four rows of a lane are contiguous.
+//   sal2    32 x u16            a_sal2 per row, same row order
+//   resid   SPB / 4 words per g residual of the block's salient columns: slot q (the q-th
+//                               salient column, ascending) of row r_j has the two-bit code
+//                               0 = +a_sal2, 2 = -a_sal2, 1 = no term (weight dropped, or
+//                               q >= number of salient columns); word q / 4 of the 8 x SPB/4
+//                               words holds rows r_0..r_3 of g at code_bit(4 j + q % 4).
+//                               SPB (slots per block) is one of 0, 4, 8, 16, 32: the smallest
+//                               that holds the largest salient count of the layer.
 //
-// Kept weights of a row-block are numbered w = g*N + k (g = group 0..15, k = rank of the
-// weight among the kept columns of the group, ascending).  Quad q = w/4, slot j = w%4.
-//   region word w/16: with qq = (w/4)%4 the code sits at bit 4j + 16(qq&1) + 2(qq>>1).
-//     => (R & 0x33333333) holds quads qq=0 (low 16 bits) and qq=1 (high 16 bits) as nibbles,
-//        ((R>>2) & 0x33333333) holds quads qq=2 and qq=3: each nibble is a byte-permute
-//        selector 0..3 into the four scale bytes.
-//   sign word w/32, stored bit = 1 for a NEGATIVE weight: with p = (w/16)%2 the bit sits at
-//     4i + off, i = j + 4(qq&1), off = {2,1,3,0}[2p + (qq>>1)], so that one shift moves the
-//     eight sign bits of a selector word onto bit 2 of its nibbles (the bit that chooses
-//     between the +scale and -scale high bytes).
-//   For odd N the last 16 weights need half a sign word: lanes l and l+16 share word l of a
-//   16-word plane; lane l < 16 uses offsets {2,1}, lane l+16 the same bits moved to {3,0}.
+// Tile bytes = 512 + 192 N + 320 + 8 SPB   (50 / 56 / 62 bytes per row and block at
+// N = 4 / 5 / 6, plus SPB / 4).
 #pragma once
 #include <stdint.h>
 
+#if defined(__CUDACC__)
+#define STB_HD __host__ __device__ __forceinline__
+#else
+#define STB_HD inline
+#endif
+
 namespace stb {
 
-constexpr uint32_t kMagic = 0x31425453u;  // "STB1"
+constexpr uint32_t kMagic = 0x32425453u;  // "STB2"
 constexpr int kBlock = 128;               // columns per block
 constexpr int kGroup = 8;                 // columns per group (M)
 constexpr int kTileRows = 32;
@@ -46,40 +65,47 @@ struct Header {          // 64 bytes at the start of the packed buffer
   int32_t n, m, N;
   int32_t nblk;          // m / 128
   int32_t ntile;         // ceil(n / 32)
-  uint32_t tiles_offset; // byte offset of tile (0,0)
-  uint64_t rt_stride;    // bytes of one row tile (all its blocks)
+  uint32_t tiles_offset; // byte offset of tile (0, 0)
+  uint64_t rt_stride;    // bytes of one row tile = nblk * tile_bytes
   uint64_t used_bytes;
   uint32_t status;       // 0 or STB_ERR_CORRUPT
-  uint32_t max_tile_bytes;
-  uint32_t pad[2];
+  uint32_t tile_bytes;
+  uint32_t spb;          // residual slots per block: 0, 4, 8, 16 or 32
+  uint32_t pad;
 };
 static_assert(sizeof(Header) == 64, "header is 64 bytes");
 
 struct BlockInfo {       // 32 bytes, one per block, right after the header
-  uint64_t salient[2];
-  uint32_t tile_off;     // byte offset of the block's tile inside a row tile
-  uint32_t nsal;         // S_b
-  uint32_t res_bytes;    // rb
-  uint32_t tile_bytes;
+  uint64_t salient[2];   // 128-bit salient-column mask
+  uint32_t nsal;         // number of salient columns
+  uint32_t pad[3];
 };
 static_assert(sizeof(BlockInfo) == 32, "block info is 32 bytes");
 
-__host__ __device__ constexpr uint32_t tile_bytes(int N, int rb) {
-  return 512u + 192u * (uint32_t)N + 320u + 32u * (uint32_t)rb;
+STB_HD constexpr int n_lo(int N) { return N < 4 ? N : 4; }
+STB_HD constexpr int n_hi(int N) { return N > 4 ? N - 4 : 0; }
+STB_HD constexpr int sign_full_words(int N) { return (n_lo(N) >> 1) + (n_hi(N) >> 1); }
+STB_HD constexpr bool sign_has_half(int N) { return (N & 1) != 0; }
+
+STB_HD constexpr uint32_t tile_bytes(int N, int spb) {
+  return 512u + 192u * (uint32_t)N + 320u + 8u * (uint32_t)spb;
 }
-__host__ __device__ constexpr uint32_t tiles_offset(int nblk) {
+STB_HD constexpr uint32_t tiles_offset(int nblk) {
   return (uint32_t)((sizeof(Header) + sizeof(BlockInfo) * (size_t)nblk + 255) / 256 * 256);
 }
-__host__ __device__ constexpr uint32_t off_region(int) { return 512u; }
-__host__ __device__ constexpr uint32_t off_sign(int N) { return 512u + 128u * (uint32_t)N; }
-__host__ __device__ constexpr uint32_t off_scale(int N) { return 512u + 192u * (uint32_t)N; }
-__host__ __device__ constexpr uint32_t off_sal2(int N) { return off_scale(N) + 256u; }
-__host__ __device__ constexpr uint32_t off_resid(int N) { return off_scale(N) + 320u; }
+STB_HD constexpr int spb_for(int max_nsal) {
+  return max_nsal == 0 ? 0 : (max_nsal <= 4 ? 4 : (max_nsal <= 8 ? 8 : (max_nsal <= 16 ? 16 : 32)));
+}
+STB_HD constexpr uint32_t off_region(int) { return 512u; }
+STB_HD constexpr uint32_t off_sign(int N) { return 512u + 128u * (uint32_t)N; }
+STB_HD constexpr uint32_t off_scale(int N) { return 512u + 192u * (uint32_t)N; }
+STB_HD constexpr uint32_t off_sal2(int N) { return off_scale(N) + 256u; }
+STB_HD constexpr uint32_t off_resid(int N) { return off_scale(N) + 320u; }
 
 // Byte offset (inside the tile) of word `iw` of a per-lane field of `nw` words that starts at
 // `base`: the words are laid out as uint4 planes, then (nw & 2) a uint2 plane, then (nw & 1)
 // a u32 plane.
-__host__ __device__ constexpr uint32_t plane_word_off(uint32_t base, int nw, int iw, int lane) {
+STB_HD constexpr uint32_t plane_word_off(uint32_t base, int nw, int iw, int lane) {
   int q4 = nw >> 2;
   if (iw < 4 * q4) return base + (uint32_t)(iw >> 2) * 512u + (uint32_t)lane * 16u + (uint32_t)(iw & 3) * 4u;
   uint32_t o = base + (uint32_t)q4 * 512u;
@@ -89,37 +115,59 @@ __host__ __device__ constexpr uint32_t plane_word_off(uint32_t base, int nw, int
   }
   return o + (uint32_t)lane * 4u;
 }
-__host__ __device__ constexpr uint32_t region_word_off(int N, int iw, int lane) {
+STB_HD constexpr uint32_t region_word_off(int N, int iw, int lane) {
   return plane_word_off(off_region(N), N, iw, lane);
 }
-// full sign words: N/2 per lane; the shared half word (odd N) follows them
-__host__ __device__ constexpr uint32_t sign_word_off(int N, int sw, int lane) {
-  return plane_word_off(off_sign(N), N >> 1, sw, lane);
+STB_HD constexpr uint32_t sign_word_off(int N, int sw, int lane) {
+  return plane_word_off(off_sign(N), sign_full_words(N), sw, lane);
 }
-__host__ __device__ constexpr uint32_t sign_half_off(int N, int lane) {
-  return off_sign(N) + 128u * (uint32_t)(N >> 1) + (uint32_t)(lane & 15) * 4u;
+STB_HD constexpr uint32_t sign_half_off(int N, int lane) {
+  return off_sign(N) + 128u * (uint32_t)sign_full_words(N) + (uint32_t)(lane & 15) * 4u;
+}
+// scale / sal2 / resid are indexed by the permuted row position p = 4 g + j of row g + 8 j
+STB_HD constexpr uint32_t scale_off(int N, int g, int j) { return off_scale(N) + (uint32_t)(4 * g + j) * 8u; }
+STB_HD constexpr uint32_t sal2_off(int N, int g, int j) { return off_sal2(N) + (uint32_t)(4 * g + j) * 2u; }
+STB_HD constexpr uint32_t resid_word_off(int N, int spb, int g, int wq) {
+  return off_resid(N) + ((uint32_t)g * (uint32_t)(spb >> 2) + (uint32_t)wq) * 4u;
 }
 
-// bit position of the 2-bit region code of kept weight w inside region word w/16
-__host__ __device__ constexpr int code_bit(int w) {
-  int j = w & 3, qq = (w >> 2) & 3;
-  return 4 * j + 16 * (qq & 1) + 2 * (qq >> 1);
+// bit position of the two-bit code number i (0..15) of a region word
+STB_HD constexpr int code_bit(int i) {
+  int slot = i & 3, qq = (i >> 2) & 3;
+  return 4 * slot + 16 * (qq & 1) + 2 * (qq >> 1);
 }
-// bit position of the sign bit of kept weight w inside sign word w/32 (lower-lane form for
-// the shared half word)
-__host__ __device__ constexpr int sign_bit(int w) {
-  int j = w & 3, qq = (w >> 2) & 3, p = (w >> 4) & 1;
-  int i = j + 4 * (qq & 1);
+// bit position of sign bit number i (0..31) of a sign word (i < 16: also the lower-lane form
+// of a shared half word)
+STB_HD constexpr int sign_bit(int i) {
+  int slot = i & 3, qq = (i >> 2) & 3, p = (i >> 4) & 1;
+  int nib = slot + 4 * (qq & 1);
   int sel = 2 * p + (qq >> 1);
   int off = sel == 0 ? 2 : (sel == 1 ? 1 : (sel == 2 ? 3 : 0));
-  return 4 * i + off;
+  return 4 * nib + off;
 }
 // shared half word: lower-lane form (offsets 2,1) <-> upper-lane form (offsets 3,0)
-__host__ __device__ constexpr uint32_t half_to_upper(uint32_t h) {
+STB_HD constexpr uint32_t half_to_upper(uint32_t h) {
   return ((h & 0x44444444u) << 1) | ((h & 0x22222222u) >> 1);
 }
-__host__ __device__ constexpr uint32_t half_from_upper(uint32_t s) {
+STB_HD constexpr uint32_t half_from_upper(uint32_t s) {
   return ((s & 0x88888888u) >> 1) | ((s & 0x11111111u) << 1);
+}
+
+// Where the code / sign of the k-th kept weight (ascending column) of slot u lives.
+struct BitPos { int word; int bit; bool half; };
+STB_HD constexpr BitPos region_pos(int N, int u, int k) {
+  const int NL = n_lo(N), NH = n_hi(N);
+  const int w = k < 4 ? u * NL + k : u * NH + (k - 4);
+  return BitPos{(k < 4 ? 0 : NL) + (w >> 4), code_bit(w & 15), false};
+}
+STB_HD constexpr BitPos sign_pos(int N, int u, int k) {
+  const int NL = n_lo(N), NH = n_hi(N);
+  const bool lo = k < 4;
+  const int w = lo ? u * NL + k : u * NH + (k - 4);
+  const int nfull = lo ? (NL >> 1) : (NH >> 1);
+  const int base = lo ? 0 : (NL >> 1);
+  if ((w >> 5) < nfull) return BitPos{base + (w >> 5), sign_bit(w & 31), false};
+  return BitPos{0, sign_bit(w & 15), true};
 }
 
 }  // namespace stb

@@ -2,24 +2,25 @@
 // tile-major streaming layout (stb_layout.cuh), plus the small host-side entry points that
 // need no kernel of their own.  Counterpart of the paper's "matrix compression" and "value
 // compression" steps (Appendix C), generalised to an 8-bit keep mask, N sign bits and 2N region
-// bits per group, five scales per row-block and the residual sign bits of salient columns.
+// bits per group, five scales per row-block and a two-bit residual code per salient column.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 #include "../../include/stb.h"
+#include "stb_decode.cuh"
 #include "stb_layout.cuh"
 
 namespace stb {
 
 // ---------------------------------------------------------------------------------------
-// Header + per-block table.  One CTA; thread 0 does the (short) prefix sum over blocks.
+// Header + per-block table.  One CTA; the salient counts give the residual slots per block.
 __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ salient,
                               uint8_t* __restrict__ packed, int* dev_status) {
   const int nblk = m / kBlock;
   Header* hdr = reinterpret_cast<Header*>(packed);
   BlockInfo* bi = reinterpret_cast<BlockInfo*>(packed + sizeof(Header));
-  __shared__ int bad;
-  if (threadIdx.x == 0) bad = 0;
+  __shared__ int bad, maxsal;
+  if (threadIdx.x == 0) { bad = 0; maxsal = 0; }
   __syncthreads();
   for (int b = threadIdx.x; b < nblk; b += blockDim.x) {
     uint64_t lo = salient[2 * b], hi = salient[2 * b + 1];
@@ -28,29 +29,26 @@ __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ 
     bi[b].salient[0] = lo;
     bi[b].salient[1] = hi;
     bi[b].nsal = (uint32_t)ns;
-    bi[b].res_bytes = (uint32_t)((ns + 7) / 8);
-    bi[b].tile_bytes = tile_bytes(N, (ns + 7) / 8);
+    bi[b].pad[0] = bi[b].pad[1] = bi[b].pad[2] = 0;
+    atomicMax(&maxsal, ns);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    uint32_t off = 0, mx = 0;
-    for (int b = 0; b < nblk; ++b) {
-      bi[b].tile_off = off;
-      off += bi[b].tile_bytes;
-      mx = bi[b].tile_bytes > mx ? bi[b].tile_bytes : mx;
-    }
     const int ntile = (n + kTileRows - 1) / kTileRows;
+    const int spb = spb_for(maxsal);
+    const uint32_t tb = tile_bytes(N, spb);
     hdr->magic = kMagic;
-    hdr->version = 1;
+    hdr->version = 2;
     hdr->n = n; hdr->m = m; hdr->N = N;
     hdr->nblk = nblk;
     hdr->ntile = ntile;
     hdr->tiles_offset = tiles_offset(nblk);
-    hdr->rt_stride = off;
-    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + (uint64_t)off * (uint64_t)ntile;
+    hdr->rt_stride = (uint64_t)tb * (uint64_t)nblk;
+    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + (uint64_t)tb * (uint64_t)nblk * (uint64_t)ntile;
     hdr->status = bad ? (uint32_t)STB_ERR_CORRUPT : 0u;
-    hdr->max_tile_bytes = mx;
-    hdr->pad[0] = hdr->pad[1] = 0;
+    hdr->tile_bytes = tb;
+    hdr->spb = (uint32_t)spb;
+    hdr->pad = 0;
     if (bad && dev_status) *dev_status = STB_ERR_CORRUPT;
   }
 }
@@ -71,16 +69,22 @@ __device__ __forceinline__ void store_planes(uint8_t* tile, uint32_t base, const
   if (NW & 1) *reinterpret_cast<uint32_t*>(tile + o + lane * 4) = w[NW - 1];
 }
 
-// One warp per tile (32 rows x one block); lane = row.  Adjacent warps take adjacent blocks
-// of the same rows, so the 16- and 32-byte pieces each lane reads share sectors with its
-// neighbours in L2.
+// One warp per tile (32 rows x one block).  Phase 1, lane = row: vector loads of the row's
+// logical fields, validation, scales and residual codes; the group fields go to shared
+// memory.  Phase 2, lane = (g, t): each lane collects its 16 (row, group) slots and builds
+// its mask / region / sign words.
+constexpr int kPackWarps = 8;
+
 template <int N>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kPackWarps * 32)
 pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
+  __shared__ uint8_t sm_keep[kPackWarps][32][16];
+  __shared__ uint8_t sm_sign[kPackWarps][32][16];
+  __shared__ uint16_t sm_region[kPackWarps][32][16];
   const int nblk = L.m / kBlock, ngrp = L.m / kGroup;
   const int ntile = (L.n + kTileRows - 1) / kTileRows;
-  const int lane = threadIdx.x & 31;
-  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const long long warp = (long long)blockIdx.x * kPackWarps + wib;
   if (warp >= (long long)ntile * nblk) return;
   const int rt = (int)(warp / nblk), b = (int)(warp % nblk);
   const int row = rt * kTileRows + lane;
@@ -89,10 +93,12 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
   Header* hdr = reinterpret_cast<Header*>(packed);
   const BlockInfo* bi = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header)) + b;
   const uint64_t sal_lo = bi->salient[0], sal_hi = bi->salient[1];
-  const int nsal = (int)bi->nsal, rb = (int)bi->res_bytes;
-  uint8_t* tile = packed + tiles_offset(nblk) + (size_t)rt * (size_t)hdr->rt_stride + bi->tile_off;
+  const int nsal = (int)bi->nsal, spb = (int)hdr->spb;
+  uint8_t* tile = packed + hdr->tiles_offset + ((size_t)rt * nblk + b) * (size_t)hdr->tile_bytes;
 
-  uint32_t keepw[4] = {0, 0, 0, 0}, signw[4] = {0, 0, 0, 0}, regw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  // ---- phase 1: lane = row ----
+  // rows past n: nothing kept, all signs "+", zero scales
+  uint32_t keepw[4] = {0, 0, 0, 0}, signw[4] = {~0u, ~0u, ~0u, ~0u}, regw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   uint32_t s2 = 0;
   uint16_t sc[5] = {0, 0, 0, 0, 0};
   if (valid) {
@@ -110,10 +116,12 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
 #pragma unroll
     for (int q = 0; q < 5; ++q) sc[q] = sp[q];
   }
+  *reinterpret_cast<uint4*>(&sm_keep[wib][lane][0]) = make_uint4(keepw[0], keepw[1], keepw[2], keepw[3]);
+  *reinterpret_cast<uint4*>(&sm_sign[wib][lane][0]) = make_uint4(signw[0], signw[1], signw[2], signw[3]);
+  *reinterpret_cast<uint4*>(&sm_region[wib][lane][0]) = make_uint4(regw[0], regw[1], regw[2], regw[3]);
+  *reinterpret_cast<uint4*>(&sm_region[wib][lane][8]) = make_uint4(regw[4], regw[5], regw[6], regw[7]);
 
   bool bad = false;
-  uint32_t R[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // region words (N used)
-  uint32_t S[4] = {0, 0, 0, 0};               // sign words ((N+1)/2 used, last is the half for odd N)
 #pragma unroll
   for (int g = 0; g < 16; ++g) {
     const uint32_t kb = (keepw[g >> 2] >> (8 * (g & 3))) & 0xFFu;
@@ -124,17 +132,10 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
       if (__popc(kb) != N) bad = true;
       if (N < 8 && ((sb >> N) != 0 || (rg >> (2 * N)) != 0)) bad = true;
     }
+    // region 3 must mark exactly the kept weights of salient columns
     uint32_t c3 = 0;
 #pragma unroll
-    for (int k = 0; k < N; ++k) {
-      const int w = g * N + k;
-      const uint32_t code = (rg >> (2 * k)) & 3u;
-      const uint32_t neg = ((sb >> k) & 1u) ^ 1u;
-      R[w >> 4] |= code << code_bit(w);
-      S[w >> 5] |= (valid ? neg : 0u) << sign_bit(w);
-      c3 |= (code == 3u ? 1u : 0u) << k;
-    }
-    // region 3 must mark exactly the kept weights of salient columns
+    for (int k = 0; k < N; ++k) c3 |= (((rg >> (2 * k)) & 3u) == 3u ? 1u : 0u) << k;
     uint32_t expect = 0, t = kb & salb;
     while (t) {
       const int c = __ffs(t) - 1;
@@ -143,37 +144,64 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
     }
     if (valid && c3 != expect) bad = true;
   }
-  // residual sign bits: none beyond S_b, none on a dropped weight
-  if (valid) {
-    if (nsal < 32 && (s2 >> nsal) != 0) bad = true;
-    int t = 0;
-#pragma unroll 1
-    for (int half = 0; half < 2; ++half) {
-      uint64_t mk = half ? sal_hi : sal_lo;
-      while (mk) {
-        const int c = __ffsll((long long)mk) - 1 + 64 * half;
-        mk &= mk - 1;
-        const uint32_t kbit = (keepw[c >> 5] >> (c & 31)) & 1u;
-        if (!kbit && ((s2 >> t) & 1u)) bad = true;
-        ++t;
-      }
-    }
-  }
 
-  // ---- write the tile, plane by plane (coalesced vector stores) ----
-  *reinterpret_cast<uint4*>(tile + lane * 16) = make_uint4(keepw[0], keepw[1], keepw[2], keepw[3]);
-  store_planes<N>(tile, off_region(N), R, lane);
-  store_planes<N / 2>(tile, off_sign(N), S, lane);
-  if (N & 1) {
-    const uint32_t h = S[N / 2];
-    const uint32_t up = __shfl_down_sync(0xFFFFFFFFu, half_to_upper(h), 16);
-    if (lane < 16) *reinterpret_cast<uint32_t*>(tile + sign_half_off(N, lane)) = h | up;
-  }
+  // scales and a_sal2, stored at the row's permuted position
+  const int pg = lane & 7, pj = lane >> 3;
   const uint32_t A = (sc[0] & 0xFFu) | ((sc[1] & 0xFFu) << 8) | ((sc[2] & 0xFFu) << 16) | ((uint32_t)(sc[3] & 0xFFu) << 24);
   const uint32_t B = (sc[0] >> 8) | ((uint32_t)(sc[1] >> 8) << 8) | ((uint32_t)(sc[2] >> 8) << 16) | ((uint32_t)(sc[3] >> 8) << 24);
-  *reinterpret_cast<uint2*>(tile + off_scale(N) + lane * 8) = make_uint2(A, B);
-  *reinterpret_cast<uint16_t*>(tile + off_sal2(N) + lane * 2) = sc[4];
-  for (int p = 0; p < rb; ++p) tile[off_resid(N) + p * 32 + lane] = (uint8_t)(s2 >> (8 * p));
+  *reinterpret_cast<uint2*>(tile + scale_off(N, pg, pj)) = make_uint2(A, B);
+  *reinterpret_cast<uint16_t*>(tile + sal2_off(N, pg, pj)) = sc[4];
+
+  // residual codes of the block's salient columns: 0 = +a_sal2, 2 = -a_sal2, 1 = no term
+  if (valid && nsal < 32 && (s2 >> nsal) != 0) bad = true;
+  {
+    int q = 0;
+    uint64_t mk = sal_lo;
+    int base = 0;
+    for (int wq = 0; wq < (spb >> 2); ++wq) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t code = 1u;
+        if (mk == 0 && base == 0) { mk = sal_hi; base = 64; }
+        if (mk != 0) {
+          const int c = __ffsll((long long)mk) - 1 + base;
+          mk &= mk - 1;
+          const uint32_t kbit = (keepw[c >> 5] >> (c & 31)) & 1u;
+          const uint32_t sbit = (s2 >> q) & 1u;
+          if (valid && !kbit && sbit) bad = true;      // a residual sign on a dropped weight
+          if (valid && kbit) code = sbit ? 0u : 2u;
+          ++q;
+        }
+        word |= code << code_bit(4 * pj + q4);
+      }
+      word |= __shfl_xor_sync(0xFFFFFFFFu, word, 8);
+      word |= __shfl_xor_sync(0xFFFFFFFFu, word, 16);
+      if (lane < 8) *reinterpret_cast<uint32_t*>(tile + resid_word_off(N, spb, lane, wq)) = word;
+    }
+  }
+  __syncwarp();
+
+  // ---- phase 2: lane = (g, t) ----
+  const int g = lane >> 2, t = lane & 3;
+  uint32_t maskw[4] = {0, 0, 0, 0}, sgn[16], reg[16];
+#pragma unroll
+  for (int u = 0; u < 16; ++u) {
+    const int j = u >> 2, sidx = u & 3;
+    const int r = g + 8 * j, grp = 4 * sidx + t;
+    maskw[j] |= (uint32_t)sm_keep[wib][r][grp] << (8 * sidx);
+    sgn[u] = sm_sign[wib][r][grp];
+    reg[u] = sm_region[wib][r][grp];
+  }
+  LaneWords<N> w;
+  build_lane_words<N>(sgn, reg, true, w);
+  *reinterpret_cast<uint4*>(tile + lane * 16) = make_uint4(maskw[0], maskw[1], maskw[2], maskw[3]);
+  store_planes<N>(tile, off_region(N), w.R, lane);
+  store_planes<LaneTile<N>::kFull>(tile, off_sign(N), w.S, lane);
+  if (sign_has_half(N)) {
+    const uint32_t up = __shfl_down_sync(0xFFFFFFFFu, half_to_upper(w.half), 16);
+    if (lane < 16) *reinterpret_cast<uint32_t*>(tile + sign_half_off(N, lane)) = w.half | up;
+  }
 
   if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) {
     hdr->status = (uint32_t)STB_ERR_CORRUPT;
@@ -185,8 +213,8 @@ template <int N>
 static cudaError_t launch_pack(const stb_logical& L, uint8_t* packed, int* dev_status,
                                cudaStream_t s) {
   const long long tiles = (long long)((L.n + kTileRows - 1) / kTileRows) * (L.m / kBlock);
-  const unsigned grid = (unsigned)((tiles + 7) / 8);
-  pack_kernel<N><<<grid, 256, 0, s>>>(L, packed, dev_status);
+  const unsigned grid = (unsigned)((tiles + kPackWarps - 1) / kPackWarps);
+  pack_kernel<N><<<grid, kPackWarps * 32, 0, s>>>(L, packed, dev_status);
   return cudaGetLastError();
 }
 
@@ -199,7 +227,7 @@ extern "C" int stb_pack_size(int n, int m, int N, size_t* bytes) {
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
   const size_t nblk = (size_t)m / stb::kBlock, ntile = ((size_t)n + 31) / 32;
-  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * (size_t)stb::tile_bytes(N, 4);
+  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * (size_t)stb::tile_bytes(N, stb::kMaxSalient);
   return STB_OK;
 }
 

@@ -1,0 +1,168 @@
+// Host-only check of the packed layout and of the byte-permute decode (compiled with nvcc, run
+// on the CPU, no GPU needed).  For random tiles it packs the logical fields with the same
+// build_lane_words the pack kernel uses, then checks that
+//   * plain_slot returns every kept weight's region code and sign at the right column,
+//   * FastRows::slot (N = 4, 5, 6) returns, for every column, the 16-bit pattern of the signed
+//     scale of the weight's region, or zero for a dropped column,
+//   * the residual selectors return the stored two-bit codes.
+// Expected values come from the logical fields directly (the definition of the format), not
+// from any packed-side code.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <vector>
+
+#include "../paper_2408_01803_b200/csrc/stb_decode.cuh"
+
+using namespace stb;
+
+static uint64_t rng_state = 0x9E3779B97F4A7C15ull;
+static uint32_t rnd() {
+  rng_state ^= rng_state << 13; rng_state ^= rng_state >> 7; rng_state ^= rng_state << 17;
+  return (uint32_t)(rng_state >> 24);
+}
+
+static uint8_t random_mask(int N) {
+  uint8_t m = 0;
+  int k = 0;
+  while (k < N) {
+    int c = rnd() % 8;
+    if (!((m >> c) & 1)) { m |= (uint8_t)(1 << c); ++k; }
+  }
+  return m;
+}
+
+template <int N>
+static int check(int trials, int spb) {
+  int errors = 0;
+  for (int trial = 0; trial < trials; ++trial) {
+    // logical tile: 32 rows x 16 groups
+    uint8_t keep[32][16], sign[32][16];
+    uint16_t region[32][16], scale[32][5];
+    uint8_t rcode[32][32];
+    for (int r = 0; r < 32; ++r) {
+      for (int g = 0; g < 16; ++g) {
+        keep[r][g] = random_mask(N);
+        sign[r][g] = (uint8_t)(rnd() & ((1u << N) - 1u));
+        uint16_t rg = 0;
+        for (int k = 0; k < N; ++k) rg |= (uint16_t)((rnd() & 3u) << (2 * k));
+        region[r][g] = rg;
+      }
+      for (int q = 0; q < 5; ++q) scale[r][q] = (uint16_t)(rnd() & 0x7FFFu);
+      for (int q = 0; q < 32; ++q) rcode[r][q] = q < spb ? (uint8_t)(rnd() % 3) : 1;
+    }
+    const uint32_t tb = tile_bytes(N, spb);
+    std::vector<uint8_t> tile(tb + 64, 0);
+    auto put32 = [&](uint32_t off, uint32_t v) { std::memcpy(&tile[off], &v, 4); };
+    auto or32 = [&](uint32_t off, uint32_t v) { uint32_t o; std::memcpy(&o, &tile[off], 4); o |= v; std::memcpy(&tile[off], &o, 4); };
+    for (int lane = 0; lane < 32; ++lane) {
+      const int g = lane >> 2, t = lane & 3;
+      uint32_t sg[16], rg[16], maskw[4] = {0, 0, 0, 0};
+      for (int u = 0; u < 16; ++u) {
+        const int j = u >> 2, s = u & 3, r = g + 8 * j, grp = 4 * s + t;
+        maskw[j] |= (uint32_t)keep[r][grp] << (8 * s);
+        sg[u] = sign[r][grp]; rg[u] = region[r][grp];
+      }
+      LaneWords<N> w;
+      build_lane_words<N>(sg, rg, true, w);
+      for (int j = 0; j < 4; ++j) put32(lane * 16 + 4 * j, maskw[j]);
+      for (int i = 0; i < N; ++i) put32(region_word_off(N, i, lane), w.R[i]);
+      for (int i = 0; i < sign_full_words(N); ++i) put32(sign_word_off(N, i, lane), w.S[i]);
+      if (sign_has_half(N)) or32(sign_half_off(N, lane), lane < 16 ? w.half : half_to_upper(w.half));
+    }
+    for (int r = 0; r < 32; ++r) {
+      const int g = r & 7, j = r >> 3;
+      uint32_t A = 0, B = 0;
+      for (int q = 0; q < 4; ++q) { A |= (uint32_t)(scale[r][q] & 0xFF) << (8 * q); B |= (uint32_t)(scale[r][q] >> 8) << (8 * q); }
+      put32(scale_off(N, g, j), A); put32(scale_off(N, g, j) + 4, B);
+      std::memcpy(&tile[sal2_off(N, g, j)], &scale[r][4], 2);
+      for (int q = 0; q < spb; ++q) or32(resid_word_off(N, spb, g, q >> 2), (uint32_t)rcode[r][q] << code_bit(4 * j + (q & 3)));
+    }
+    // every offset must stay inside the tile
+    if (off_resid(N) + 8u * spb != tb) { ++errors; std::printf("N=%d tile size mismatch\n", N); }
+
+    for (int lane = 0; lane < 32; ++lane) {
+      const int g = lane >> 2, t = lane & 3;
+      LaneTile<N> lt;
+      load_lane_tile<N>(tile.data(), lane, lt);
+      for (int u = 0; u < 16; ++u) {
+        const int j = u >> 2, s = u & 3, r = g + 8 * j, grp = 4 * s + t;
+        uint32_t code[8], neg[8];
+        plain_slot<N>(lt, u, code, neg);
+        int k = 0;
+        for (int c = 0; c < 8; ++c) {
+          uint32_t wc = 4, wn = 0;
+          if ((keep[r][grp] >> c) & 1) {
+            wc = (region[r][grp] >> (2 * k)) & 3u;
+            wn = ((sign[r][grp] >> k) & 1u) ^ 1u;
+            ++k;
+          }
+          if (code[c] != wc || neg[c] != wn) {
+            if (++errors < 10) std::printf("plain N=%d lane %d u %d c %d: got (%u,%u) want (%u,%u)\n", N, lane, u, c, code[c], neg[c], wc, wn);
+          }
+        }
+      }
+      for (int j = 0; j < 4; ++j) {
+        const int r = g + 8 * j;
+        for (int q = 0; q < 4; ++q)
+          if (scale_bits<N>(lt, j, q) != scale[r][q]) { if (++errors < 10) std::printf("scale N=%d\n", N); }
+        if (sal2_bits<N>(lt, j) != scale[r][4]) { if (++errors < 10) std::printf("sal2 N=%d\n", N); }
+        for (int q = 0; q < spb; ++q) {
+          uint32_t word;
+          std::memcpy(&word, &tile[resid_word_off(N, spb, g, q >> 2)], 4);
+          if (resid_code(word, j, q & 3) != rcode[r][q]) { if (++errors < 10) std::printf("resid code N=%d\n", N); }
+          if (((resid_selector(word, j) >> (4 * (q & 3))) & 0xFu) != rcode[r][q]) { if (++errors < 10) std::printf("resid selector N=%d\n", N); }
+        }
+      }
+      if constexpr (N >= 4 && N <= 6) {
+        FastRows<N> fr;
+        fr.init(lt, lt.A, lt.B);
+        for (int j = 0; j < 4; ++j) {
+          uint32_t XL = 0, XH = 0;
+          if (N == 5) fr.high(j, 0, XL, XH);
+          for (int s = 0; s < 4; ++s) {
+            if (N == 6 && (s & 1) == 0) fr.high(j, s >> 1, XL, XH);
+            const int r = g + 8 * j, grp = 4 * s + t;
+            const uint32_t kb = keep_byte_of(lt.mask, j, s);
+            if (kb != keep[r][grp]) { if (++errors < 10) std::printf("keep byte N=%d\n", N); }
+            uint32_t f[4];
+            fr.slot(j, s, position_selector(kb), XL, XH, f);
+            int k = 0;
+            for (int c = 0; c < 8; ++c) {
+              uint32_t want = 0;
+              if ((keep[r][grp] >> c) & 1) {
+                const uint32_t code = (region[r][grp] >> (2 * k)) & 3u;
+                const uint32_t ng = ((sign[r][grp] >> k) & 1u) ^ 1u;
+                want = scale[r][code] ^ (ng << 15);
+                ++k;
+              }
+              const uint32_t got = (f[c >> 1] >> (16 * (c & 1))) & 0xFFFFu;
+              if (got != want) {
+                if (++errors < 10) std::printf("fast N=%d lane %d j %d s %d c %d: got %04x want %04x\n", N, lane, j, s, c, got, want);
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+  return errors;
+}
+
+int main() {
+  int e = 0;
+  e += check<1>(4, 0); e += check<2>(4, 4); e += check<3>(4, 8); e += check<4>(8, 4); e += check<5>(8, 16);
+  e += check<6>(8, 32); e += check<7>(4, 4); e += check<8>(4, 0); e += check<4>(2, 0); e += check<6>(2, 8);
+  // position selector: rank of each kept column, 7 for dropped ones
+  for (uint32_t m = 0; m < 256; ++m) {
+    const uint32_t p = position_selector(m);
+    int r = 0;
+    for (int c = 0; c < 8; ++c) {
+      const uint32_t nib = (p >> (4 * c)) & 0xFu;
+      if ((m >> c) & 1u) { if (nib != (uint32_t)(r & 7)) ++e; ++r; }
+      else if (nib != 7u) ++e;
+    }
+  }
+  std::printf("%s: %d errors\n", e ? "FAIL" : "OK", e);
+  return e ? 1 : 0;
+}

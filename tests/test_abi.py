@@ -29,12 +29,13 @@ def test_every_declared_symbol_is_exported(stb):
 
 
 def test_pack_size_formula_and_errors(stb):
-    # 50 / 56 / 62 bytes per row-block at 4:8 / 5:8 / 6:8 plus at most 4 residual bytes
+    # 50 / 56 / 62 bytes per row-block at 4:8 / 5:8 / 6:8 plus at most 8 residual bytes
+    # (two bits for each of up to 32 salient columns)
     for N, per in ((4, 50), (5, 56), (6, 62)):
         n, m = 4096, 4096
         hdr = (64 + 32 * (m // 128) + 255) // 256 * 256
-        assert stb.pack_size(n, m, N) == hdr + (n // 32) * (m // 128) * 32 * (per + 4)
-    assert stb.pack_size(33, 128, 4) == 256 + 2 * 32 * 54      # ragged rows pad to a tile of 32
+        assert stb.pack_size(n, m, N) == hdr + (n // 32) * (m // 128) * 32 * (per + 8)
+    assert stb.pack_size(33, 128, 4) == 256 + 2 * 32 * 58      # ragged rows pad to a tile of 32
     for args, code in (((0, 128, 4), stb.STB_ERR_SHAPE), ((8, 100, 4), stb.STB_ERR_SHAPE),
                        ((8, 0, 4), stb.STB_ERR_SHAPE), ((8, 128, 0), stb.STB_ERR_NM), ((8, 128, 9), stb.STB_ERR_NM)):
         with pytest.raises(stb.StbError) as e:
@@ -65,3 +66,18 @@ def test_host_side_argument_checks_launch_nothing(stb):
     assert lib.stb_dequant(one, 32, 128, 4, one, stb.STB_F32, 64, null) == stb.STB_ERR_ARG
     assert lib.stb_layer_stack(None, 1, null, null) == stb.STB_ERR_ARG
     assert stb.status_str(stb.STB_ERR_TIMEOUT).startswith("a bounded")
+
+
+def test_packed_layout_and_byte_permute_decode_on_the_host(tmp_path):
+    """tests/host_layout_check.cu: the layout's index arithmetic, the pack-side word builder and the
+    byte-permute decode used by the tensor-core kernels, compiled for the host and checked against the
+    logical fields for N = 1..8."""
+    import shutil
+    import subprocess
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    exe = str(tmp_path / "host_layout_check")
+    subprocess.check_call([nvcc, "-std=c++17", "-O1", "-Wno-deprecated-gpu-targets", "-o", exe,
+                           os.path.join(ROOT, "tests", "host_layout_check.cu")])
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0, out.stdout[-2000:]
+    assert "OK: 0 errors" in out.stdout

@@ -83,9 +83,9 @@ def test_full_size_layers_sampled_rows(stb, N, n, m):
     layer = stb.pack_numpy(d)
     info = layer.info()
     assert info["status"] == 0
-    nres = sum(-(-bin(int(a) | (int(b) << 64)).count("1") // 8) for a, b in d["salient"])
-    per = {4: 50, 5: 56, 6: 62}[N]
-    assert info["stream_bytes"] == (n // 32) * 32 * (per * (m // 128) + nres)
+    # residual field: two bits per slot, 4 slots per block here (at most 3 salient columns)
+    per = {4: 50, 5: 56, 6: 62}[N] + 1
+    assert info["stream_bytes"] == (n // 32) * 32 * per * (m // 128)
     g = np.random.default_rng(N)
     rows = np.sort(g.choice(n, size=192, replace=False)).astype(np.int32)
     rows[:4] = [0, 1, n - 2, n - 1]
@@ -102,6 +102,24 @@ def test_full_size_layers_sampled_rows(stb, N, n, m):
     sub = oracle.Logical(len(rows), m, N, d["keep"][rows].copy(), d["sign"][rows].copy(), d["region"][rows].copy(),
                          d["sign2"][rows].copy(), d["salient"], d["scale"][rows].copy())
     assert np.array_equal(Wg[torch.from_numpy(rows.astype(np.int64)).cuda()].cpu().numpy(), oracle.decode(sub))
+
+
+@pytest.mark.parametrize("N,max_salient", [(4, 7), (5, 14), (6, 30), (6, 32), (3, 20)])
+def test_many_salient_columns(stb, N, max_salient):
+    """Blocks with up to 8 / 16 / 32 salient columns use the wider residual fields."""
+    import torch
+    n, m = 70, 512
+    d = si.logical_layer(n, m, N, 400 + max_salient, max_salient=max_salient)
+    L = oracle.Logical(**d)
+    What = oracle.decode(L)
+    layer = stb.pack_numpy(d)
+    assert layer.info()["status"] == 0
+    most = max(bin(int(a) | (int(b) << 64)).count("1") for a, b in d["salient"])
+    spb = 4 if most <= 4 else 8 if most <= 8 else 16 if most <= 16 else 32
+    assert layer.info()["stream_bytes"] == 96 * 4 * (26 + 6 * N + spb // 4)
+    assert np.array_equal(stb.dequant(layer).cpu().numpy(), What)
+    for batch in (1, 5, 8, 13):
+        _check_gemv(stb, layer, What, m, batch, 30 + batch)
 
 
 def test_pack_flags_corrupt_layers(stb):
