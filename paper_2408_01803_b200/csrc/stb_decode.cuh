@@ -39,7 +39,7 @@ STB_HD uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
 template <int N>
 struct LaneTile {
   static constexpr int kFull = sign_full_words(N);
-  uint32_t mask[4];                     // word j = row g + 8 j: byte s = keep byte of group 4 s + t
+  uint32_t mask[4];                     // word j = row g + 8 j: byte s = keep-mask index of group 4 s + t
   uint32_t R[N];                        // region words (low part, then high part)
   uint32_t S[kFull > 0 ? kFull : 1];    // full sign words (low part, then high part)
   uint32_t half;                        // shared half sign word, already in lower-lane form
@@ -133,7 +133,7 @@ STB_HD void build_lane_words(const uint32_t (&sign)[16], const uint32_t (&region
 template <int N>
 STB_HD void plain_slot(const LaneTile<N>& t, int u, uint32_t (&out_code)[8], uint32_t (&out_neg)[8]) {
   const int j = u >> 2, s = u & 3;
-  const uint32_t kb = (t.mask[j] >> (8 * s)) & 0xFFu;
+  const uint32_t kb = mask_from_index(N, (t.mask[j] >> (8 * s)) & 0xFFu);
   int k = 0;
   for (int c = 0; c < 8; ++c) {
     out_code[c] = 4u; out_neg[c] = 0u;
@@ -207,6 +207,10 @@ struct FastRows {
   // Slot (j, s) -> f[0..3]: columns (0,1), (2,3), (4,5), (6,7) as 16-bit pairs (low half =
   // lower column).  P = position selector of the slot's keep byte.
   STB_HD void slot(int j, int s, uint32_t P, uint32_t XL, uint32_t XH, uint32_t (&f)[4]) const {
+    slot2(j, s, P, P >> 16, XL, XH, f);
+  }
+  // same, with the selectors of columns 0..3 (P0) and 4..7 (P1) in separate words
+  STB_HD void slot2(int j, int s, uint32_t P0, uint32_t P1, uint32_t XL, uint32_t XH, uint32_t (&f)[4]) const {
     const uint32_t sel = ((s & 2) ? o[j] : e[j]) >> (16 * (s & 1));
     const uint32_t lo0 = prmt(A[j], A[j], sel), hi0 = prmt(Bp[j], Bn[j], sel);
     uint32_t lo1 = 0, hi1 = 0;
@@ -217,9 +221,8 @@ struct FastRows {
       lo1 = prmt(XL, 0u, 0x4440u + (uint32_t)s);
       hi1 = prmt(XH, 0u, 0x4440u + (uint32_t)s);
     }
-    const uint32_t P1 = P >> 16;
-    const uint32_t pl0 = prmt(lo0, lo1, P), pl1 = prmt(lo0, lo1, P1);
-    const uint32_t ph0 = prmt(hi0, hi1, P), ph1 = prmt(hi0, hi1, P1);
+    const uint32_t pl0 = prmt(lo0, lo1, P0), pl1 = prmt(lo0, lo1, P1);
+    const uint32_t ph0 = prmt(hi0, hi1, P0), ph1 = prmt(hi0, hi1, P1);
     f[0] = prmt(pl0, ph0, 0x5140u);
     f[1] = prmt(pl0, ph0, 0x7362u);
     f[2] = prmt(pl1, ph1, 0x5140u);
@@ -237,7 +240,8 @@ STB_HD uint32_t position_selector(uint32_t keep_byte) {
   }
   return p;
 }
-STB_HD uint32_t keep_byte_of(const uint32_t (&mask)[4], int j, int s) {
+// keep-mask index of slot (j, s)
+STB_HD uint32_t keep_index_of(const uint32_t (&mask)[4], int j, int s) {
   return prmt(mask[j], 0u, 0x4440u + (uint32_t)s);
 }
 

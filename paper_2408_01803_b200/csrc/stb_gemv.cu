@@ -23,37 +23,34 @@ namespace stb {
 // slice.  Each warp streams its tiles from HBM into a private ring in shared memory with 1-D
 // bulk copies (kDepth tiles in flight), reads a tile into registers, decodes it slot by slot
 // into fp16 operand registers (stb_decode.cuh) and multiplies with m16n8k16 tensor-core
-// instructions: A = 16 rows x 16 columns of W^, B = the staged activations (8 batch rows),
-// fp32 accumulators in registers for the whole run.  The residual term of the salient columns
-// goes through the same instruction, with the salient slots of 16 / SPB blocks as its K
-// dimension.  Partial sums: warps through shared memory, CTAs of the cluster through
-// distributed shared memory, both in a fixed order.
+// instructions: A = 16 rows x 16 columns of W^, B = the activations (8 batch rows), read
+// through L1 (they are shared by every CTA of the SM), fp32 accumulators in registers for the
+// whole run.  The residual term of the salient columns goes through the same instruction, with
+// the salient slots of 16 / SPB blocks as its K dimension.  Partial sums: warps through shared
+// memory, CTAs of the cluster through distributed shared memory, both in a fixed order.
 constexpr int kDepth = 4;
 constexpr long long kWaitLimit = 2000000000ll;     // about a second of SM clocks
 
 struct GemvSmem {
-  uint32_t bars, xs, xsal, ring, part, total;       // byte offsets
-  uint32_t xstride, tile_stride;
+  uint32_t bars, ring, part, total;                 // byte offsets
+  uint32_t tile_stride;
 };
-__host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int batch, int bpp, int ksplit, int NB) {
+__host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int ksplit, int NB) {
   GemvSmem s;
-  s.bars = 1024;
-  s.xs = s.bars + (uint32_t)(warps * kDepth * 8);
-  s.xs = (s.xs + 15u) & ~15u;
-  s.xstride = (uint32_t)bpp * 256u + 64u;
-  s.xsal = s.xs + (uint32_t)batch * s.xstride;
-  s.ring = s.xsal + (uint32_t)batch * (uint32_t)bpp * 64u;
-  s.ring = (s.ring + 127u) & ~127u;
-  s.tile_stride = (tile_bytes(N, kMaxSalient) + 127u) & ~127u;
+  s.bars = kPosTableEntries * 8;                     // the position table comes first
+  s.ring = (s.bars + (uint32_t)(warps * kDepth * 8) + 127u) & ~127u;
+  s.tile_stride = (tile_bytes(N) + 127u) & ~127u;
   s.part = s.ring + (uint32_t)(warps * kDepth) * s.tile_stride;
   s.total = s.part + (uint32_t)ksplit * 32u * 8u * (uint32_t)NB * 4u;
   return s;
 }
 
+__device__ __forceinline__ int ilog2(int v) { return 31 - __clz(v); }
+
 template <int N, int NB>
 __global__ void __launch_bounds__(256)
 gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* __restrict__ x, int batch,
-                size_t ldx, void* __restrict__ y, int y_f16, size_t ldy, int* dev_status, int ksplit, int bpp) {
+                size_t ldx, void* __restrict__ y, int y_f16, size_t ldy, int* dev_status, int lg_ksplit, int bpp) {
   extern __shared__ __align__(128) uint8_t smem[];
   const Header* hdr = reinterpret_cast<const Header*>(packed);
   // every CTA of a cluster takes the same branch here (the header is the same for all)
@@ -62,20 +59,21 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
     return;
   }
   const int nblk = m / kBlock;
+  const int ksplit = 1 << lg_ksplit;
   const int warps = (int)(blockDim.x >> 5);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
-  const int kpart = (int)(blockIdx.x % (unsigned)ksplit), rt = (int)(blockIdx.x / (unsigned)ksplit);
+  const int kpart = (int)(blockIdx.x & (unsigned)(ksplit - 1)), rt = (int)(blockIdx.x >> lg_ksplit);
   const int b0 = kpart * bpp, b1 = min(nblk, b0 + bpp);
   const int nbp = max(b1 - b0, 0);
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
-  const uint32_t tbytes = hdr->tile_bytes;
+  constexpr uint32_t tbytes = tile_bytes(N);
   const int spb = (int)hdr->spb;
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
-  const GemvSmem L = gemv_smem(N, warps, batch, bpp, ksplit, NB);
+  const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)hdr->ntile +
+                            (size_t)rt * nblk * resid_tile_bytes(spb);
+  const GemvSmem L = gemv_smem(N, warps, ksplit, NB);
 
-  uint32_t* ptab = reinterpret_cast<uint32_t*>(smem);
-  uint8_t* xs = smem + L.xs;
-  __half* xsal = reinterpret_cast<__half*>(smem + L.xsal);
+  const uint2* ptab = reinterpret_cast<const uint2*>(smem);
   uint8_t* ring = smem + L.ring + (size_t)warp * kDepth * L.tile_stride;
   const uint32_t bar0 = smem_u32(smem + L.bars) + (uint32_t)warp * kDepth * 8u;
 
@@ -84,7 +82,8 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
   const int wb0 = b0 + warp * per, wb1 = min(b1, wb0 + per);
   const int cnt = max(wb1 - wb0, 0);
 
-  // start the weight stream before anything else
+  // Start the weight stream before anything else.  The packed layer is never written by a GEMV,
+  // so under a programmatic dependent launch this may run while the previous layer still computes.
   if (lane == 0) {
     for (int i = 0; i < kDepth; ++i) mbar_init(bar0 + 8u * i, 1);
     fence_async_smem();
@@ -93,32 +92,13 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
       bulk_g2s(smem_u32(ring + (size_t)i * L.tile_stride), rtbase + (size_t)(wb0 + i) * tbytes, tbytes, bar0 + 8u * i);
     }
   }
+  for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x) reinterpret_cast<uint2*>(smem)[i] = g_pos_table.v[N][i];
 
-  // stage the activations of this CTA's columns, the salient-column activations and the table
-  for (int i = threadIdx.x; i < 256; i += blockDim.x) ptab[i] = g_pos_table.v[i];
-  for (int bt = 0; bt < batch; ++bt) {
-    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)bt * ldx + (size_t)b0 * kBlock);
-    uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)bt * L.xstride);
-    for (int i = threadIdx.x; i < nbp * 16; i += blockDim.x) dst[i] = __ldg(src + i);
-  }
-  if (spb > 0) {
-    for (int i = threadIdx.x; i < nbp * batch; i += blockDim.x) {
-      const int bl = i % nbp, bt = i / nbp;
-      const BlockInfo* bi = binfo + b0 + bl;
-      __half* dst = xsal + ((size_t)bt * bpp + bl) * spb;
-      const __half* xr = x + (size_t)bt * ldx + (size_t)(b0 + bl) * kBlock;
-      int q = 0;
-      for (int h = 0; h < 2; ++h) {
-        uint64_t mk = bi->salient[h];
-        while (mk && q < spb) {
-          const int c = __ffsll((long long)mk) - 1 + 64 * h;
-          mk &= mk - 1;
-          dst[q++] = xr[c];
-        }
-      }
-      for (; q < spb; ++q) dst[q] = __ushort_as_half((unsigned short)0);
-    }
-  }
+  // Everything below reads the activations (the previous layer's output) or writes y: wait for the
+  // previous grid of the stream to have completed (no-op without a programmatic launch), then let
+  // the next grid start its own weight stream.
+  grid_dependency_wait();
+  grid_launch_dependents();
   __syncthreads();
 
   float acc[2][NB][4];
@@ -129,32 +109,37 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
 #pragma unroll
       for (int d = 0; d < 4; ++d) acc[a][c][d] = 0.0f;
 
-  // residual bookkeeping: 16 / SPB blocks share one residual instruction (K = 16 salient slots)
-  const int bpr = spb == 0 ? 1 : (spb >= 16 ? 1 : 16 / spb);     // blocks per residual instruction
-  const int wpb = spb >= 16 ? 4 : (spb >> 2);                     // words of a block per instruction
+  // Residual bookkeeping: 16 / SPB blocks share one residual instruction (K = 16 salient slots):
+  // lane t keeps the residual word of block (it % bpr) == t / wpb, word t % wpb of that block.
+  const int lg_bpr = spb == 0 || spb >= 16 ? 0 : 4 - ilog2(spb);          // blocks per residual instruction
+  const int lg_wpb = spb >= 16 ? 2 : (spb == 8 ? 1 : 0);                  // words of a block per instruction
+  const int bpr_mask = (1 << lg_bpr) - 1;
+  const int my_pos = t >> lg_wpb, my_wq = t & ((1 << lg_wpb) - 1);
+  const uint32_t my_resid_off = spb > 0 ? resid_word_off(spb, g, my_wq) : 0u;
   uint32_t rword = 0x55555555u, rword2 = 0x55555555u, rsal0 = 0, rsal1 = 0;
-  int rblk = 0;
+  int rblk = b0;
   bool failed = false;
+  const __half* xrow[NB];
+#pragma unroll
+  for (int c = 0; c < NB; ++c) xrow[c] = g + 8 * c < batch ? x + (size_t)(g + 8 * c) * ldx + t * 8 : nullptr;
 
   for (int it = 0; it < cnt; ++it) {
-    const int slot = it % kDepth;
+    const int slot = it & (kDepth - 1);
     const uint32_t bar = bar0 + 8u * slot;
+    const int b = wb0 + it;
+    const bool mine = spb > 0 && (it & bpr_mask) == my_pos;
+    if (mine) {
+      const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb) + my_resid_off;
+      rword = __ldg(reinterpret_cast<const uint32_t*>(rp));
+      if (spb == 32) rword2 = __ldg(reinterpret_cast<const uint32_t*>(rp + 16));
+      rblk = b;
+    }
     // all lanes poll; the verdict is made warp-uniform so that nobody is left at a __syncwarp
     if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(it / kDepth) & 1u, kWaitLimit))) { failed = true; break; }
     const uint8_t* tile = ring + (size_t)slot * L.tile_stride;
     LaneTile<N> lt;
     load_lane_tile<N>(tile, lane, lt);
-    const int b = wb0 + it;
-    if (spb > 0) {
-      const int pos = it % bpr;
-      if (bpr == 1 || t / wpb == pos) {
-        const int wq = bpr == 1 ? t : t % wpb;
-        rword = *reinterpret_cast<const uint32_t*>(tile + resid_word_off(N, spb, g, wq));
-        if (spb == 32) rword2 = *reinterpret_cast<const uint32_t*>(tile + resid_word_off(N, spb, g, wq + 4));
-        rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1];
-        rblk = b - b0;
-      }
-    }
+    if (mine) { rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1]; }
     __syncwarp();
     if (lane == 0 && it + kDepth < cnt) {          // refill the slot that was just read
       fence_async_smem();
@@ -169,21 +154,20 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
 #pragma unroll
       for (int j = 0; j < 4; ++j) fr.high(j, 0, XL[j], XH[j]);
     }
-    const uint8_t* xb = xs + (size_t)(b - b0) * 256 + t * 16;
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
       uint4 xf[NB];
 #pragma unroll
       for (int c = 0; c < NB; ++c) {
         xf[c] = make_uint4(0, 0, 0, 0);
-        if (g + 8 * c < batch) xf[c] = *reinterpret_cast<const uint4*>(xb + (size_t)(g + 8 * c) * L.xstride + s * 64);
+        if (xrow[c]) xf[c] = ldg_nc_v4(xrow[c] + (size_t)b * kBlock + s * 32);
       }
       uint32_t f[4][4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         if (N == 6 && (s & 1) == 0) fr.high(j, s >> 1, XL[j], XH[j]);
-        const uint32_t P = ptab[keep_byte_of(lt.mask, j, s)];
-        fr.slot(j, s, P, XL[j], XH[j], f[j]);
+        const uint2 P = ptab[keep_index_of(lt.mask, j, s)];
+        fr.slot2(j, s, P.x, P.y, XL[j], XH[j], f[j]);
       }
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt)
@@ -194,12 +178,11 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
         }
     }
 
-    // residual term: once the salient slots of `bpr` blocks are collected (or at the end)
-    if (spb > 0 && ((it % bpr) == bpr - 1 || it == cnt - 1)) {
+    // residual term: once the salient slots of 16 / SPB blocks are collected (or at the end)
+    if (spb > 0 && ((it & bpr_mask) == bpr_mask || it == cnt - 1)) {
 #pragma unroll 1
       for (int pass = 0; pass < (spb == 32 ? 2 : 1); ++pass) {
         const uint32_t rw = pass ? rword2 : rword;
-        const int wq = (bpr == 1 ? t : t % wpb) + 4 * pass;
         uint32_t fa[4][2];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -211,11 +194,16 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
           fa[j][0] = prmt(lo4, hi4, 0x5140u);
           fa[j][1] = prmt(lo4, hi4, 0x7362u);
         }
+        // the four salient columns behind this lane's residual word
+        const uint32_t cw = __ldg(reinterpret_cast<const uint32_t*>(binfo[rblk].cols + 4 * (my_wq + 4 * pass)));
 #pragma unroll
         for (int c = 0; c < NB; ++c) {
           uint2 xr = make_uint2(0, 0);
-          if (g + 8 * c < batch)
-            xr = *reinterpret_cast<const uint2*>(xsal + ((size_t)(g + 8 * c) * bpp + rblk) * spb + wq * 4);
+          if (xrow[c]) {
+            const unsigned short* xq = reinterpret_cast<const unsigned short*>(xrow[c] - t * 8 + (size_t)rblk * kBlock);
+            xr.x = (uint32_t)__ldg(xq + (cw & 0xFFu)) | ((uint32_t)__ldg(xq + ((cw >> 8) & 0xFFu)) << 16);
+            xr.y = (uint32_t)__ldg(xq + ((cw >> 16) & 0xFFu)) | ((uint32_t)__ldg(xq + (cw >> 24)) << 16);
+          }
           mma16816(acc[0][c], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
           mma16816(acc[1][c], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
         }
@@ -280,9 +268,11 @@ static int env_int(const char* name) {
   return e ? atoi(e) : 0;
 }
 
-// Launch shape: ksplit CTAs per row tile and warps per CTA, chosen so that a warp gets a run of
-// a few tiles and the grid has several CTAs per SM (small CTAs spread evenly over the 148 SMs).
-static void gemv_shape(int n, int m, int batch, int& ksplit, int& warps) {
+// Launch shape: ksplit CTAs per row tile and warps per CTA.  A warp should get a run of several
+// tiles (its ring then streams while it decodes) and the grid should have at least two CTAs per
+// SM while leaving room on the SM for the next layer's CTAs, which start their own weight
+// stream early (programmatic dependent launch).
+static void gemv_shape(int n, int m, int& ksplit, int& warps) {
   static int f_ks = -1, f_w = -1;
   if (f_ks < 0) { f_ks = env_int("STB_GEMV_KSPLIT"); f_w = env_int("STB_GEMV_WARPS"); }
   const int ntile = (n + kTileRows - 1) / kTileRows, nblk = m / kBlock;
@@ -290,21 +280,21 @@ static void gemv_shape(int n, int m, int batch, int& ksplit, int& warps) {
   int ks = 1;
   if (f_ks == 1 || f_ks == 2 || f_ks == 4 || f_ks == 8) ks = f_ks;
   else
-    while (ks < 8 && ntile * ks < 592 && nblk / (2 * ks) >= 2 * warps) ks *= 2;
+    while (ks < 8 && ntile * ks < 296 && nblk / (2 * ks * warps) >= 4) ks *= 2;
   while (ks > 1 && ks > nblk) ks /= 2;
-  // the activations of a CTA's slice must fit in shared memory
-  while (ks < 8 && (size_t)batch * ((size_t)((nblk + ks - 1) / ks) * 320 + 64) > 96 * 1024) ks *= 2;
   ksplit = ks;
 }
 
+// `chained`: launch as a programmatic dependent of the previous kernel of the stream (only used
+// between the GEMVs of one stb_layer_stack call, whose packed layers nobody writes meanwhile).
 template <int N, int NB>
 static cudaError_t launch_mma(const uint8_t* packed, int n, int m, const __half* x, int batch, size_t ldx,
-                              void* y, int y_f16, size_t ldy, int* dev_status, cudaStream_t s) {
+                              void* y, int y_f16, size_t ldy, int* dev_status, cudaStream_t s, bool chained) {
   const int ntile = (n + kTileRows - 1) / kTileRows, nblk = m / kBlock;
   int ksplit, warps;
-  gemv_shape(n, m, batch, ksplit, warps);
+  gemv_shape(n, m, ksplit, warps);
   const int bpp = (nblk + ksplit - 1) / ksplit;
-  const GemvSmem L = gemv_smem(N, warps, batch, bpp, ksplit, NB);
+  const GemvSmem L = gemv_smem(N, warps, ksplit, NB);
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(gemv_mma_kernel<N, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -317,11 +307,15 @@ static cudaError_t launch_mma(const uint8_t* packed, int n, int m, const __half*
   cfg.blockDim = dim3((unsigned)(warps * 32), 1, 1);
   cfg.dynamicSmemBytes = L.total;
   cfg.stream = s;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)ksplit; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  cfg.attrs = at; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemv_mma_kernel<N, NB>, packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status, ksplit, bpp);
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = chained ? 2 : 1;
+  int lg = 0;
+  while ((1 << lg) < ksplit) ++lg;
+  return cudaLaunchKernelEx(&cfg, gemv_mma_kernel<N, NB>, packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status, lg, bpp);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -344,6 +338,8 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
   const int spb = (int)hdr->spb;
+  const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)hdr->ntile +
+                            (size_t)rt * nblk * resid_tile_bytes(spb);
 
   float acc[4][BT];
 #pragma unroll
@@ -378,7 +374,7 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
             const float s1 = neg[c] ? -1.0f : 1.0f;
             if (code[c] == 3u) {
               const int q = qbase + __popc(salb & ((1u << c) - 1u));
-              const uint32_t word = q < spb ? *reinterpret_cast<const uint32_t*>(tile + resid_word_off(N, spb, g, q >> 2)) : 0x55555555u;
+              const uint32_t word = q < spb ? *reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, q >> 2)) : 0x55555555u;
               const float s2 = resid_code(word, j, q & 3) == 0u ? 1.0f : -1.0f;
               w = __fadd_rn(s1 * alpha[3], s2 * alpha[4]);
             } else {
@@ -447,8 +443,8 @@ static cudaError_t launch_general(const uint8_t* packed, int n, int m, const __h
 
 }  // namespace stb
 
-extern "C" int stb_gemv(const void* packed, int n, int m, int N, const void* x, int batch, size_t ldx,
-                        void* y, stb_dtype ydt, size_t ldy, int* dev_status, void* stream) {
+static int gemv_impl(const void* packed, int n, int m, int N, const void* x, int batch, size_t ldx,
+                     void* y, stb_dtype ydt, size_t ldy, int* dev_status, void* stream, bool chained) {
   if (!packed || !x || !y) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
@@ -463,13 +459,13 @@ extern "C" int stb_gemv(const void* packed, int n, int m, int N, const void* x, 
   static const bool force_general = stb::env_int("STB_GEMV_GENERAL") != 0;
   if (N >= 4 && N <= 6 && !force_general) {
     if (batch <= 8) {
-      if (N == 4) e = stb::launch_mma<4, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
-      else if (N == 5) e = stb::launch_mma<5, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
-      else e = stb::launch_mma<6, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+      if (N == 4) e = stb::launch_mma<4, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
+      else if (N == 5) e = stb::launch_mma<5, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
+      else e = stb::launch_mma<6, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
     } else {
-      if (N == 4) e = stb::launch_mma<4, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
-      else if (N == 5) e = stb::launch_mma<5, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
-      else e = stb::launch_mma<6, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s);
+      if (N == 4) e = stb::launch_mma<4, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
+      else if (N == 5) e = stb::launch_mma<5, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
+      else e = stb::launch_mma<6, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
     }
     return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
   }
@@ -486,12 +482,19 @@ extern "C" int stb_gemv(const void* packed, int n, int m, int N, const void* x, 
   return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
 }
 
+extern "C" int stb_gemv(const void* packed, int n, int m, int N, const void* x, int batch, size_t ldx,
+                        void* y, stb_dtype ydt, size_t ldy, int* dev_status, void* stream) {
+  return gemv_impl(packed, n, m, N, x, batch, ldx, y, ydt, ldy, dev_status, stream, false);
+}
+
 extern "C" int stb_layer_stack(const stb_step* steps, int count, int* dev_status, void* stream) {
   if (!steps || count < 0) return STB_ERR_ARG;
+  static const bool no_pdl = stb::env_int("STB_NO_PDL") != 0;
   for (int i = 0; i < count; ++i) {
     const stb_step& st = steps[i];
-    int rc = stb_gemv(st.packed, st.n, st.m, st.N, st.in, st.batch, st.ldin, st.out, st.odt, st.ldout,
-                      dev_status, stream);
+    // steps after the first start their weight stream while the previous step drains
+    int rc = gemv_impl(st.packed, st.n, st.m, st.N, st.in, st.batch, st.ldin, st.out, st.odt, st.ldout,
+                       dev_status, stream, i > 0 && !no_pdl);
     if (rc != STB_OK) return rc;
   }
   return STB_OK;

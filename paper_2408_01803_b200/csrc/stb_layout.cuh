@@ -1,10 +1,11 @@
 // Packed ("streaming") layout of an N:8 structured-binary layer, shared by the CUDA kernels.
-// Plain C++ (no CUDA types) so that the index arithmetic can also be compiled and checked on
-// the host.
+// Host + device code, so that the index arithmetic can also be compiled and checked on the
+// host.
 //
 // The unit of the layout is a TILE: 32 output rows x one 128-column block; all tiles of a layer
-// have the same size and follow each other in (row tile, block) order after a header and a
-// per-block table.  Inside a tile the work is split the way a warp-level tensor-core
+// have the same size, which depends on N alone, and follow each other in (row tile, block)
+// order after a header and a per-block table.  The residual codes of the salient columns, whose
+// size depends on the layer's salient counts, follow the tiles in the same order.  Inside a tile the work is split the way a warp-level tensor-core
 // instruction (m16n8k16) splits a 16 x 16 operand: lane = 4 g + t  (g = 0..7, t = 0..3) owns
 //     rows    r_j = g + 8 j      (j = 0..3) of the tile and, of each of them,
 //     groups  G_s = 4 s + t      (s = 0..3) of the block (a group = 8 columns),
@@ -14,7 +15,11 @@
 //
 // Every field is stored lane-major so that a warp reads it with coalesced vector loads:
 //
-//   mask    32 x uint4          byte u of the lane's 16 bytes = keep byte of slot u
+//   mask    32 x uint4          byte u of the lane's 16 bytes = keep mask of slot u, stored as its
+//                               INDEX among the C(8, N) masks with N bits set (increasing
+//                               numeric order): the same 8 bits, but a lookup table keyed by it
+//                               has at most 70 entries, which keeps shared-memory lookups by the
+//                               32 lanes of a warp nearly free of bank conflicts
 //   region  N words per lane    two-bit region codes, 16 per word, of the lane's 16 N kept
 //                               weights: first the "low" part (ranks k < min(N, 4) of every
 //                               slot, weight number wl = u NL + k), then the "high" part
@@ -32,6 +37,7 @@
 //                               are stored in the order p = 4 (r % 8) + r / 8, so that the
 //                               four rows of a lane are contiguous.
 //   sal2    32 x u16            a_sal2 per row, same row order
+// and, outside the tile, in the residual region (8 SPB bytes per tile):
 //   resid   SPB / 4 words per g residual of the block's salient columns: slot q (the q-th
 //                               salient column, ascending) of row r_j has the two-bit code
 //                               0 = +a_sal2, 2 = -a_sal2, 1 = no term (weight dropped, or
@@ -40,8 +46,8 @@
 //                               SPB (slots per block) is one of 0, 4, 8, 16, 32: the smallest
 //                               that holds the largest salient count of the layer.
 //
-// Tile bytes = 512 + 192 N + 320 + 8 SPB   (50 / 56 / 62 bytes per row and block at
-// N = 4 / 5 / 6, plus SPB / 4).
+// Tile bytes = 512 + 192 N + 320   (50 / 56 / 62 bytes per row and block at N = 4 / 5 / 6),
+// plus 8 SPB bytes per tile (SPB / 4 per row and block) in the residual region.
 #pragma once
 #include <stdint.h>
 
@@ -71,25 +77,25 @@ struct Header {          // 64 bytes at the start of the packed buffer
   uint32_t status;       // 0 or STB_ERR_CORRUPT
   uint32_t tile_bytes;
   uint32_t spb;          // residual slots per block: 0, 4, 8, 16 or 32
-  uint32_t pad;
+  uint32_t pad;          // the residual region starts at tiles_offset + rt_stride * ntile
 };
 static_assert(sizeof(Header) == 64, "header is 64 bytes");
 
-struct BlockInfo {       // 32 bytes, one per block, right after the header
+struct BlockInfo {       // 64 bytes, one per block, right after the header
   uint64_t salient[2];   // 128-bit salient-column mask
   uint32_t nsal;         // number of salient columns
   uint32_t pad[3];
+  uint8_t cols[32];      // the salient columns (0..127) in ascending order; unused entries 0
 };
-static_assert(sizeof(BlockInfo) == 32, "block info is 32 bytes");
+static_assert(sizeof(BlockInfo) == 64, "block info is 64 bytes");
 
 STB_HD constexpr int n_lo(int N) { return N < 4 ? N : 4; }
 STB_HD constexpr int n_hi(int N) { return N > 4 ? N - 4 : 0; }
 STB_HD constexpr int sign_full_words(int N) { return (n_lo(N) >> 1) + (n_hi(N) >> 1); }
 STB_HD constexpr bool sign_has_half(int N) { return (N & 1) != 0; }
 
-STB_HD constexpr uint32_t tile_bytes(int N, int spb) {
-  return 512u + 192u * (uint32_t)N + 320u + 8u * (uint32_t)spb;
-}
+STB_HD constexpr uint32_t tile_bytes(int N) { return 512u + 192u * (uint32_t)N + 320u; }
+STB_HD constexpr uint32_t resid_tile_bytes(int spb) { return 8u * (uint32_t)spb; }
 STB_HD constexpr uint32_t tiles_offset(int nblk) {
   return (uint32_t)((sizeof(Header) + sizeof(BlockInfo) * (size_t)nblk + 255) / 256 * 256);
 }
@@ -100,7 +106,6 @@ STB_HD constexpr uint32_t off_region(int) { return 512u; }
 STB_HD constexpr uint32_t off_sign(int N) { return 512u + 128u * (uint32_t)N; }
 STB_HD constexpr uint32_t off_scale(int N) { return 512u + 192u * (uint32_t)N; }
 STB_HD constexpr uint32_t off_sal2(int N) { return off_scale(N) + 256u; }
-STB_HD constexpr uint32_t off_resid(int N) { return off_scale(N) + 320u; }
 
 // Byte offset (inside the tile) of word `iw` of a per-lane field of `nw` words that starts at
 // `base`: the words are laid out as uint4 planes, then (nw & 2) a uint2 plane, then (nw & 1)
@@ -127,8 +132,9 @@ STB_HD constexpr uint32_t sign_half_off(int N, int lane) {
 // scale / sal2 / resid are indexed by the permuted row position p = 4 g + j of row g + 8 j
 STB_HD constexpr uint32_t scale_off(int N, int g, int j) { return off_scale(N) + (uint32_t)(4 * g + j) * 8u; }
 STB_HD constexpr uint32_t sal2_off(int N, int g, int j) { return off_sal2(N) + (uint32_t)(4 * g + j) * 2u; }
-STB_HD constexpr uint32_t resid_word_off(int N, int spb, int g, int wq) {
-  return off_resid(N) + ((uint32_t)g * (uint32_t)(spb >> 2) + (uint32_t)wq) * 4u;
+// byte offset of residual word wq of lane group g inside a tile's 8 SPB residual bytes
+STB_HD constexpr uint32_t resid_word_off(int spb, int g, int wq) {
+  return ((uint32_t)g * (uint32_t)(spb >> 2) + (uint32_t)wq) * 4u;
 }
 
 // bit position of the two-bit code number i (0..15) of a region word
@@ -151,6 +157,44 @@ STB_HD constexpr uint32_t half_to_upper(uint32_t h) {
 }
 STB_HD constexpr uint32_t half_from_upper(uint32_t s) {
   return ((s & 0x88888888u) >> 1) | ((s & 0x11111111u) << 1);
+}
+
+// Keep-mask index <-> keep mask.
+struct MaskTables {
+  uint8_t index[9][256];   // [N][mask] -> index (0 for a mask that does not have N bits)
+  uint8_t mask[9][72];     // [N][index] -> mask
+  uint8_t count[9];        // C(8, N)
+};
+constexpr MaskTables make_mask_tables() {
+  MaskTables t{};
+  for (int N = 0; N <= 8; ++N) {
+    int k = 0;
+    for (uint32_t m = 0; m < 256; ++m) {
+      int pc = 0;
+      for (int c = 0; c < 8; ++c) pc += (m >> c) & 1u;
+      if (pc == N) { t.index[N][m] = (uint8_t)k; t.mask[N][k] = (uint8_t)m; ++k; }
+    }
+    t.count[N] = (uint8_t)k;
+  }
+  return t;
+}
+constexpr MaskTables kMaskTables = make_mask_tables();
+#if defined(__CUDACC__)
+__device__ const MaskTables g_mask_tables = make_mask_tables();
+#endif
+STB_HD uint32_t mask_index(int N, uint32_t mask) {
+#if defined(__CUDA_ARCH__)
+  return g_mask_tables.index[N][mask & 0xFFu];
+#else
+  return kMaskTables.index[N][mask & 0xFFu];
+#endif
+}
+STB_HD uint32_t mask_from_index(int N, uint32_t idx) {
+#if defined(__CUDA_ARCH__)
+  return g_mask_tables.mask[N][idx < 72u ? idx : 0u];
+#else
+  return kMaskTables.mask[N][idx < 72u ? idx : 0u];
+#endif
 }
 
 // Where the code / sign of the k-th kept weight (ascending column) of slot u lives.

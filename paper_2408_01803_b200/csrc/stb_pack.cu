@@ -30,13 +30,23 @@ __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ 
     bi[b].salient[1] = hi;
     bi[b].nsal = (uint32_t)ns;
     bi[b].pad[0] = bi[b].pad[1] = bi[b].pad[2] = 0;
+    int q = 0;
+    for (int h = 0; h < 2; ++h) {
+      uint64_t mk = h ? hi : lo;
+      while (mk && q < kMaxSalient) {
+        bi[b].cols[q++] = (uint8_t)(__ffsll((long long)mk) - 1 + 64 * h);
+        mk &= mk - 1;
+      }
+    }
+    for (; q < kMaxSalient; ++q) bi[b].cols[q] = 0;
     atomicMax(&maxsal, ns);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     const int ntile = (n + kTileRows - 1) / kTileRows;
     const int spb = spb_for(maxsal);
-    const uint32_t tb = tile_bytes(N, spb);
+    const uint32_t tb = tile_bytes(N);
+    const uint64_t tiles = (uint64_t)nblk * (uint64_t)ntile;
     hdr->magic = kMagic;
     hdr->version = 2;
     hdr->n = n; hdr->m = m; hdr->N = N;
@@ -44,7 +54,7 @@ __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ 
     hdr->ntile = ntile;
     hdr->tiles_offset = tiles_offset(nblk);
     hdr->rt_stride = (uint64_t)tb * (uint64_t)nblk;
-    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + (uint64_t)tb * (uint64_t)nblk * (uint64_t)ntile;
+    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + ((uint64_t)tb + resid_tile_bytes(spb)) * tiles;
     hdr->status = bad ? (uint32_t)STB_ERR_CORRUPT : 0u;
     hdr->tile_bytes = tb;
     hdr->spb = (uint32_t)spb;
@@ -95,6 +105,8 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
   const uint64_t sal_lo = bi->salient[0], sal_hi = bi->salient[1];
   const int nsal = (int)bi->nsal, spb = (int)hdr->spb;
   uint8_t* tile = packed + hdr->tiles_offset + ((size_t)rt * nblk + b) * (size_t)hdr->tile_bytes;
+  uint8_t* resid = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
+                   ((size_t)rt * nblk + b) * (size_t)resid_tile_bytes(spb);
 
   // ---- phase 1: lane = row ----
   // rows past n: nothing kept, all signs "+", zero scales
@@ -177,7 +189,7 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
       }
       word |= __shfl_xor_sync(0xFFFFFFFFu, word, 8);
       word |= __shfl_xor_sync(0xFFFFFFFFu, word, 16);
-      if (lane < 8) *reinterpret_cast<uint32_t*>(tile + resid_word_off(N, spb, lane, wq)) = word;
+      if (lane < 8) *reinterpret_cast<uint32_t*>(resid + resid_word_off(spb, lane, wq)) = word;
     }
   }
   __syncwarp();
@@ -189,7 +201,7 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
   for (int u = 0; u < 16; ++u) {
     const int j = u >> 2, sidx = u & 3;
     const int r = g + 8 * j, grp = 4 * sidx + t;
-    maskw[j] |= (uint32_t)sm_keep[wib][r][grp] << (8 * sidx);
+    maskw[j] |= mask_index(N, sm_keep[wib][r][grp]) << (8 * sidx);
     sgn[u] = sm_sign[wib][r][grp];
     reg[u] = sm_region[wib][r][grp];
   }
@@ -227,7 +239,7 @@ extern "C" int stb_pack_size(int n, int m, int N, size_t* bytes) {
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
   const size_t nblk = (size_t)m / stb::kBlock, ntile = ((size_t)n + 31) / 32;
-  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * (size_t)stb::tile_bytes(N, stb::kMaxSalient);
+  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * (size_t)(stb::tile_bytes(N) + stb::resid_tile_bytes(stb::kMaxSalient));
   return STB_OK;
 }
 
@@ -271,7 +283,7 @@ extern "C" int stb_packed_info(const void* packed, stb_info* info, void* stream)
   info->n = h.n; info->m = h.m; info->N = h.N;
   info->status = (int)h.status;
   info->used_bytes = h.used_bytes;
-  info->stream_bytes = h.rt_stride * (uint64_t)h.ntile;
+  info->stream_bytes = (h.rt_stride + (uint64_t)stb::resid_tile_bytes((int)h.spb) * (uint64_t)h.nblk) * (uint64_t)h.ntile;
   return STB_OK;
 }
 

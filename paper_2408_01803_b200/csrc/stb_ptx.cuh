@@ -5,21 +5,27 @@
 
 namespace stb {
 
-// position selectors of all 256 keep bytes (see position_selector in stb_decode.cuh)
-struct PosTable { uint32_t v[256]; };
+// Position selectors by keep-mask index (see position_selector in stb_decode.cuh): entry
+// [N][i] is {selector of columns 0..3, selector of columns 4..7} of the i-th mask with N bits,
+// each in the low 16 bits of a word.
+struct PosTable { uint2 v[9][72]; };
 constexpr PosTable make_pos_table() {
   PosTable t{};
-  for (uint32_t m = 0; m < 256; ++m) {
-    uint32_t p = 0, r = 0;
-    for (int c = 0; c < 8; ++c) {
-      if ((m >> c) & 1u) { p |= (r & 7u) << (4 * c); ++r; }
-      else p |= 7u << (4 * c);
+  for (int N = 0; N <= 8; ++N) {
+    int k = 0;
+    for (uint32_t m = 0; m < 256; ++m) {
+      uint32_t p = 0, r = 0;
+      for (int c = 0; c < 8; ++c) {
+        if ((m >> c) & 1u) { p |= (r & 7u) << (4 * c); ++r; }
+        else p |= 7u << (4 * c);
+      }
+      if ((int)r == N) { t.v[N][k].x = p & 0xFFFFu; t.v[N][k].y = p >> 16; ++k; }
     }
-    t.v[m] = p;
   }
   return t;
 }
 __device__ const PosTable g_pos_table = make_pos_table();
+constexpr int kPosTableEntries = 72;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -56,6 +62,18 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Programmatic dependent launch: wait until the grid this one depends on has completed and its
+// memory is visible (no-op for an ordinary launch) / allow the dependent grid to be scheduled.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// 16-byte read-only load through L1
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
 }
 
 // D(16x8, fp32) += A(16x16, fp16, row) * B(16x8, fp16, col)

@@ -51,8 +51,8 @@ static int check(int trials, int spb) {
       for (int q = 0; q < 5; ++q) scale[r][q] = (uint16_t)(rnd() & 0x7FFFu);
       for (int q = 0; q < 32; ++q) rcode[r][q] = q < spb ? (uint8_t)(rnd() % 3) : 1;
     }
-    const uint32_t tb = tile_bytes(N, spb);
-    std::vector<uint8_t> tile(tb + 64, 0);
+    const uint32_t tb = tile_bytes(N);
+    std::vector<uint8_t> tile(tb + 64, 0), resid(resid_tile_bytes(spb) + 64, 0);
     auto put32 = [&](uint32_t off, uint32_t v) { std::memcpy(&tile[off], &v, 4); };
     auto or32 = [&](uint32_t off, uint32_t v) { uint32_t o; std::memcpy(&o, &tile[off], 4); o |= v; std::memcpy(&tile[off], &o, 4); };
     for (int lane = 0; lane < 32; ++lane) {
@@ -60,7 +60,7 @@ static int check(int trials, int spb) {
       uint32_t sg[16], rg[16], maskw[4] = {0, 0, 0, 0};
       for (int u = 0; u < 16; ++u) {
         const int j = u >> 2, s = u & 3, r = g + 8 * j, grp = 4 * s + t;
-        maskw[j] |= (uint32_t)keep[r][grp] << (8 * s);
+        maskw[j] |= mask_index(N, keep[r][grp]) << (8 * s);
         sg[u] = sign[r][grp]; rg[u] = region[r][grp];
       }
       LaneWords<N> w;
@@ -76,10 +76,17 @@ static int check(int trials, int spb) {
       for (int q = 0; q < 4; ++q) { A |= (uint32_t)(scale[r][q] & 0xFF) << (8 * q); B |= (uint32_t)(scale[r][q] >> 8) << (8 * q); }
       put32(scale_off(N, g, j), A); put32(scale_off(N, g, j) + 4, B);
       std::memcpy(&tile[sal2_off(N, g, j)], &scale[r][4], 2);
-      for (int q = 0; q < spb; ++q) or32(resid_word_off(N, spb, g, q >> 2), (uint32_t)rcode[r][q] << code_bit(4 * j + (q & 3)));
+      for (int q = 0; q < spb; ++q) {
+        uint32_t o;
+        std::memcpy(&o, &resid[resid_word_off(spb, g, q >> 2)], 4);
+        o |= (uint32_t)rcode[r][q] << code_bit(4 * j + (q & 3));
+        std::memcpy(&resid[resid_word_off(spb, g, q >> 2)], &o, 4);
+      }
     }
     // every offset must stay inside the tile
-    if (off_resid(N) + 8u * spb != tb) { ++errors; std::printf("N=%d tile size mismatch\n", N); }
+    if (sal2_off(N, 7, 3) + 2u != tb || resid_word_off(spb ? spb : 4, 7, (spb ? spb : 4) / 4 - 1) + 4u != resid_tile_bytes(spb ? spb : 4)) {
+      ++errors; std::printf("N=%d tile size mismatch\n", N);
+    }
 
     for (int lane = 0; lane < 32; ++lane) {
       const int g = lane >> 2, t = lane & 3;
@@ -109,7 +116,7 @@ static int check(int trials, int spb) {
         if (sal2_bits<N>(lt, j) != scale[r][4]) { if (++errors < 10) std::printf("sal2 N=%d\n", N); }
         for (int q = 0; q < spb; ++q) {
           uint32_t word;
-          std::memcpy(&word, &tile[resid_word_off(N, spb, g, q >> 2)], 4);
+          std::memcpy(&word, &resid[resid_word_off(spb, g, q >> 2)], 4);
           if (resid_code(word, j, q & 3) != rcode[r][q]) { if (++errors < 10) std::printf("resid code N=%d\n", N); }
           if (((resid_selector(word, j) >> (4 * (q & 3))) & 0xFu) != rcode[r][q]) { if (++errors < 10) std::printf("resid selector N=%d\n", N); }
         }
@@ -123,7 +130,7 @@ static int check(int trials, int spb) {
           for (int s = 0; s < 4; ++s) {
             if (N == 6 && (s & 1) == 0) fr.high(j, s >> 1, XL, XH);
             const int r = g + 8 * j, grp = 4 * s + t;
-            const uint32_t kb = keep_byte_of(lt.mask, j, s);
+            const uint32_t kb = mask_from_index(N, keep_index_of(lt.mask, j, s));
             if (kb != keep[r][grp]) { if (++errors < 10) std::printf("keep byte N=%d\n", N); }
             uint32_t f[4];
             fr.slot(j, s, position_selector(kb), XL, XH, f);
@@ -153,6 +160,19 @@ int main() {
   int e = 0;
   e += check<1>(4, 0); e += check<2>(4, 4); e += check<3>(4, 8); e += check<4>(8, 4); e += check<5>(8, 16);
   e += check<6>(8, 32); e += check<7>(4, 4); e += check<8>(4, 0); e += check<4>(2, 0); e += check<6>(2, 8);
+  // keep-mask index: a bijection between the masks with N bits and 0..C(8,N)-1, in increasing order
+  for (int N = 0; N <= 8; ++N) {
+    int k = 0;
+    for (uint32_t m = 0; m < 256; ++m) {
+      int pc = 0;
+      for (int c = 0; c < 8; ++c) pc += (m >> c) & 1;
+      if (pc != N) continue;
+      if (mask_index(N, m) != (uint32_t)k || mask_from_index(N, k) != m) ++e;
+      ++k;
+    }
+    const int want[9] = {1, 8, 28, 56, 70, 56, 28, 8, 1};
+    if (k != want[N] || kMaskTables.count[N] != want[N]) ++e;
+  }
   // position selector: rank of each kept column, 7 for dropped ones
   for (uint32_t m = 0; m < 256; ++m) {
     const uint32_t p = position_selector(m);
