@@ -21,14 +21,21 @@ namespace stb {
 // Grid: one thread-block cluster of `ksplit` CTAs per row tile (32 rows); CTA k of the cluster
 // takes the k-th slice of the 128-column blocks and its warps take contiguous runs of that
 // slice.  Each warp streams its tiles from HBM into a private ring in shared memory with 1-D
-// bulk copies (kDepth tiles in flight), reads a tile into registers, decodes it slot by slot
+// bulk copies (kChunk tiles per copy, kDepth copies in flight), reads a tile into registers, decodes it slot by slot
 // into fp16 operand registers (stb_decode.cuh) and multiplies with m16n8k16 tensor-core
 // instructions: A = 16 rows x 16 columns of W^, B = the activations (8 batch rows), read
 // through L1 (they are shared by every CTA of the SM), fp32 accumulators in registers for the
 // whole run.  The residual term of the salient columns goes through the same instruction, with
 // the salient slots of 16 / SPB blocks as its K dimension.  Partial sums: warps through shared
 // memory, CTAs of the cluster through distributed shared memory, both in a fixed order.
-constexpr int kDepth = 4;
+#ifndef STB_GEMV_DEPTH
+#define STB_GEMV_DEPTH 4
+#endif
+#ifndef STB_GEMV_CHUNK
+#define STB_GEMV_CHUNK 1
+#endif
+constexpr int kDepth = STB_GEMV_DEPTH;     // ring slots per warp
+constexpr int kChunk = STB_GEMV_CHUNK;     // tiles per bulk copy (consecutive blocks of a row tile are contiguous)
 constexpr long long kWaitLimit = 2000000000ll;     // about a second of SM clocks
 
 struct GemvSmem {
@@ -39,7 +46,7 @@ __host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int ksplit, int 
   GemvSmem s;
   s.bars = kPosTableEntries * 8;                     // the position table comes first
   s.ring = (s.bars + (uint32_t)(warps * kDepth * 8) + 127u) & ~127u;
-  s.tile_stride = (tile_bytes(N) + 127u) & ~127u;
+  s.tile_stride = (kChunk * tile_bytes(N) + 127u) & ~127u;      // one ring slot = one chunk of tiles
   s.part = s.ring + (uint32_t)(warps * kDepth) * s.tile_stride;
   s.total = s.part + (uint32_t)ksplit * 32u * 8u * (uint32_t)NB * 4u;
   return s;
@@ -87,9 +94,10 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
   if (lane == 0) {
     for (int i = 0; i < kDepth; ++i) mbar_init(bar0 + 8u * i, 1);
     fence_async_smem();
-    for (int i = 0; i < kDepth && i < cnt; ++i) {
-      mbar_expect_tx(bar0 + 8u * i, tbytes);
-      bulk_g2s(smem_u32(ring + (size_t)i * L.tile_stride), rtbase + (size_t)(wb0 + i) * tbytes, tbytes, bar0 + 8u * i);
+    for (int i = 0; i < kDepth && i * kChunk < cnt; ++i) {
+      const uint32_t bytes = (uint32_t)min(kChunk, cnt - i * kChunk) * tbytes;
+      mbar_expect_tx(bar0 + 8u * i, bytes);
+      bulk_g2s(smem_u32(ring + (size_t)i * L.tile_stride), rtbase + (size_t)(wb0 + i * kChunk) * tbytes, bytes, bar0 + 8u * i);
     }
   }
   for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x) reinterpret_cast<uint2*>(smem)[i] = g_pos_table.v[N][i];
@@ -124,7 +132,8 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
   for (int c = 0; c < NB; ++c) xrow[c] = g + 8 * c < batch ? x + (size_t)(g + 8 * c) * ldx + t * 8 : nullptr;
 
   for (int it = 0; it < cnt; ++it) {
-    const int slot = it & (kDepth - 1);
+    const int ch = it / kChunk, kin = it - ch * kChunk;     // chunk and tile inside the chunk
+    const int slot = ch % kDepth;
     const uint32_t bar = bar0 + 8u * slot;
     const int b = wb0 + it;
     const bool mine = spb > 0 && (it & bpr_mask) == my_pos;
@@ -135,16 +144,20 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
       rblk = b;
     }
     // all lanes poll; the verdict is made warp-uniform so that nobody is left at a __syncwarp
-    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(it / kDepth) & 1u, kWaitLimit))) { failed = true; break; }
-    const uint8_t* tile = ring + (size_t)slot * L.tile_stride;
+    if (kin == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(ch / kDepth) & 1u, kWaitLimit))) { failed = true; break; }
+    const uint8_t* tile = ring + (size_t)slot * L.tile_stride + (size_t)kin * tbytes;
     LaneTile<N> lt;
     load_lane_tile<N>(tile, lane, lt);
     if (mine) { rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1]; }
-    __syncwarp();
-    if (lane == 0 && it + kDepth < cnt) {          // refill the slot that was just read
-      fence_async_smem();
-      mbar_expect_tx(bar, tbytes);
-      bulk_g2s(smem_u32(tile), rtbase + (size_t)(b + kDepth) * tbytes, tbytes, bar);
+    if (kin == kChunk - 1 || it == cnt - 1) {      // the whole chunk is in registers or consumed
+      __syncwarp();
+      const int nxt = (ch + kDepth) * kChunk;      // first tile of the chunk that reuses this slot
+      if (lane == 0 && nxt < cnt) {
+        const uint32_t bytes = (uint32_t)min(kChunk, cnt - nxt) * tbytes;
+        fence_async_smem();
+        mbar_expect_tx(bar, bytes);
+        bulk_g2s(smem_u32(ring + (size_t)slot * L.tile_stride), rtbase + (size_t)(wb0 + nxt) * tbytes, bytes, bar);
+      }
     }
 
     FastRows<N> fr;
@@ -154,27 +167,32 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
 #pragma unroll
       for (int j = 0; j < 4; ++j) fr.high(j, 0, XL[j], XH[j]);
     }
+    // all table lookups and activation loads of the tile are issued up front
+    uint2 P[16];
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {
-      uint4 xf[NB];
+    for (int u = 0; u < 16; ++u) P[u] = ptab[keep_index_of(lt.mask, u >> 2, u & 3)];
+    uint4 xf[4][NB];
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
 #pragma unroll
       for (int c = 0; c < NB; ++c) {
-        xf[c] = make_uint4(0, 0, 0, 0);
-        if (xrow[c]) xf[c] = ldg_nc_v4(xrow[c] + (size_t)b * kBlock + s * 32);
+        xf[s][c] = make_uint4(0, 0, 0, 0);
+        if (xrow[c]) xf[s][c] = ldg_nc_v4(xrow[c] + (size_t)b * kBlock + s * 32);
       }
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
       uint32_t f[4][4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         if (N == 6 && (s & 1) == 0) fr.high(j, s >> 1, XL[j], XH[j]);
-        const uint2 P = ptab[keep_index_of(lt.mask, j, s)];
-        fr.slot2(j, s, P.x, P.y, XL[j], XH[j], f[j]);
+        fr.slot2(j, s, P[4 * j + s].x, P[4 * j + s].y, XL[j], XH[j], f[j]);
       }
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
         for (int c = 0; c < NB; ++c) {
-          mma16816(acc[mt][c], f[2 * mt][0], f[2 * mt + 1][0], f[2 * mt][1], f[2 * mt + 1][1], xf[c].x, xf[c].y);
-          mma16816(acc[mt][c], f[2 * mt][2], f[2 * mt + 1][2], f[2 * mt][3], f[2 * mt + 1][3], xf[c].z, xf[c].w);
+          mma16816(acc[mt][c], f[2 * mt][0], f[2 * mt + 1][0], f[2 * mt][1], f[2 * mt + 1][1], xf[s][c].x, xf[s][c].y);
+          mma16816(acc[mt][c], f[2 * mt][2], f[2 * mt + 1][2], f[2 * mt][3], f[2 * mt + 1][3], xf[s][c].z, xf[s][c].w);
         }
     }
 
