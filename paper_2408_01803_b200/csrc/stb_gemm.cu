@@ -1,23 +1,402 @@
-// stb_gemm: prefill GEMM on the tensor cores (placeholder translation unit until the tcgen05
-// kernel lands; the entry points exist so that the library exports its whole C ABI).
+// stb_gemm: prefill GEMM  Y[t][i] = sum_j W^[i][j] X[t][j]  on the 5th-generation tensor cores
+// (tcgen05.mma, fp32 accumulators in tensor memory).  The compute-bound prefilling stage of
+// Appendix C.2: N = sequence length x batch tokens against one packed layer.
+//
+// One CTA computes a 128 (rows of W^) x 256 (tokens) tile of the output, D = A B^T with
+//   A = 128 x 64 bf16 slice of W^, decoded from the packed tiles into shared memory in the
+//       K-major 128-byte-swizzled layout the tensor core reads,
+//   B = 256 x 64 bf16 slice of X, brought in by TMA with the same swizzle,
+// in a ring of kStages stages over K.  Warp roles:
+//   warp 0      TMA producer (one lane): X slices
+//   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage, tcgen05.commit frees
+//               the stage; also allocates / frees the 256 TMEM columns
+//   warps 2..5  decode: warp w owns rows 32 (w % 4) .. +31 of the tile = one packed row tile;
+//               per 128-column block it loads the lane's words (prefetching the next block),
+//               converts the four fp16 scales of its rows to bf16 (RN-even) and writes the two
+//               64-column halves of the block into two stages; afterwards the same warps read
+//               the accumulator (TMEM lanes 32 (w % 4) ..) and store Y.
+// Every wait on an mbarrier is bounded; a wait that runs out sets an abort flag (all roles then
+// leave their loops), reports STB_ERR_TIMEOUT through dev_status and the CTA still frees TMEM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include "../../include/stb.h"
+#include "stb_decode.cuh"
 #include "stb_layout.cuh"
+#include "stb_ptx.cuh"
+
+namespace stb {
+
+constexpr int kBM = 128;          // rows of W^ per CTA (UMMA M)
+constexpr int kBN = 256;          // tokens per CTA (UMMA N)
+constexpr int kBK = 64;           // K per stage: one 128-byte swizzle row of bf16
+constexpr int kStages = 4;
+constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
+constexpr uint32_t kStageB = kBN * kBK * 2;      // 32 KB
+constexpr uint32_t kGemmTab = 0;                                   // position table (576 B)
+constexpr uint32_t kGemmBars = 1024;                               // full[4], empty[4], accum, tmem slot, abort
+constexpr uint32_t kGemmA = 2048;                                  // 1024-byte aligned stages
+constexpr uint32_t kGemmB = kGemmA + kStages * kStageA;
+constexpr uint32_t kGemmSmem = kGemmB + kStages * kStageB;         // 198656 B
+constexpr long long kGemmWaitLimit = 2000000000ll;
+
+// ---- tcgen05 / TMA wrappers ---------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                 "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                 "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+               : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major, 128-byte-swizzled operand tile (rows of 128
+// bytes, groups of 8 rows 1024 bytes apart): start address, stride byte offset 1024,
+// descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                  // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset
+  d |= (uint64_t)1 << 46;                  // version
+  d |= (uint64_t)2 << 61;                  // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+
+// Bounded mbarrier wait with a CTA-wide abort flag (a volatile int in shared memory).
+__device__ __forceinline__ bool gemm_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kGemmWaitLimit) { *abort_flag = 1; return false; }
+  }
+  return true;
+}
+
+__device__ __forceinline__ uint32_t bf16_bits(uint32_t h16) {
+  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((unsigned short)h16))));
+}
+
+// ------------------------------------------------------------------------------------------
+template <int N>
+__global__ void __launch_bounds__(192, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict__ packed, int n, int m, int T,
+            void* __restrict__ Y, int y_bf16, size_t ldy, float* __restrict__ ws, int ksplit, int bps,
+            uint32_t box_bytes, int* dev_status) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const Header* hdr = reinterpret_cast<const Header*>(packed);
+  if (!header_matches(hdr, n, m, N)) {
+    if (threadIdx.x == 0 && dev_status) *dev_status = STB_ERR_CORRUPT;
+    return;
+  }
+  const int nblk = m / kBlock, ntile = hdr->ntile;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tt = blockIdx.x, mt = blockIdx.y, kz = blockIdx.z;
+  const int b0 = kz * bps, b1 = min(nblk, b0 + bps);
+  const int nstage = 2 * max(b1 - b0, 0);              // 64-column stages of this CTA
+
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar_full = sbase + kGemmBars, bar_empty = bar_full + 8 * kStages, bar_accum = bar_empty + 8 * kStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kGemmBars + 8 * (2 * kStages + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kGemmBars + 8 * (2 * kStages + 1) + 8);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 5); mbar_init(bar_empty + 8 * i, 1); }
+    mbar_init(bar_accum, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x) reinterpret_cast<uint2*>(smem + kGemmTab)[i] = g_pos_table.v[N][i];
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kBN);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      for (int it = 0; it < nstage; ++it) {
+        const int s = it % kStages;
+        if (!gemm_wait(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) break;
+        mbar_expect_tx(bar_full + 8 * s, box_bytes);
+        tma_load_2d(sbase + kGemmB + s * kStageB, &xmap, (b0 * 2 + it) * kBK, tt * kBN, bar_full + 8 * s);
+      }
+      if (*abort_flag) {       // let copies in flight land before the CTA gives its shared memory up
+        const long long t0 = clock64();
+        while (clock64() - t0 < 200000) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      for (int it = 0; it < nstage; ++it) {
+        const int s = it % kStages;
+        if (!gemm_wait(bar_full + 8 * s, (uint32_t)(it / kStages) & 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint64_t ad = umma_desc(sbase + kGemmA + s * kStageA), bd = umma_desc(sbase + kGemmB + s * kStageB);
+#pragma unroll
+        for (int kk = 0; kk < kBK / 16; ++kk)
+          umma_bf16(tmem_d, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(bar_empty + 8 * s);          // the stage is free once these MMAs have read it
+      }
+      umma_commit(bar_accum);                    // all MMAs issued so far have completed
+    }
+  } else {
+    // ---------------- decode warps ----------------
+    const int q = warp & 3;                       // row quarter of the tile = TMEM lane quarter
+    const int g = lane >> 2, t = lane & 3;
+    const int rtile = mt * 4 + q;                 // packed row tile
+    const bool live = rtile < ntile;
+    const uint2* ptab = reinterpret_cast<const uint2*>(smem + kGemmTab);
+    const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+    const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
+    const int spb = (int)hdr->spb;
+    const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
+                              (size_t)rtile * nblk * resid_tile_bytes(spb);
+    constexpr uint32_t tbytes = tile_bytes(N);
+    LaneTile<N> cur = {}, nxt = {};
+    if (live && b0 < b1) load_lane_tile<N>(rtbase + (size_t)b0 * tbytes, lane, cur);
+    bool ok = true;
+    for (int b = b0; b < b1 && ok; ++b) {
+      if (live && b + 1 < b1) load_lane_tile<N>(rtbase + (size_t)(b + 1) * tbytes, lane, nxt);
+      // bf16 scale bytes of the lane's four rows
+      uint32_t A16[4], B16[4];
+      float a1f[4], a2f[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint32_t v = live ? bf16_bits(scale_bits<N>(cur, j, c)) : 0u;
+          lo |= (v & 0xFFu) << (8 * c);
+          hi |= (v >> 8) << (8 * c);
+        }
+        A16[j] = lo; B16[j] = hi;
+        a1f[j] = live ? __half2float(__ushort_as_half((unsigned short)scale_bits<N>(cur, j, 3))) : 0.f;
+        a2f[j] = live ? __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(cur, j))) : 0.f;
+      }
+      FastRows<N> fr;
+      fr.init(cur, A16, B16);
+      uint32_t XL[4] = {0, 0, 0, 0}, XH[4] = {0, 0, 0, 0};
+      if (N == 5) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) fr.high(j, 0, XL[j], XH[j]);
+      }
+      const int nsal = live ? (int)binfo[b].nsal : 0;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int it = 2 * (b - b0) + h, s = it % kStages;
+        if (!gemm_wait(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        uint8_t* As = smem + kGemmA + s * kStageA;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl) {
+            const int sidx = 2 * h + sl;                       // slot s of the block, group 4 sidx + t
+            uint32_t f[4] = {0, 0, 0, 0};
+            if (live) {
+              if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
+              const uint2 P = ptab[keep_index_of(cur.mask, j, sidx)];
+              fr.slot2(j, sidx, P.x, P.y, XL[j], XH[j], f);
+            }
+            const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
+            *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
+          }
+        }
+        // salient columns of this half: bf16( fl32( s1 a_sal1 + s2 a_sal2 ) ), slot sq handled by lane t = sq % 4
+        if (nsal > 0) {
+          __syncwarp();
+          for (int sq = t; sq < nsal; sq += 4) {
+            const int c = binfo[b].cols[sq];
+            if ((c >> 6) != h) continue;
+            const uint32_t word = __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2)));
+            const int c64 = c & 63;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t rc = resid_code(word, j, sq & 3);
+              if (rc == 1u) continue;
+              unsigned short* pv = reinterpret_cast<unsigned short*>(As + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
+              const bool neg1 = (*pv & 0x8000u) != 0;
+              const float v = __fadd_rn(neg1 ? -a1f[j] : a1f[j], rc == 0u ? a2f[j] : -a2f[j]);
+              *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+            }
+          }
+        }
+        fence_async_smem();          // generic-proxy writes -> visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_full + 8 * s);
+      }
+      if (live && b + 1 < b1) cur = nxt;
+    }
+
+    // ---------------- epilogue: TMEM -> registers -> Y ----------------
+    if (gemm_wait(bar_accum, 0u, abort_flag) && nstage > 0) {
+      tc_fence_after();
+      const int row = mt * kBM + 32 * q + lane;                // output feature (row of W^)
+      float* wsz = ws ? ws + (size_t)kz * (size_t)T * (size_t)n : nullptr;
+#pragma unroll 1
+      for (int cc = 0; cc < kBN / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(tmem_d + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * cc), r);
+        if (row < n) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int tok = tt * kBN + 32 * cc + i;
+            if (tok < T) {
+              const float v = __uint_as_float(r[i]);
+              if (wsz) wsz[(size_t)tok * n + row] = v;
+              else if (y_bf16) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(v);
+              else static_cast<float*>(Y)[(size_t)tok * ldy + row] = v;
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // the MMA thread makes sure the tensor core is done with TMEM before it is freed
+  if (warp == 1 && lane == 0) gemm_wait(bar_accum, 0u, abort_flag);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_d, kBN);
+  if (threadIdx.x == 0 && *abort_flag && dev_status) *dev_status = STB_ERR_TIMEOUT;
+}
+
+// Split-K reduction: Y[t][i] = sum_z ws[z][t][i], in z order.
+__global__ void gemm_reduce_kernel(const float* __restrict__ ws, int ksplit, int n, int T, void* __restrict__ Y,
+                                   int y_bf16, size_t ldy) {
+  const size_t total = (size_t)T * n;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    float s = 0.0f;
+    for (int z = 0; z < ksplit; ++z) s += ws[(size_t)z * total + i];
+    const size_t tok = i / n, row = i % n;
+    if (y_bf16) static_cast<__nv_bfloat16*>(Y)[tok * ldy + row] = __float2bfloat16_rn(s);
+    else static_cast<float*>(Y)[tok * ldy + row] = s;
+  }
+}
+
+// K split: only when the output tiles alone cannot fill the 148 SMs
+static int gemm_ksplit(int n, int m, int T) {
+  static int forced = -1;
+  if (forced < 0) { const char* e = getenv("STB_GEMM_KSPLIT"); forced = e ? atoi(e) : 0; }
+  const int tiles = ((n + kBM - 1) / kBM) * ((T + kBN - 1) / kBN), nblk = m / kBlock;
+  int ks = 1;
+  if (forced >= 1 && forced <= 16) ks = forced;
+  else if (tiles < 100) ks = 148 / tiles;
+  if (ks > 16) ks = 16;
+  while (ks > 1 && nblk / ks < 4) --ks;
+  if (ks < 1) ks = 1;
+  const int bps = (nblk + ks - 1) / ks;          // blocks per split; every split gets at least one
+  return (nblk + bps - 1) / bps;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+template <int N>
+static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T, size_t ldx, void* Y, int y_bf16,
+                       size_t ldy, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t s) {
+  const int ks = gemm_ksplit(n, m, T);
+  if (ks > 1 && (!ws || ws_bytes < (size_t)ks * T * n * sizeof(float))) return STB_ERR_SIZE;
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return STB_ERR_CUDA;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)T};
+  const cuuint64_t strides[1] = {(cuuint64_t)ldx * 2};
+  const cuuint32_t box_rows = (cuuint32_t)(T < kBN ? T : kBN);
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return STB_ERR_ARG;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem) != cudaSuccess) return STB_ERR_CUDA;
+    attr_done = true;
+  }
+  const int nblk = m / kBlock, bps = (nblk + ks - 1) / ks;
+  dim3 grid((unsigned)((T + kBN - 1) / kBN), (unsigned)((n + kBM - 1) / kBM), (unsigned)ks);
+  gemm_kernel<N><<<grid, 192, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, ks > 1 ? static_cast<float*>(ws) : nullptr,
+                                              ks, bps, box_rows * kBK * 2, dev_status);
+  if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
+  if (ks > 1) {
+    gemm_reduce_kernel<<<148 * 4, 256, 0, s>>>(static_cast<const float*>(ws), ks, n, T, Y, y_bf16, ldy);
+    if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
+  }
+  return STB_OK;
+}
+
+}  // namespace stb
 
 extern "C" int stb_gemm_workspace(int n, int m, int N, int T, size_t* bytes) {
   if (!bytes) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0 || T < 1) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
-  *bytes = 0;
+  const int ks = stb::gemm_ksplit(n, m, T);
+  *bytes = ks > 1 ? (size_t)ks * (size_t)T * (size_t)n * sizeof(float) : 0;
   return STB_OK;
 }
 
 extern "C" int stb_gemm(const void* packed, int n, int m, int N, const void* X, int T, size_t ldx,
                         void* Y, stb_dtype ydt, size_t ldy, void* ws, size_t ws_bytes,
                         int* dev_status, void* stream) {
-  (void)packed; (void)n; (void)m; (void)N; (void)X; (void)T; (void)ldx; (void)Y; (void)ydt;
-  (void)ldy; (void)ws; (void)ws_bytes; (void)dev_status; (void)stream;
-  return STB_ERR_UNSUPPORTED;
+  if (!packed || !X || !Y) return STB_ERR_ARG;
+  if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0 || T < 1) return STB_ERR_SHAPE;
+  if (N < 1 || N > 8) return STB_ERR_NM;
+  if (N < 4 || N > 6) return STB_ERR_UNSUPPORTED;          // the tensor-core decode covers N = 4, 5, 6
+  if (ydt != STB_F32 && ydt != STB_BF16) return STB_ERR_UNSUPPORTED;
+  if (ldx < (size_t)m || ldy < (size_t)n || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u)) return STB_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const uint8_t* p = static_cast<const uint8_t*>(packed);
+  const int y_bf16 = ydt == STB_BF16;
+  switch (N) {
+    case 4: return stb::launch_gemm<4>(p, n, m, X, T, ldx, Y, y_bf16, ldy, ws, ws_bytes, dev_status, s);
+    case 5: return stb::launch_gemm<5>(p, n, m, X, T, ldx, Y, y_bf16, ldy, ws, ws_bytes, dev_status, s);
+    default: return stb::launch_gemm<6>(p, n, m, X, T, ldx, Y, y_bf16, ldy, ws, ws_bytes, dev_status, s);
+  }
 }

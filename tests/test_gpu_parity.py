@@ -188,3 +188,74 @@ def test_layer_stack_chains_layers_with_per_layer_N(stb):
         got = bufs[k + 1].double().cpu().numpy()
         tol = TOL * np.abs(y_ref).max() + (2.0 ** -11 * np.abs(y_ref).max() if k < 2 else 0)
         assert np.abs(got - y_ref).max() <= tol
+
+
+def _check_gemm(stb, layer, L, T, seed, out_dtype=None, rows=None, toks=None):
+    """stb_gemm against the float64 dequantise-then-matmul on bf16 activations."""
+    import torch
+    x = si.activations(T, L.m, seed, "bf16")                       # float32 values exactly representable in bf16
+    xd = torch.from_numpy(x).cuda().to(torch.bfloat16)
+    assert np.array_equal(xd.float().cpu().numpy(), x)
+    y = stb.gemm(layer, xd, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    assert int(layer.dev_status.item()) == 0
+    if rows is None:
+        y_ref = oracle.matmul(oracle.decode(L), x.astype(np.float64))
+        got = y.double().cpu().numpy()
+    else:
+        y_ref = oracle.layer_rows(L, rows, x[toks].astype(np.float64))
+        got = y.double().cpu().numpy()[np.ix_(toks, rows)]
+    scale = np.abs(y_ref).max()
+    tol = TOL * scale + (2.0 ** -8 * scale if out_dtype is not None else 0.0)   # one bf16 rounding of the result
+    err = np.abs(got - y_ref).max()
+    assert err <= tol, (err, tol)
+    return err / scale
+
+
+@pytest.mark.parametrize("N", [4, 5, 6])
+@pytest.mark.parametrize("n,m,T", [(40, 256, 1), (100, 384, 37), (128, 128, 256), (300, 512, 300), (257, 1024, 513)])
+def test_gemm_quantized_layers(stb, N, n, m, T):
+    """Prefill GEMM on quantizer output: ragged rows (n not a multiple of 128), ragged tokens, several
+    K stages, one and several output tiles."""
+    import torch
+    L = _quantized(n, m, N, 2000 + 10 * N + n)
+    layer = stb.pack_numpy(_fields(L))
+    _check_gemm(stb, layer, L, T, 50 + T)
+    _check_gemm(stb, layer, L, T, 51 + T, out_dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("N,max_salient", [(4, 7), (6, 30)])
+def test_gemm_many_salient_columns(stb, N, max_salient):
+    d = si.logical_layer(200, 512, N, 500 + max_salient, max_salient=max_salient)
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    _check_gemm(stb, layer, L, 70, 9)
+
+
+def test_gemm_split_k_uses_the_workspace(stb):
+    """Few output tiles and a long K: the launch splits K, partial sums go through the caller's workspace."""
+    import torch
+    n, m, N, T = 128, 4096, 4, 200
+    d = si.logical_layer(n, m, N, 610)
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    assert stb.gemm_workspace(n, m, N, T) >= 2 * T * n * 4
+    _check_gemm(stb, layer, L, T, 11)
+    x = torch.zeros(T, m, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(stb.StbError) as e:                      # workspace too small: refused on the host
+        stb._check(stb._lib.stb_gemm(stb._ptr(layer.buf), n, m, N, stb._ptr(x), T, m, stb._ptr(torch.empty(T, n, device="cuda")),
+                                     stb.STB_F32, n, None, 0, stb._ptr(layer.dev_status), stb._stream()), "stb_gemm")
+    assert e.value.status == stb.STB_ERR_SIZE
+
+
+@pytest.mark.parametrize("n,m", [(8192, 8192), (1024, 8192)])
+def test_gemm_full_size_sampled(stb, n, m):
+    """LLaMA-2-70B prefill shapes at 4:8, 2048 tokens: sampled (token, row) pairs against the oracle."""
+    N, T = 4, 2048
+    d = si.logical_layer(n, m, N, si.seed_for(4, n // 1024))
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    g = np.random.default_rng(n)
+    rows = np.unique(np.concatenate([[0, 1, n - 1], g.choice(n, 96, replace=False)])).astype(np.int32)
+    toks = np.unique(np.concatenate([[0, 255, 256, T - 1], g.choice(T, 40, replace=False)]))
+    _check_gemm(stb, layer, L, T, si.seed_for(4, 9), rows=rows, toks=toks)
