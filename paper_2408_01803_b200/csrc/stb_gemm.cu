@@ -10,7 +10,9 @@
 //   warp 0      TMA producer (one lane): X slices
 //   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage, tcgen05.commit frees
 //               the stage; also allocates / frees the 256 TMEM columns
-//   warps 2..5  decode: warp w owns rows 32 (w % 4) .. +31 of the tile = one packed row tile;
+//   warps 2..   decode: warp w works on rows 32 (w % 4) .. +31 of the tile = one packed row tile;
+//               kGroups warps share a row tile, each taking 4 / kGroups of the four rows a lane
+//               owns (one warp alone per scheduler would be bound by instruction latency);
 //               per 128-column block it loads the lane's words (prefetching the next block),
 //               converts the four fp16 scales of its rows to bf16 (RN-even) and writes the two
 //               64-column halves of the block into two stages; afterwards the same warps read
@@ -35,6 +37,11 @@ constexpr int kBM = 128;          // rows of W^ per CTA (UMMA M)
 constexpr int kBN = 256;          // tokens per CTA (UMMA N)
 constexpr int kBK = 64;           // K per stage: one 128-byte swizzle row of bf16
 constexpr int kStages = 4;
+#ifndef STB_GEMM_GROUPS
+#define STB_GEMM_GROUPS 2
+#endif
+constexpr int kGroups = STB_GEMM_GROUPS;                // decode warps per 32-row quarter: 1, 2 or 4
+constexpr int kGemmThreads = 64 + 128 * kGroups;
 constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
 constexpr uint32_t kStageB = kBN * kBK * 2;      // 32 KB
 constexpr uint32_t kGemmTab = 0;                                   // position table (576 B)
@@ -92,11 +99,15 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
 // Instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 
-// Bounded mbarrier wait with a CTA-wide abort flag (a volatile int in shared memory).
+// Bounded mbarrier wait with a CTA-wide abort flag (a volatile int in shared memory).  The two
+// single-lane roles back off between polls so that their spinning does not take issue slots from
+// the decode warps that share their schedulers.
+template <bool kBackoff = false>
 __device__ __forceinline__ bool gemm_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
+    if (kBackoff) __nanosleep(32);
     if (*abort_flag) return false;
     if (clock64() - t0 > kGemmWaitLimit) { *abort_flag = 1; return false; }
   }
@@ -107,9 +118,129 @@ __device__ __forceinline__ uint32_t bf16_bits(uint32_t h16) {
   return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half((unsigned short)h16))));
 }
 
+// What a decode warp needs to know.
+struct DecodeArgs {
+  const uint8_t* packed; const Header* hdr; uint8_t* smem; volatile int* abort_flag;
+  uint32_t bar_full, bar_empty;
+  int mt, b0, b1, nblk, ntile, q, lane;
+};
+
+// Decode role of one warp: rows J0 .. J0 + NJ - 1 (of the four rows g + 8 j each lane owns) of
+// packed row tile 4 mt + q, for every block of the CTA's K range, written into the A stages.
+template <int N, int J0, int NJ>
+__device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
+  const uint8_t* packed = da.packed;
+  const Header* hdr = da.hdr;
+  uint8_t* smem = da.smem;
+  volatile int* abort_flag = da.abort_flag;
+  const uint32_t bar_full = da.bar_full, bar_empty = da.bar_empty;
+  const int mt = da.mt, b0 = da.b0, b1 = da.b1, nblk = da.nblk, ntile = da.ntile, q = da.q, lane = da.lane;
+    const int g = lane >> 2, t = lane & 3;
+    const int rtile = mt * 4 + q;                 // packed row tile
+    const bool live = rtile < ntile;
+    const uint2* ptab = reinterpret_cast<const uint2*>(smem + kGemmTab);
+    const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+    const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
+    const int spb = (int)hdr->spb;
+    const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
+                              (size_t)rtile * nblk * resid_tile_bytes(spb);
+    constexpr uint32_t tbytes = tile_bytes(N);
+    LaneTile<N> cur = {}, nxt = {};
+    // salient metadata of a block, fetched one block ahead like the tile: the count, and for the
+    // lane's slots t, t + 4 (slots beyond 8 are fetched on demand) the column bytes and residual words
+    struct Sal { int nsal; uint32_t cw[2], rw[2]; };
+    auto load_sal = [&](int b, Sal& z) {
+      z.nsal = (int)__ldg(&binfo[b].nsal);
+      z.cw[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols));
+      z.cw[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + 1);
+      const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb);
+      z.rw[0] = spb > 0 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 0))) : 0x55555555u;
+      z.rw[1] = spb > 4 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 1))) : 0x55555555u;
+    };
+    Sal csal = {0, {0, 0}, {0, 0}}, nsalv = {0, {0, 0}, {0, 0}};
+    if (live && b0 < b1) { load_lane_tile<N>(rtbase + (size_t)b0 * tbytes, lane, cur); load_sal(b0, csal); }
+    bool ok = true;
+    for (int b = b0; b < b1 && ok; ++b) {
+      if (live && b + 1 < b1) { load_lane_tile<N>(rtbase + (size_t)(b + 1) * tbytes, lane, nxt); load_sal(b + 1, nsalv); }
+      // bf16 scale bytes of the lane's four rows
+      uint32_t A16[4] = {0, 0, 0, 0}, B16[4] = {0, 0, 0, 0};
+      float a1f[4] = {0.f, 0.f, 0.f, 0.f}, a2f[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int j = J0; j < J0 + NJ; ++j) {
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint32_t v = live ? bf16_bits(scale_bits<N>(cur, j, c)) : 0u;
+          lo |= (v & 0xFFu) << (8 * c);
+          hi |= (v >> 8) << (8 * c);
+        }
+        A16[j] = lo; B16[j] = hi;
+        a1f[j] = live ? __half2float(__ushort_as_half((unsigned short)scale_bits<N>(cur, j, 3))) : 0.f;
+        a2f[j] = live ? __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(cur, j))) : 0.f;
+      }
+      FastRows<N> fr;
+      fr.init(cur, A16, B16);
+      uint32_t XL[4] = {0, 0, 0, 0}, XH[4] = {0, 0, 0, 0};
+      if (N == 5) {
+#pragma unroll
+        for (int j = J0; j < J0 + NJ; ++j) fr.high(j, 0, XL[j], XH[j]);
+      }
+      const int nsal = live ? csal.nsal : 0;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int it = 2 * (b - b0) + h, s = it % kStages;
+        if (!gemm_wait(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        uint8_t* As = smem + kGemmA + s * kStageA;
+#pragma unroll
+        for (int j = J0; j < J0 + NJ; ++j) {
+          uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl) {
+            const int sidx = 2 * h + sl;                       // slot s of the block, group 4 sidx + t
+            uint32_t f[4] = {0, 0, 0, 0};
+            if (live) {
+              if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
+              const uint2 P = ptab[keep_index_of(cur.mask, j, sidx)];
+              fr.slot2(j, sidx, P.x, P.y, XL[j], XH[j], f);
+            }
+            const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
+            *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
+          }
+        }
+        // salient columns of this half: bf16( fl32( s1 a_sal1 + s2 a_sal2 ) ), slot sq handled by lane t = sq % 4
+        if (nsal > 0) {
+          __syncwarp();
+          for (int i = 0; 4 * i + t < nsal; ++i) {
+            const int sq = 4 * i + t;
+            const uint32_t cwd = i == 0 ? csal.cw[0] : (i == 1 ? csal.cw[1] : __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + i));
+            const int c = (int)((cwd >> (8 * t)) & 0xFFu);
+            if ((c >> 6) != h) continue;
+            const uint32_t word = i == 0 ? csal.rw[0] : (i == 1 ? csal.rw[1] :
+                __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, i))));
+            const int c64 = c & 63;
+#pragma unroll
+            for (int j = J0; j < J0 + NJ; ++j) {
+              const uint32_t rc = resid_code(word, j, sq & 3);
+              if (rc == 1u) continue;
+              unsigned short* pv = reinterpret_cast<unsigned short*>(As + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
+              const bool neg1 = (*pv & 0x8000u) != 0;
+              const float v = __fadd_rn(neg1 ? -a1f[j] : a1f[j], rc == 0u ? a2f[j] : -a2f[j]);
+              *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+            }
+          }
+        }
+        fence_async_smem();          // generic-proxy writes -> visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_full + 8 * s);
+      }
+      if (live && b + 1 < b1) { cur = nxt; csal = nsalv; }
+    }
+
+}
+
 // ------------------------------------------------------------------------------------------
 template <int N>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict__ packed, int n, int m, int T,
             void* __restrict__ Y, int y_bf16, size_t ldy, float* __restrict__ ws, int ksplit, int bps,
             uint32_t box_bytes, int* dev_status) {
@@ -131,7 +262,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kGemmBars + 8 * (2 * kStages + 1) + 8);
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 5); mbar_init(bar_empty + 8 * i, 1); }
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 1 + 4 * kGroups); mbar_init(bar_empty + 8 * i, 1); }
     mbar_init(bar_accum, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -149,7 +280,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     if (lane == 0) {
       for (int it = 0; it < nstage; ++it) {
         const int s = it % kStages;
-        if (!gemm_wait(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) break;
+        if (!gemm_wait<true>(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) break;
         mbar_expect_tx(bar_full + 8 * s, box_bytes);
         tma_load_2d(sbase + kGemmB + s * kStageB, &xmap, (b0 * 2 + it) * kBK, tt * kBN, bar_full + 8 * s);
       }
@@ -163,7 +294,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     if (lane == 0) {
       for (int it = 0; it < nstage; ++it) {
         const int s = it % kStages;
-        if (!gemm_wait(bar_full + 8 * s, (uint32_t)(it / kStages) & 1u, abort_flag)) break;
+        if (!gemm_wait<true>(bar_full + 8 * s, (uint32_t)(it / kStages) & 1u, abort_flag)) break;
         tc_fence_after();
         const uint64_t ad = umma_desc(sbase + kGemmA + s * kStageA), bd = umma_desc(sbase + kGemmB + s * kStageB);
 #pragma unroll
@@ -175,100 +306,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     }
   } else {
     // ---------------- decode warps ----------------
-    const int q = warp & 3;                       // row quarter of the tile = TMEM lane quarter
-    const int g = lane >> 2, t = lane & 3;
-    const int rtile = mt * 4 + q;                 // packed row tile
-    const bool live = rtile < ntile;
-    const uint2* ptab = reinterpret_cast<const uint2*>(smem + kGemmTab);
-    const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
-    const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
-    const int spb = (int)hdr->spb;
-    const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                              (size_t)rtile * nblk * resid_tile_bytes(spb);
-    constexpr uint32_t tbytes = tile_bytes(N);
-    LaneTile<N> cur = {}, nxt = {};
-    if (live && b0 < b1) load_lane_tile<N>(rtbase + (size_t)b0 * tbytes, lane, cur);
-    bool ok = true;
-    for (int b = b0; b < b1 && ok; ++b) {
-      if (live && b + 1 < b1) load_lane_tile<N>(rtbase + (size_t)(b + 1) * tbytes, lane, nxt);
-      // bf16 scale bytes of the lane's four rows
-      uint32_t A16[4], B16[4];
-      float a1f[4], a2f[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        uint32_t lo = 0, hi = 0;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t v = live ? bf16_bits(scale_bits<N>(cur, j, c)) : 0u;
-          lo |= (v & 0xFFu) << (8 * c);
-          hi |= (v >> 8) << (8 * c);
-        }
-        A16[j] = lo; B16[j] = hi;
-        a1f[j] = live ? __half2float(__ushort_as_half((unsigned short)scale_bits<N>(cur, j, 3))) : 0.f;
-        a2f[j] = live ? __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(cur, j))) : 0.f;
-      }
-      FastRows<N> fr;
-      fr.init(cur, A16, B16);
-      uint32_t XL[4] = {0, 0, 0, 0}, XH[4] = {0, 0, 0, 0};
-      if (N == 5) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) fr.high(j, 0, XL[j], XH[j]);
-      }
-      const int nsal = live ? (int)binfo[b].nsal : 0;
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int it = 2 * (b - b0) + h, s = it % kStages;
-        if (!gemm_wait(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-        uint8_t* As = smem + kGemmA + s * kStageA;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
-#pragma unroll
-          for (int sl = 0; sl < 2; ++sl) {
-            const int sidx = 2 * h + sl;                       // slot s of the block, group 4 sidx + t
-            uint32_t f[4] = {0, 0, 0, 0};
-            if (live) {
-              if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
-              const uint2 P = ptab[keep_index_of(cur.mask, j, sidx)];
-              fr.slot2(j, sidx, P.x, P.y, XL[j], XH[j], f);
-            }
-            const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
-            *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
-          }
-        }
-        // salient columns of this half: bf16( fl32( s1 a_sal1 + s2 a_sal2 ) ), slot sq handled by lane t = sq % 4
-        if (nsal > 0) {
-          __syncwarp();
-          for (int sq = t; sq < nsal; sq += 4) {
-            const int c = binfo[b].cols[sq];
-            if ((c >> 6) != h) continue;
-            const uint32_t word = __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2)));
-            const int c64 = c & 63;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint32_t rc = resid_code(word, j, sq & 3);
-              if (rc == 1u) continue;
-              unsigned short* pv = reinterpret_cast<unsigned short*>(As + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
-              const bool neg1 = (*pv & 0x8000u) != 0;
-              const float v = __fadd_rn(neg1 ? -a1f[j] : a1f[j], rc == 0u ? a2f[j] : -a2f[j]);
-              *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-            }
-          }
-        }
-        fence_async_smem();          // generic-proxy writes -> visible to the tensor core
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_full + 8 * s);
-      }
-      if (live && b + 1 < b1) cur = nxt;
+    const int gi = (warp - 2) >> 2;               // decode group: which of the lane's four rows this warp takes
+    DecodeArgs da;
+    da.packed = packed; da.hdr = hdr; da.smem = smem; da.abort_flag = abort_flag;
+    da.bar_full = bar_full; da.bar_empty = bar_empty;
+    da.mt = mt; da.b0 = b0; da.b1 = b1; da.nblk = nblk; da.ntile = ntile; da.q = warp & 3; da.lane = lane;
+    if (kGroups == 1) decode_rows<N, 0, 4>(da);
+    else if (kGroups == 2) { if (gi == 0) decode_rows<N, 0, 2>(da); else decode_rows<N, 2, 2>(da); }
+    else {
+      if (gi == 0) decode_rows<N, 0, 1>(da);
+      else if (gi == 1) decode_rows<N, 1, 1>(da);
+      else if (gi == 2) decode_rows<N, 2, 1>(da);
+      else decode_rows<N, 3, 1>(da);
     }
 
     // ---------------- epilogue: TMEM -> registers -> Y ----------------
+    const int q = warp & 3;                        // TMEM lane quarter of this warp
     if (gemm_wait(bar_accum, 0u, abort_flag) && nstage > 0) {
       tc_fence_after();
       const int row = mt * kBM + 32 * q + lane;                // output feature (row of W^)
       float* wsz = ws ? ws + (size_t)kz * (size_t)T * (size_t)n : nullptr;
 #pragma unroll 1
-      for (int cc = 0; cc < kBN / 32; ++cc) {
+      for (int cc = gi; cc < kBN / 32; cc += kGroups) {        // the groups share the 8 column chunks
         uint32_t r[32];
         tmem_ld32(tmem_d + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * cc), r);
         if (row < n) {
@@ -288,7 +347,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
   }
 
   // the MMA thread makes sure the tensor core is done with TMEM before it is freed
-  if (warp == 1 && lane == 0) gemm_wait(bar_accum, 0u, abort_flag);
+  if (warp == 1 && lane == 0) gemm_wait<true>(bar_accum, 0u, abort_flag);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_d, kBN);
@@ -361,7 +420,7 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
   }
   const int nblk = m / kBlock, bps = (nblk + ks - 1) / ks;
   dim3 grid((unsigned)((T + kBN - 1) / kBN), (unsigned)((n + kBM - 1) / kBM), (unsigned)ks);
-  gemm_kernel<N><<<grid, 192, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, ks > 1 ? static_cast<float*>(ws) : nullptr,
+  gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, ks > 1 ? static_cast<float*>(ws) : nullptr,
                                               ks, bps, box_rows * kBK * 2, dev_status);
   if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   if (ks > 1) {
