@@ -186,53 +186,73 @@ __device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
         for (int j = J0; j < J0 + NJ; ++j) fr.high(j, 0, XL[j], XH[j]);
       }
       const int nsal = live ? csal.nsal : 0;
+      // position selectors of the warp's slots of this block, looked up before the stage waits
+      uint2 P[4][4];
+#pragma unroll
+      for (int j = J0; j < J0 + NJ; ++j)
+#pragma unroll
+        for (int sidx = 0; sidx < 4; ++sidx) P[j][sidx] = live ? ptab[keep_index_of(cur.mask, j, sidx)] : make_uint2(0, 0);
+      // Salient patches of this block: (salient slot sq, row j) pairs, nsal * NJ of them, dealt to
+      // the four lanes t of a lane group; the first one per lane is prepared here.
+      const int np = nsal * NJ;
+      int pc0 = -1, pj0 = J0; uint32_t prc0 = 1u;          // column, row, residual code of patch t
+      if (t < np) {
+        const int sq = t / NJ;
+        pj0 = J0 + t % NJ;
+        const uint32_t cwd = sq < 4 ? csal.cw[0] : (sq < 8 ? csal.cw[1] : __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + (sq >> 2)));
+        pc0 = (int)((cwd >> (8 * (sq & 3))) & 0xFFu);
+        const uint32_t word = sq < 4 ? csal.rw[0] : (sq < 8 ? csal.rw[1] :
+            __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2))));
+        prc0 = resid_code(word, pj0, sq & 3);
+      }
+      // both 64-column halves of the block go out together: two consecutive stages
+      const int it0 = 2 * (b - b0), s0 = it0 % kStages, s1 = (it0 + 1) % kStages;
+      if (!gemm_wait(bar_empty + 8 * s0, ((uint32_t)(it0 / kStages) & 1u) ^ 1u, abort_flag) ||
+          !gemm_wait(bar_empty + 8 * s1, ((uint32_t)((it0 + 1) / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      uint8_t* Ah[2] = {smem + kGemmA + s0 * kStageA, smem + kGemmA + s1 * kStageA};
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        const int it = 2 * (b - b0) + h, s = it % kStages;
-        if (!gemm_wait(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-        uint8_t* As = smem + kGemmA + s * kStageA;
 #pragma unroll
         for (int j = J0; j < J0 + NJ; ++j) {
-          uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
+          uint8_t* rowp = Ah[h] + (size_t)(4 * q + j) * 1024 + g * 128;
 #pragma unroll
           for (int sl = 0; sl < 2; ++sl) {
             const int sidx = 2 * h + sl;                       // slot s of the block, group 4 sidx + t
             uint32_t f[4] = {0, 0, 0, 0};
             if (live) {
               if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
-              const uint2 P = ptab[keep_index_of(cur.mask, j, sidx)];
-              fr.slot2(j, sidx, P.x, P.y, XL[j], XH[j], f);
+              fr.slot2(j, sidx, P[j][sidx].x, P[j][sidx].y, XL[j], XH[j], f);
             }
             const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
             *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
           }
         }
-        // salient columns of this half: bf16( fl32( s1 a_sal1 + s2 a_sal2 ) ), slot sq handled by lane t = sq % 4
-        if (nsal > 0) {
-          __syncwarp();
-          for (int i = 0; 4 * i + t < nsal; ++i) {
-            const int sq = 4 * i + t;
-            const uint32_t cwd = i == 0 ? csal.cw[0] : (i == 1 ? csal.cw[1] : __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + i));
-            const int c = (int)((cwd >> (8 * t)) & 0xFFu);
-            if ((c >> 6) != h) continue;
-            const uint32_t word = i == 0 ? csal.rw[0] : (i == 1 ? csal.rw[1] :
-                __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, i))));
-            const int c64 = c & 63;
-#pragma unroll
-            for (int j = J0; j < J0 + NJ; ++j) {
-              const uint32_t rc = resid_code(word, j, sq & 3);
-              if (rc == 1u) continue;
-              unsigned short* pv = reinterpret_cast<unsigned short*>(As + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
-              const bool neg1 = (*pv & 0x8000u) != 0;
-              const float v = __fadd_rn(neg1 ? -a1f[j] : a1f[j], rc == 0u ? a2f[j] : -a2f[j]);
-              *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-            }
-          }
-        }
-        fence_async_smem();          // generic-proxy writes -> visible to the tensor core
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_full + 8 * s);
       }
+      // salient columns: bf16( fl32( s1 a_sal1 + s2 a_sal2 ) ) replaces the value the main decode
+      // wrote (whose sign is s1); patch p = t + 4 i of the block's list belongs to lane t
+      if (nsal > 0) {
+        __syncwarp();
+        for (int p = t; p < np; p += 4) {
+          int c = pc0, j = pj0; uint32_t rc = prc0;
+          if (p >= 4) {
+            const int sq = p / NJ;
+            j = J0 + p % NJ;
+            c = binfo[b].cols[sq];
+            rc = resid_code(__ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2))), j, sq & 3);
+          }
+          if (rc == 1u) continue;
+          const int c64 = c & 63;
+          unsigned short* pv = reinterpret_cast<unsigned short*>(Ah[c >> 6] + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
+          const bool neg1 = (*pv & 0x8000u) != 0;
+          const float a1 = j == 0 ? a1f[0] : (j == 1 ? a1f[1] : (j == 2 ? a1f[2] : a1f[3]));
+          const float a2 = j == 0 ? a2f[0] : (j == 1 ? a2f[1] : (j == 2 ? a2f[2] : a2f[3]));
+          const float v = __fadd_rn(neg1 ? -a1 : a1, rc == 0u ? a2 : -a2);
+          *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+        }
+      }
+      fence_async_smem();          // generic-proxy writes -> visible to the tensor core
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(bar_full + 8 * s0); mbar_arrive(bar_full + 8 * s1); }
       if (live && b + 1 < b1) { cur = nxt; csal = nsalv; }
     }
 
