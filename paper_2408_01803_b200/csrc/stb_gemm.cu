@@ -2,14 +2,16 @@
 // (tcgen05.mma, fp32 accumulators in tensor memory).  The compute-bound prefilling stage of
 // Appendix C.2: N = sequence length x batch tokens against one packed layer.
 //
-// One CTA computes a 128 (rows of W^) x 256 (tokens) tile of the output, D = A B^T with
+// One CTA computes a 128 (rows of W^) x 256 kAcc (tokens) tile of the output, D = A B^T with
 //   A = 128 x 64 bf16 slice of W^, decoded from the packed tiles into shared memory in the
 //       K-major 128-byte-swizzled layout the tensor core reads,
-//   B = 256 x 64 bf16 slice of X, brought in by TMA with the same swizzle,
+//   B = kAcc slices of 256 x 64 bf16 of X, brought in by TMA with the same swizzle; every decoded
+//       A stage is multiplied with all of them (kAcc accumulators of 256 TMEM columns), which
+//       divides the decode work per flop by kAcc,
 // in a ring of kStages stages over K.  Warp roles:
 //   warp 0      TMA producer (one lane): X slices
 //   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage, tcgen05.commit frees
-//               the stage; also allocates / frees the 256 TMEM columns
+//               and accumulator, tcgen05.commit frees the stage; also allocates / frees TMEM
 //   warps 2..   decode: warp w works on rows 32 (w % 4) .. +31 of the tile = one packed row tile;
 //               kGroups warps share a row tile, each taking 4 / kGroups of the four rows a lane
 //               owns (one warp alone per scheduler would be bound by instruction latency);
@@ -34,16 +36,21 @@
 namespace stb {
 
 constexpr int kBM = 128;          // rows of W^ per CTA (UMMA M)
-constexpr int kBN = 256;          // tokens per CTA (UMMA N)
+constexpr int kBN = 256;          // tokens per accumulator (UMMA N)
+#ifndef STB_GEMM_ACC
+#define STB_GEMM_ACC 2
+#endif
+constexpr int kAcc = STB_GEMM_ACC;              // accumulators per CTA: a decoded A stage is used kAcc times
+constexpr int kTok = kBN * kAcc;                // tokens per CTA
 constexpr int kBK = 64;           // K per stage: one 128-byte swizzle row of bf16
-constexpr int kStages = 4;
+constexpr int kStages = kAcc == 1 ? 4 : 2;
 #ifndef STB_GEMM_GROUPS
-#define STB_GEMM_GROUPS 2
+#define STB_GEMM_GROUPS 4
 #endif
 constexpr int kGroups = STB_GEMM_GROUPS;                // decode warps per 32-row quarter: 1, 2 or 4
 constexpr int kGemmThreads = 64 + 128 * kGroups;
 constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
-constexpr uint32_t kStageB = kBN * kBK * 2;      // 32 KB
+constexpr uint32_t kStageB = kTok * kBK * 2;     // 32 KB per accumulator
 constexpr uint32_t kGemmTab = 0;                                   // position table (576 B)
 constexpr uint32_t kGemmBars = 1024;                               // full[4], empty[4], accum, tmem slot, abort
 constexpr uint32_t kGemmA = 2048;                                  // 1024-byte aligned stages
@@ -205,6 +212,7 @@ __device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
             __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2))));
         prc0 = resid_code(word, pj0, sq & 3);
       }
+      if constexpr (kStages >= 4) {
       // both 64-column halves of the block go out together: two consecutive stages
       const int it0 = 2 * (b - b0), s0 = it0 % kStages, s1 = (it0 + 1) % kStages;
       if (!gemm_wait(bar_empty + 8 * s0, ((uint32_t)(it0 / kStages) & 1u) ^ 1u, abort_flag) ||
@@ -253,6 +261,53 @@ __device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
       fence_async_smem();          // generic-proxy writes -> visible to the tensor core
       __syncwarp();
       if (lane == 0) { mbar_arrive(bar_full + 8 * s0); mbar_arrive(bar_full + 8 * s1); }
+      } else {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int it = 2 * (b - b0) + h, st = it % kStages;
+        if (!gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        uint8_t* As = smem + kGemmA + st * kStageA;
+#pragma unroll
+        for (int j = J0; j < J0 + NJ; ++j) {
+          uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl) {
+            const int sidx = 2 * h + sl;
+            uint32_t f[4] = {0, 0, 0, 0};
+            if (live) {
+              if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
+              fr.slot2(j, sidx, P[j][sidx].x, P[j][sidx].y, XL[j], XH[j], f);
+            }
+            const int chunk = 4 * sl + t;
+            *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
+          }
+        }
+        if (nsal > 0) {
+          __syncwarp();
+          for (int p = t; p < np; p += 4) {
+            int c = pc0, j = pj0; uint32_t rc = prc0;
+            if (p >= 4) {
+              const int sq = p / NJ;
+              j = J0 + p % NJ;
+              c = binfo[b].cols[sq];
+              rc = resid_code(__ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2))), j, sq & 3);
+            }
+            if ((c >> 6) != h || rc == 1u) continue;
+            const int c64 = c & 63;
+            unsigned short* pv = reinterpret_cast<unsigned short*>(As + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
+            const bool neg1 = (*pv & 0x8000u) != 0;
+            const float a1 = j == 0 ? a1f[0] : (j == 1 ? a1f[1] : (j == 2 ? a1f[2] : a1f[3]));
+            const float a2 = j == 0 ? a2f[0] : (j == 1 ? a2f[1] : (j == 2 ? a2f[2] : a2f[3]));
+            const float v = __fadd_rn(neg1 ? -a1 : a1, rc == 0u ? a2 : -a2);
+            *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_full + 8 * st);
+      }
+      }
+      if (!ok) break;
       if (live && b + 1 < b1) { cur = nxt; csal = nsalv; }
     }
 
@@ -289,7 +344,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     fence_async_smem();
   }
   for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x) reinterpret_cast<uint2*>(smem + kGemmTab)[i] = g_pos_table.v[N][i];
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kBN);
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTok);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -301,8 +356,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
       for (int it = 0; it < nstage; ++it) {
         const int s = it % kStages;
         if (!gemm_wait<true>(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) break;
-        mbar_expect_tx(bar_full + 8 * s, box_bytes);
-        tma_load_2d(sbase + kGemmB + s * kStageB, &xmap, (b0 * 2 + it) * kBK, tt * kBN, bar_full + 8 * s);
+        mbar_expect_tx(bar_full + 8 * s, box_bytes * kAcc);
+#pragma unroll
+        for (int a = 0; a < kAcc; ++a)
+          tma_load_2d(sbase + kGemmB + s * kStageB + a * (kBN * kBK * 2), &xmap, (b0 * 2 + it) * kBK, tt * kTok + a * kBN, bar_full + 8 * s);
       }
       if (*abort_flag) {       // let copies in flight land before the CTA gives its shared memory up
         const long long t0 = clock64();
@@ -316,10 +373,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
         const int s = it % kStages;
         if (!gemm_wait<true>(bar_full + 8 * s, (uint32_t)(it / kStages) & 1u, abort_flag)) break;
         tc_fence_after();
-        const uint64_t ad = umma_desc(sbase + kGemmA + s * kStageA), bd = umma_desc(sbase + kGemmB + s * kStageB);
+        const uint64_t ad = umma_desc(sbase + kGemmA + s * kStageA);
 #pragma unroll
-        for (int kk = 0; kk < kBK / 16; ++kk)
-          umma_bf16(tmem_d, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+        for (int a = 0; a < kAcc; ++a) {
+          const uint64_t bd = umma_desc(sbase + kGemmB + s * kStageB + a * (kBN * kBK * 2));
+#pragma unroll
+          for (int kk = 0; kk < kBK / 16; ++kk)
+            umma_bf16(tmem_d + (uint32_t)(a * kBN), ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+        }
         umma_commit(bar_empty + 8 * s);          // the stage is free once these MMAs have read it
       }
       umma_commit(bar_accum);                    // all MMAs issued so far have completed
@@ -347,13 +408,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
       const int row = mt * kBM + 32 * q + lane;                // output feature (row of W^)
       float* wsz = ws ? ws + (size_t)kz * (size_t)T * (size_t)n : nullptr;
 #pragma unroll 1
-      for (int cc = gi; cc < kBN / 32; cc += kGroups) {        // the groups share the 8 column chunks
+      for (int cc = gi; cc < kTok / 32; cc += kGroups) {       // the groups share the column chunks
         uint32_t r[32];
         tmem_ld32(tmem_d + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * cc), r);
         if (row < n) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const int tok = tt * kBN + 32 * cc + i;
+            const int tok = tt * kTok + 32 * cc + i;
             if (tok < T) {
               const float v = __uint_as_float(r[i]);
               if (wsz) wsz[(size_t)tok * n + row] = v;
@@ -370,7 +431,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
   if (warp == 1 && lane == 0) gemm_wait<true>(bar_accum, 0u, abort_flag);
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_d, kBN);
+  if (warp == 1) tmem_dealloc(tmem_d, kTok);
   if (threadIdx.x == 0 && *abort_flag && dev_status) *dev_status = STB_ERR_TIMEOUT;
 }
 
@@ -391,7 +452,7 @@ __global__ void gemm_reduce_kernel(const float* __restrict__ ws, int ksplit, int
 static int gemm_ksplit(int n, int m, int T) {
   static int forced = -1;
   if (forced < 0) { const char* e = getenv("STB_GEMM_KSPLIT"); forced = e ? atoi(e) : 0; }
-  const int tiles = ((n + kBM - 1) / kBM) * ((T + kBN - 1) / kBN), nblk = m / kBlock;
+  const int tiles = ((n + kBM - 1) / kBM) * ((T + kTok - 1) / kTok), nblk = m / kBlock;
   int ks = 1;
   if (forced >= 1 && forced <= 16) ks = forced;
   else if (tiles < 100) ks = 148 / tiles;
@@ -439,7 +500,7 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
     attr_done = true;
   }
   const int nblk = m / kBlock, bps = (nblk + ks - 1) / ks;
-  dim3 grid((unsigned)((T + kBN - 1) / kBN), (unsigned)((n + kBM - 1) / kBM), (unsigned)ks);
+  dim3 grid((unsigned)((T + kTok - 1) / kTok), (unsigned)((n + kBM - 1) / kBM), (unsigned)ks);
   gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, ks > 1 ? static_cast<float*>(ws) : nullptr,
                                               ks, bps, box_rows * kBK * 2, dev_status);
   if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
