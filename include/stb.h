@@ -132,6 +132,25 @@ int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size
              stb_dtype ydt, size_t ldy, void *ws, size_t ws_bytes, int *dev_status,
              void *stream);
 
+/* stb_gemm without a workspace argument (the paper has no counterpart: this entry point exists
+ * for the integration, not for the method).  Some hosts of this library may not allocate device
+ * memory while they run: a serving process that gave its whole memory budget to one arena at
+ * start-up, or a latency-critical loop in which a cudaMalloc (which synchronises the device)
+ * is forbidden.  For them the split-K partial sums go into a fixed 8 MiB array that is part of
+ * the library image: every GPU that loads the library holds these 8 MiB until the process
+ * exits.  Same arguments, results and errors as stb_gemm, except:
+ *   - a call whose stb_gemm_workspace() exceeds 8 MiB returns STB_ERR_SIZE and launches
+ *     nothing (use stb_gemm with your own workspace for it);
+ *   - the first call on each device looks the array's device address up (with that device
+ *     current); make that first call outside any stream capture;
+ *   - all calls share the one array.  It keeps whatever the last call left there; nothing in
+ *     it has to start at zero, because every call writes each partial sum before reading it.
+ *     Two calls that may run on the GPU at the same time (different streams) would overwrite
+ *     each other's partial sums: keep calls of this entry point on one stream, or order them.
+ * It calls no allocation routine of CUDA or of any library. */
+int stb_gemm_noalloc(const void *packed, int n, int m, int N, const void *X, int T, size_t ldx,
+                     void *Y, stb_dtype ydt, size_t ldy, int *dev_status, void *stream);
+
 /* Runs `count` GEMV steps in order on one stream; every step carries its own N (layer-wise
  * N:M assignment, Section 3.3).  steps is a HOST array.  Launches only. */
 int stb_layer_stack(const stb_step *steps, int count, int *dev_status, void *stream);

@@ -21,7 +21,7 @@ STB_ERR_UNSUPPORTED, STB_ERR_CORRUPT, STB_ERR_TIMEOUT, STB_ERR_CUDA = 5, 6, 7, 8
 STB_F16, STB_BF16, STB_F32 = 0, 1, 2
 
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv",
-           "stb_gemm_workspace", "stb_gemm", "stb_layer_stack", "stb_layer_stack_host", "stb_status_str"]
+           "stb_gemm_workspace", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host", "stb_status_str"]
 
 
 class StbError(RuntimeError):
@@ -60,6 +60,7 @@ def _load():
     lib.stb_gemv.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_gemm_workspace.argtypes = [i, i, i, i, p(z)]
     lib.stb_gemm.argtypes = [v, i, i, i, v, i, z, v, i, z, v, z, v, v]
+    lib.stb_gemm_noalloc.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_layer_stack.argtypes = [p(_Step), i, v, v]
     lib.stb_layer_stack_host.argtypes = [p(_Step), i, v, z, v, z, v, v]
     lib.stb_status_str.argtypes = [i]
@@ -198,6 +199,20 @@ def gemm(layer: PackedLayer, X, out=None, out_dtype=None, ws=None, stream=None):
     _check(_lib.stb_gemm(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(X), T, X.stride(0), _ptr(out),
                          ydt, out.stride(0), _ptr(ws), (ws.numel() * ws.element_size()) if ws is not None else 0,
                          _ptr(layer.dev_status), _stream(stream)), "stb_gemm")
+    return out
+
+
+def gemm_noalloc(layer: PackedLayer, X, out, stream=None):
+    """stb_gemm_noalloc: like gemm(), for hosts that may not allocate device memory while running:
+    the caller brings X and `out` (fp32 or bf16 [T][n]); split-K partial sums use the 8 MiB array
+    built into the library.  Raises StbError(STB_ERR_SIZE) for shapes that need more."""
+    import torch
+    assert X.dtype == torch.bfloat16 and X.is_cuda and X.dim() == 2 and X.stride(1) == 1
+    assert out.is_cuda and out.dim() == 2 and out.stride(1) == 1 and out.shape == (X.shape[0], layer.n)
+    ydt = {torch.float32: STB_F32, torch.bfloat16: STB_BF16}[out.dtype]
+    _check(_lib.stb_gemm_noalloc(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(X), X.shape[0], X.stride(0),
+                                 _ptr(out), ydt, out.stride(0), _ptr(layer.dev_status), _stream(stream)),
+           "stb_gemm_noalloc")
     return out
 
 

@@ -540,3 +540,44 @@ extern "C" int stb_gemm(const void* packed, int n, int m, int N, const void* X, 
     default: return stb::launch_gemm<6>(p, n, m, X, T, ldx, Y, y_bf16, ldy, ws, ws_bytes, dev_status, s);
   }
 }
+
+// ------------------------------------------------------------------------------------------
+// stb_gemm_noalloc: stb_gemm for callers that can hand over no workspace.  The split-K partial
+// sums live in a fixed array inside the library image instead of a caller's buffer.
+namespace stb {
+constexpr size_t kNoAllocScratchBytes = 8u << 20;                       // 8 MiB per device, resident until exit
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocScratchBytes / sizeof(float)];
+}  // namespace stb
+
+extern "C" int stb_gemm_noalloc(const void* packed, int n, int m, int N, const void* X, int T, size_t ldx,
+                                void* Y, stb_dtype ydt, size_t ldy, int* dev_status, void* stream) {
+  if (!packed || !X || !Y) return STB_ERR_ARG;
+  if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0 || T < 1) return STB_ERR_SHAPE;
+  if (N < 1 || N > 8) return STB_ERR_NM;
+  if (N < 4 || N > 6) return STB_ERR_UNSUPPORTED;
+  if (ydt != STB_F32 && ydt != STB_BF16) return STB_ERR_UNSUPPORTED;
+  if (ldx < (size_t)m || ldy < (size_t)n || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u)) return STB_ERR_ARG;
+  size_t need = 0;
+  const int rc = stb_gemm_workspace(n, m, N, T, &need);
+  if (rc != STB_OK) return rc;
+  if (need > stb::kNoAllocScratchBytes) return STB_ERR_SIZE;           // this shape needs the caller-workspace entry point
+  // The array's name is only a host-side handle: ask the runtime for its address on the current
+  // device, once per device, and give the kernels that address.
+  static float* scratch_of_device[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return STB_ERR_CUDA;
+  if (!scratch_of_device[dev]) {
+    float* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), stb::g_noalloc_scratch) != cudaSuccess || !p) return STB_ERR_CUDA;
+    scratch_of_device[dev] = p;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const uint8_t* pk = static_cast<const uint8_t*>(packed);
+  const int y_bf16 = ydt == STB_BF16;
+  float* ws = scratch_of_device[dev];
+  switch (N) {
+    case 4: return stb::launch_gemm<4>(pk, n, m, X, T, ldx, Y, y_bf16, ldy, ws, stb::kNoAllocScratchBytes, dev_status, s);
+    case 5: return stb::launch_gemm<5>(pk, n, m, X, T, ldx, Y, y_bf16, ldy, ws, stb::kNoAllocScratchBytes, dev_status, s);
+    default: return stb::launch_gemm<6>(pk, n, m, X, T, ldx, Y, y_bf16, ldy, ws, stb::kNoAllocScratchBytes, dev_status, s);
+  }
+}
