@@ -291,6 +291,93 @@ def gemv_table(stb, torch, wl, pk):
     return out, ctx
 
 
+def gemm_table(stb, torch, pk):
+    """Prefill GEMM (stb_gemm, tcgen05) on the LLaMA-2-70B linear shapes at 4:8, 2048 bf16 tokens, with a
+    dense bf16 cuBLAS GEMM (torch.matmul) of the same shape beside it.  The two tall / wide FFN layers
+    are built on the device by repeating the rows / column blocks of the 8192 x 8192 logical layer
+    (valid layers of the same format; the kernel's work does not depend on the values)."""
+    T, N = 2048, 4
+    base = si.logical_layer(8192, 8192, N, si.seed_for(4, 0))
+    kv = si.logical_layer(1024, 8192, N, si.seed_for(4, 1))
+    views = {"keep": np.uint8, "sign": np.uint8, "region": np.int16, "sign2": np.int32, "salient": np.int64, "scale": np.int16}
+
+    def up(d):
+        return {k: torch.from_numpy(np.ascontiguousarray(d[k]).view(v)).cuda() for k, v in views.items()}
+
+    def rows_x(t, times):      # 28672 = 3.5 x 8192 rows
+        return {k: (v if k == "salient" else torch.cat([v] * 3 + [v[:4096]], 0).contiguous()) for k, v in t.items()}
+
+    def cols_x(t):             # 28672 = 3.5 x 8192 columns (whole 128-column blocks)
+        out = {}
+        for k, v in t.items():
+            if k == "salient":
+                out[k] = torch.cat([v] * 3 + [v[:32]], 0).contiguous()
+            else:
+                half = v.shape[1] // 2
+                out[k] = torch.cat([v] * 3 + [v[:, :half]], 1).contiguous()
+        return out
+
+    b = up(base)
+    cases = [("q/o 8192x8192", 8192, 8192, b), ("k/v 1024x8192", 1024, 8192, up(kv)),
+             ("gate/up 28672x8192", 28672, 8192, rows_x(b, 3.5)), ("down 8192x28672", 8192, 28672, cols_x(b))]
+    out = []
+    for name, n, m, t in cases:
+        lay = stb.pack(n, m, N, t["keep"], t["sign"], t["region"], t["sign2"], t["salient"], t["scale"])
+        torch.cuda.synchronize()
+        assert int(lay.dev_status.item()) == 0, name
+        x = torch.randn(T, m, device="cuda").to(torch.bfloat16)
+        y = torch.empty(T, n, dtype=torch.bfloat16, device="cuda")
+        need = stb.gemm_workspace(n, m, N, T)
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+        flush = torch.empty(160 << 20, dtype=torch.uint8, device="cuda")
+
+        def timed(fn, reps=8):
+            for _ in range(3):
+                fn()
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+            for e0, e1 in ev:
+                flush.zero_()                      # L2 flush between timed iterations
+                e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            return 1e3 * float(np.median([e0.elapsed_time(e1) for e0, e1 in ev]))
+
+        us = timed(lambda: stb.gemm(lay, x, out=y, ws=ws))
+        assert int(lay.dev_status.item()) == 0
+        W = torch.randn(n, m, device="cuda").to(torch.bfloat16)
+        usd = timed(lambda: torch.matmul(x, W.t(), out=y))
+        fl = 2.0 * n * m * T
+        out.append({"layer": name, "n": n, "m": m, "tokens": T, "N": N, "us": round(us, 1), "dense_TFLOPs": round(fl / us / 1e6, 1),
+                    "frac_of_measured_bf16_burst": round(fl / us / 1e6 / pk["bf16_tflops"], 4),
+                    "frac_of_measured_bf16_sustained": round(fl / us / 1e6 / pk["bf16_tflops_sustained"], 4),
+                    "useful_TFLOPs": round(fl * N / 8 / us / 1e6, 1), "split_k_workspace_MB": round(need / 1e6, 1),
+                    "cublas_bf16_us": round(usd, 1), "cublas_bf16_TFLOPs": round(fl / usd / 1e6, 1)})
+        del lay, W, x, y, ws, flush
+        torch.cuda.empty_cache()
+    return out
+
+
+def pack_timing(stb, torch, wl):
+    """stb_pack (two launches) on the gate layer: logical bytes read + packed bytes written per second."""
+    d = wl.logical[0]
+    n, m, N = d["n"], d["m"], d["N"]
+    views = {"keep": np.uint8, "sign": np.uint8, "region": np.int16, "sign2": np.int32, "salient": np.int64, "scale": np.int16}
+    t = {k: torch.from_numpy(np.ascontiguousarray(d[k]).view(v)).cuda() for k, v in views.items()}
+    buf = torch.empty(stb.pack_size(n, m, N), dtype=torch.uint8, device="cuda")
+    fn = lambda: stb.pack(n, m, N, t["keep"], t["sign"], t["region"], t["sign2"], t["salient"], t["scale"], buf=buf)
+    for _ in range(3):
+        fn()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(10):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * e0.elapsed_time(e1) / 10
+    moved = sum(v.numel() * v.element_size() for v in t.values()) + wl.infos[0]["used_bytes"]
+    return {"layer": "gate 11008x4096 6:8", "us": round(us, 1), "bytes_moved_MB": round(moved / 1e6, 2), "GBps": round(moved / us / 1e3, 1)}
+
+
 def cuda_arm(args):
     import torch
     import torch.distributed as dist
@@ -398,14 +485,19 @@ def cuda_arm(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": None,
-                     "kernel": "stb::gemv_fast_kernel<6>", "peak_source": pk["_source"],
+                     "kernel": "stb::gemv_mma_kernel<6,1>", "peak_source": pk["_source"],
                      "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
-                     "note": "launch_us = timed region / launches (includes the gaps between launches)"},
+                     "note": "launch_us = timed region / launches (includes the gaps between launches); the decode is "
+                             "bound by the integer pipe (2 warp-instructions/clk/SM): about 0.51 of HBM peak at best for 6:8",
+                     "alu_bound": {"int_lane_ops_per_s": 148 * 64 * 1.965e9, "int_instr_per_tile": 350,
+                                   "floor_us_per_layer": 6.6}},
     }
     if world == 1 and not args.no_extras:
         tab, ctx = gemv_table(stb, torch, wl, pk)
         line["gemv_layers"] = tab
         line["dense_context"] = ctx
+        line["gemm_prefill"] = gemm_table(stb, torch, pk)
+        line["pack"] = pack_timing(stb, torch, wl)
         line["paper_context"] = ("paper's own kernel (2:4 1-bit GEMM, RTX 4090): up to 17.85x over ABQ-LLM 2-bit, "
                                  "263.45 TFLOPS = 79.74% of that GPU's sparse tensor-core peak at sequence length 8192")
     if world == 1 and not args.no_cpu:
