@@ -54,11 +54,32 @@ __host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int ksplit, int 
 
 __device__ __forceinline__ int ilog2(int v) { return 31 - __clz(v); }
 
+// Up to kMaxFused layers that read the same activations (q / k / v, gate / up) run as one grid:
+// row tiles [tile_start[i], tile_start[i + 1]) of the grid belong to layer i.
+constexpr int kMaxFused = 4;
+struct GemvLayers {
+  const uint8_t* packed[kMaxFused];
+  void* y[kMaxFused];
+  size_t ldy[kMaxFused];
+  int n[kMaxFused];
+  int y_f16[kMaxFused];
+  int tile_start[kMaxFused + 1];
+  int count;
+};
+
 template <int N, int NB>
 __global__ void __launch_bounds__(256)
-gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* __restrict__ x, int batch,
-                size_t ldx, void* __restrict__ y, int y_f16, size_t ldy, int* dev_status, int lg_ksplit, int bpp) {
+gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* __restrict__ x, int batch,
+                size_t ldx, int* dev_status, int lg_ksplit, int bpp) {
   extern __shared__ __align__(128) uint8_t smem[];
+  int li = 0, rt_all = (int)(blockIdx.x >> lg_ksplit);
+#pragma unroll
+  for (int i = 1; i < kMaxFused; ++i)
+    if (i < layers.count && rt_all >= layers.tile_start[i]) li = i;
+  const uint8_t* __restrict__ packed = layers.packed[li];
+  void* __restrict__ y = layers.y[li];
+  const size_t ldy = layers.ldy[li];
+  const int n = layers.n[li], y_f16 = layers.y_f16[li];
   const Header* hdr = reinterpret_cast<const Header*>(packed);
   // every CTA of a cluster takes the same branch here (the header is the same for all)
   if (!header_matches(hdr, n, m, N)) {
@@ -69,7 +90,7 @@ gemv_mma_kernel(const uint8_t* __restrict__ packed, int n, int m, const __half* 
   const int ksplit = 1 << lg_ksplit;
   const int warps = (int)(blockDim.x >> 5);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
-  const int kpart = (int)(blockIdx.x & (unsigned)(ksplit - 1)), rt = (int)(blockIdx.x >> lg_ksplit);
+  const int kpart = (int)(blockIdx.x & (unsigned)(ksplit - 1)), rt = rt_all - layers.tile_start[li];
   const int b0 = kpart * bpp, b1 = min(nblk, b0 + bpp);
   const int nbp = max(b1 - b0, 0);
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
@@ -306,11 +327,11 @@ static void gemv_shape(int n, int m, int& ksplit, int& warps) {
 // `chained`: launch as a programmatic dependent of the previous kernel of the stream (only used
 // between the GEMVs of one stb_layer_stack call, whose packed layers nobody writes meanwhile).
 template <int N, int NB>
-static cudaError_t launch_mma(const uint8_t* packed, int n, int m, const __half* x, int batch, size_t ldx,
-                              void* y, int y_f16, size_t ldy, int* dev_status, cudaStream_t s, bool chained) {
-  const int ntile = (n + kTileRows - 1) / kTileRows, nblk = m / kBlock;
+static cudaError_t launch_mma(const GemvLayers& layers, int m, const __half* x, int batch, size_t ldx,
+                              int* dev_status, cudaStream_t s, bool chained) {
+  const int ntile = layers.tile_start[layers.count], nblk = m / kBlock;
   int ksplit, warps;
-  gemv_shape(n, m, ksplit, warps);
+  gemv_shape(ntile * kTileRows, m, ksplit, warps);
   const int bpp = (nblk + ksplit - 1) / ksplit;
   const GemvSmem L = gemv_smem(N, warps, ksplit, NB);
   static bool attr_done = false;
@@ -326,14 +347,29 @@ static cudaError_t launch_mma(const uint8_t* packed, int n, int m, const __half*
   cfg.dynamicSmemBytes = L.total;
   cfg.stream = s;
   cudaLaunchAttribute at[2];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = (unsigned)ksplit; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = chained ? 2 : 1;
+  int na = 0;
+  if (ksplit > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = (unsigned)ksplit; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  if (chained) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at; cfg.numAttrs = na;
   int lg = 0;
   while ((1 << lg) < ksplit) ++lg;
-  return cudaLaunchKernelEx(&cfg, gemv_mma_kernel<N, NB>, packed, n, m, x, batch, ldx, y, y_f16, ldy, dev_status, lg, bpp);
+  return cudaLaunchKernelEx(&cfg, gemv_mma_kernel<N, NB>, layers, m, x, batch, ldx, dev_status, lg, bpp);
+}
+
+template <int NB>
+static cudaError_t launch_mma_n(int N, const GemvLayers& layers, int m, const __half* x, int batch, size_t ldx,
+                                int* dev_status, cudaStream_t s, bool chained) {
+  if (N == 4) return launch_mma<4, NB>(layers, m, x, batch, ldx, dev_status, s, chained);
+  if (N == 5) return launch_mma<5, NB>(layers, m, x, batch, ldx, dev_status, s, chained);
+  return launch_mma<6, NB>(layers, m, x, batch, ldx, dev_status, s, chained);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -476,15 +512,11 @@ static int gemv_impl(const void* packed, int n, int m, int N, const void* x, int
   cudaError_t e = cudaSuccess;
   static const bool force_general = stb::env_int("STB_GEMV_GENERAL") != 0;
   if (N >= 4 && N <= 6 && !force_general) {
-    if (batch <= 8) {
-      if (N == 4) e = stb::launch_mma<4, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
-      else if (N == 5) e = stb::launch_mma<5, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
-      else e = stb::launch_mma<6, 1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
-    } else {
-      if (N == 4) e = stb::launch_mma<4, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
-      else if (N == 5) e = stb::launch_mma<5, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
-      else e = stb::launch_mma<6, 2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s, chained);
-    }
+    stb::GemvLayers layers = {};
+    layers.packed[0] = p; layers.y[0] = y; layers.ldy[0] = ldy; layers.n[0] = n; layers.y_f16[0] = y_f16;
+    layers.tile_start[0] = 0; layers.tile_start[1] = (n + stb::kTileRows - 1) / stb::kTileRows; layers.count = 1;
+    e = batch <= 8 ? stb::launch_mma_n<1>(N, layers, m, xh, batch, ldx, dev_status, s, chained)
+                   : stb::launch_mma_n<2>(N, layers, m, xh, batch, ldx, dev_status, s, chained);
     return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
   }
   switch (N) {
@@ -505,15 +537,54 @@ extern "C" int stb_gemv(const void* packed, int n, int m, int N, const void* x, 
   return gemv_impl(packed, n, m, N, x, batch, ldx, y, ydt, ldy, dev_status, stream, false);
 }
 
+// Steps i..j-1 can share one grid when they read the same activations with the same batch, m and N
+// (4, 5 or 6) and none of them writes what another reads: same-input projections of a decoder
+// layer (q / k / v, gate / up).
+static bool can_fuse(const stb_step& a, const stb_step& b) {
+  return a.in == b.in && a.ldin == b.ldin && a.batch == b.batch && a.m == b.m && a.N == b.N && a.N >= 4 && a.N <= 6 &&
+         b.out != a.in && b.packed && b.out && b.n >= 1 && (b.odt == STB_F32 || b.odt == STB_F16) && b.ldout >= (size_t)b.n;
+}
+
 extern "C" int stb_layer_stack(const stb_step* steps, int count, int* dev_status, void* stream) {
   if (!steps || count < 0) return STB_ERR_ARG;
   static const bool no_pdl = stb::env_int("STB_NO_PDL") != 0;
-  for (int i = 0; i < count; ++i) {
+  static const bool no_fuse = stb::env_int("STB_NO_FUSE") != 0 || stb::env_int("STB_GEMV_GENERAL") != 0;
+  int i = 0;
+  while (i < count) {
     const stb_step& st = steps[i];
+    int j = i + 1;
+    if (!no_fuse)
+      while (j < count && j - i < stb::kMaxFused && can_fuse(st, steps[j])) ++j;
     // steps after the first start their weight stream while the previous step drains
-    int rc = gemv_impl(st.packed, st.n, st.m, st.N, st.in, st.batch, st.ldin, st.out, st.odt, st.ldout,
-                       dev_status, stream, i > 0 && !no_pdl);
-    if (rc != STB_OK) return rc;
+    const bool chained = i > 0 && !no_pdl;
+    if (j - i == 1) {
+      int rc = gemv_impl(st.packed, st.n, st.m, st.N, st.in, st.batch, st.ldin, st.out, st.odt, st.ldout,
+                         dev_status, stream, chained);
+      if (rc != STB_OK) return rc;
+    } else {
+      // validate the first step like stb_gemv does; can_fuse has checked what differs in the others
+      if (!st.packed || !st.in || !st.out) return STB_ERR_ARG;
+      if (st.n < 1 || st.m < stb::kBlock || st.m % stb::kBlock != 0) return STB_ERR_SHAPE;
+      if (st.batch < 1 || st.batch > 16) return STB_ERR_SIZE;
+      if (st.odt != STB_F32 && st.odt != STB_F16) return STB_ERR_UNSUPPORTED;
+      if (st.ldin < (size_t)st.m || st.ldout < (size_t)st.n || (st.ldin % 8) != 0 || (reinterpret_cast<uintptr_t>(st.in) & 15u))
+        return STB_ERR_ARG;
+      stb::GemvLayers layers = {};
+      layers.count = j - i;
+      layers.tile_start[0] = 0;
+      for (int k = i; k < j; ++k) {
+        const stb_step& sk = steps[k];
+        layers.packed[k - i] = static_cast<const uint8_t*>(sk.packed);
+        layers.y[k - i] = sk.out; layers.ldy[k - i] = sk.ldout; layers.n[k - i] = sk.n; layers.y_f16[k - i] = sk.odt == STB_F16;
+        layers.tile_start[k - i + 1] = layers.tile_start[k - i] + (sk.n + stb::kTileRows - 1) / stb::kTileRows;
+      }
+      cudaStream_t s = static_cast<cudaStream_t>(stream);
+      const __half* xh = static_cast<const __half*>(st.in);
+      cudaError_t e = st.batch <= 8 ? stb::launch_mma_n<1>(st.N, layers, st.m, xh, st.batch, st.ldin, dev_status, s, chained)
+                                    : stb::launch_mma_n<2>(st.N, layers, st.m, xh, st.batch, st.ldin, dev_status, s, chained);
+      if (e != cudaSuccess) return STB_ERR_CUDA;
+    }
+    i = j;
   }
   return STB_OK;
 }

@@ -190,6 +190,33 @@ def test_layer_stack_chains_layers_with_per_layer_N(stb):
         assert np.abs(got - y_ref).max() <= tol
 
 
+@pytest.mark.parametrize("batch", [1, 5, 16])
+def test_layer_stack_runs_same_input_layers_as_one_grid(stb, batch):
+    """An MLP-shaped stack: gate and up read the same input (one fused launch, different row counts and
+    output types), down reads gate's fp16 output; every layer is checked against the oracle fed the
+    same input."""
+    import torch
+    m, n1, n2, N = 384, 200, 136, 6
+    dg, du, dd = si.logical_layer(n1, m, N, 71), si.logical_layer(n2, m, N, 72), si.logical_layer(96, 256, N, 73)
+    lg, lu, ld = (stb.pack_numpy(d) for d in (dg, du, dd))
+    x = torch.from_numpy(si.activations(batch, m, 74)).cuda()
+    hg = torch.zeros(batch, 256, dtype=torch.float16, device="cuda")        # wider than n1: ldout > n
+    hu = torch.zeros(batch, n2, dtype=torch.float32, device="cuda")
+    y = torch.zeros(batch, 96, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stb.layer_stack([(lg, x, hg), (lu, x, hu), (ld, hg, y)], dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    xin = x.double().cpu().numpy()
+    for d, out, n, extra in ((dg, hg, n1, 2.0 ** -11), (du, hu, n2, 0.0)):
+        ref = oracle.matmul(oracle.decode(oracle.Logical(**d)), xin)
+        got = out.double().cpu().numpy()[:, :n]
+        assert np.abs(got - ref).max() <= (TOL + extra) * np.abs(ref).max()
+    assert (hg.cpu().numpy()[:, n1:] == 0).all()                             # columns past n untouched
+    ref = oracle.matmul(oracle.decode(oracle.Logical(**dd)), hg.double().cpu().numpy())
+    assert np.abs(y.double().cpu().numpy() - ref).max() <= TOL * np.abs(ref).max()
+
+
 def _check_gemm(stb, layer, L, T, seed, out_dtype=None, rows=None, toks=None):
     """stb_gemm against the float64 dequantise-then-matmul on bf16 activations."""
     import torch
