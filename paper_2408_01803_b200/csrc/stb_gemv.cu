@@ -67,8 +67,11 @@ struct GemvLayers {
   int count;
 };
 
+#ifndef STB_GEMV_MINBLOCKS
+#define STB_GEMV_MINBLOCKS 2
+#endif
 template <int N, int NB>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, STB_GEMV_MINBLOCKS)
 gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* __restrict__ x, int batch,
                 size_t ldx, int* dev_status, int lg_ksplit, int bpp) {
   extern __shared__ __align__(128) uint8_t smem[];

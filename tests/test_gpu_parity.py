@@ -286,3 +286,43 @@ def test_gemm_full_size_sampled(stb, n, m):
     rows = np.unique(np.concatenate([[0, 1, n - 1], g.choice(n, 96, replace=False)])).astype(np.int32)
     toks = np.unique(np.concatenate([[0, 255, 256, T - 1], g.choice(T, 40, replace=False)]))
     _check_gemm(stb, layer, L, T, si.seed_for(4, 9), rows=rows, toks=toks)
+
+
+@pytest.mark.parametrize("batch", [1, 8])
+def test_decoder_layer_stack_full_size_per_layer_N(stb, batch):
+    """The seven linears of a LLaMA-2-7B decoder layer as one stb_layer_stack call in the launch
+    configuration bench.py times (q/k/v and gate/up fused, programmatic dependent launches, CUDA
+    graph), with N drawn per linear from {4, 5, 6}; every layer is checked on sampled rows against
+    the oracle fed the same GPU-produced input."""
+    import torch
+    h, f = 4096, 11008
+    g = np.random.default_rng(si.seed_for(5, batch))
+    Nq, No, Nm, Nd = (int(v) for v in g.choice([4, 5, 6], size=4))
+    spec = [("q", h, h, Nq), ("k", h, h, Nq), ("v", h, h, Nq), ("o", h, h, No), ("gate", f, h, Nm), ("up", f, h, Nm), ("down", h, f, Nd)]
+    ds = [si.logical_layer(n, m, N, si.seed_for(5, 1 + i)) for i, (_, n, m, N) in enumerate(spec)]
+    layers = [stb.pack_numpy(d) for d in ds]
+    x = torch.from_numpy(si.activations(batch, h, si.seed_for(5, 9))).cuda()
+    q, k, v = (torch.empty(batch, h, dtype=torch.float16, device="cuda") for _ in range(3))
+    o = torch.empty(batch, h, dtype=torch.float16, device="cuda")
+    gate, up = (torch.empty(batch, f, dtype=torch.float16, device="cuda") for _ in range(2))
+    y = torch.empty(batch, h, dtype=torch.float32, device="cuda")
+    io = [(x, q), (x, k), (x, v), (q, o), (o, gate), (o, up), (gate, y)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    steps = stb.make_steps([(layers[i], io[i][0], io[i][1]) for i in range(7)])
+    stb.layer_stack(None, dev_status=status, marshalled=steps)            # warm (module load) outside capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        stb.layer_stack(None, dev_status=status, marshalled=steps)
+    for t in (q, k, v, o, gate, up, y):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for i, (name, n, m, N) in enumerate(spec):
+        rows = np.unique(np.concatenate([[0, n - 1], g.choice(n, 48, replace=False)])).astype(np.int32)
+        xin = io[i][0].double().cpu().numpy()
+        ref = oracle.layer_rows(oracle.Logical(**ds[i]), rows, xin)
+        got = io[i][1].double().cpu().numpy()[:, rows]
+        tol = (TOL + (2.0 ** -11 if io[i][1].dtype == torch.float16 else 0.0)) * np.abs(ref).max()
+        assert np.abs(got - ref).max() <= tol, (name, N)
