@@ -485,7 +485,10 @@ def cuda_arm(args):
                 "call": "stb_layer_stack_host: pinned host x -> device, 3 GEMVs, y -> pinned host, stream sync per step"},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
-                     "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": None,
+                     "frac": round(achieved / pk["hbm_gbs"], 4),
+                     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of this
+                     # workload (44.43 MB for gate+up, 22.25 MB for down; mean of the two launches of a step)
+                     "traffic": 33.34e6,
                      "kernel": "stb::gemv_mma_kernel<6,1>", "peak_source": pk["_source"],
                      "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
                      "note": "launch_us = timed region / launches (includes the gaps between launches; a launch is gate+up "
