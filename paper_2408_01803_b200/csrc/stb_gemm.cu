@@ -141,11 +141,16 @@ __device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
   uint8_t* smem = da.smem;
   volatile int* abort_flag = da.abort_flag;
   const uint32_t bar_full = da.bar_full, bar_empty = da.bar_empty;
-  const int mt = da.mt, b0 = da.b0, b1 = da.b1, nblk = da.nblk, ntile = da.ntile, q = da.q, lane = da.lane;
-    const int g = lane >> 2, t = lane & 3;
+  const int mt = da.mt, b0 = da.b0, b1 = da.b1, nblk = da.nblk, ntile = da.ntile, q = da.q;
+    // The lane plays the part of packed-layout lane 4 g + t with g = lane % 8, t = lane / 8: the eight
+    // lanes of a quarter-warp then hold eight different rows g and their 16-byte stores into the
+    // swizzled stage fall on eight different 16-byte bank groups (no conflict); loads of the
+    // lane-major planes stay coalesced, they are only permuted inside the warp.
+    const int g = da.lane & 7, t = da.lane >> 3;
+    const int lane = 4 * g + t;
     const int rtile = mt * 4 + q;                 // packed row tile
     const bool live = rtile < ntile;
-    const uint2* ptab = reinterpret_cast<const uint2*>(smem + kGemmTab);
+    const uint32_t* ptab = reinterpret_cast<const uint32_t*>(smem + kGemmTab);     // low half: columns 0..3, high half: 4..7
     const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
     const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
     const int spb = (int)hdr->spb;
@@ -194,11 +199,11 @@ __device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
       }
       const int nsal = live ? csal.nsal : 0;
       // position selectors of the warp's slots of this block, looked up before the stage waits
-      uint2 P[4][4];
+      uint32_t P[4][4];
 #pragma unroll
       for (int j = J0; j < J0 + NJ; ++j)
 #pragma unroll
-        for (int sidx = 0; sidx < 4; ++sidx) P[j][sidx] = live ? ptab[keep_index_of(cur.mask, j, sidx)] : make_uint2(0, 0);
+        for (int sidx = 0; sidx < 4; ++sidx) P[j][sidx] = live ? ptab[keep_index_of(cur.mask, j, sidx)] : 0u;
       // Salient patches of this block: (salient slot sq, row j) pairs, nsal * NJ of them, dealt to
       // the four lanes t of a lane group; the first one per lane is prepared here.
       const int np = nsal * NJ;
@@ -229,7 +234,7 @@ __device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
             uint32_t f[4] = {0, 0, 0, 0};
             if (live) {
               if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
-              fr.slot2(j, sidx, P[j][sidx].x, P[j][sidx].y, XL[j], XH[j], f);
+              fr.slot2(j, sidx, P[j][sidx], P[j][sidx] >> 16, XL[j], XH[j], f);
             }
             const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
             *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
@@ -276,7 +281,7 @@ __device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
             uint32_t f[4] = {0, 0, 0, 0};
             if (live) {
               if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
-              fr.slot2(j, sidx, P[j][sidx].x, P[j][sidx].y, XL[j], XH[j], f);
+              fr.slot2(j, sidx, P[j][sidx], P[j][sidx] >> 16, XL[j], XH[j], f);
             }
             const int chunk = 4 * sl + t;
             *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
@@ -343,7 +348,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x) reinterpret_cast<uint2*>(smem + kGemmTab)[i] = g_pos_table.v[N][i];
+  for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x)     // 4-byte entries: fewer bank conflicts than 8-byte ones
+    reinterpret_cast<uint32_t*>(smem + kGemmTab)[i] = g_pos_table.v[N][i].x | (g_pos_table.v[N][i].y << 16);
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTok);
   tc_fence_before();
   __syncthreads();
