@@ -368,6 +368,75 @@ def gemm_table(stb, torch, pk):
     return out
 
 
+def stack_tables(stb, torch, pk):
+    """Whole decoder stacks as single stb_layer_stack calls (the other decode workloads):
+      * one LLaMA-2-13B decoder block at 5:8, batch 1 (q/k/v, o, gate/up, down chained on one stream);
+      * all 224 linears of a 32-layer LLaMA-2-7B stack with N drawn per decoder layer from {4, 5, 6}
+        (seeded), batch 1, 8 and 64.
+    One logical layer is drawn per (shape, N) and packed once per use at its own address (the kernels'
+    work does not depend on the values), so that the 2.5-3.1 GB of a 7B stack are all distinct memory."""
+    out = []
+
+    def build(shapes, Ns):
+        cache, layers = {}, []
+        for (name, n, m), N in zip(shapes, Ns):
+            key = (n, m, N)
+            if key not in cache:
+                cache[key] = stb.pack_numpy(si.logical_layer(n, m, N, si.seed_for(5, len(cache))))
+            base = cache[key]
+            used = base.info()["used_bytes"]
+            layers.append((name, stb.PackedLayer(n, m, N, base.buf[:used].clone(), base.dev_status), base.info()["stream_bytes"]))
+        return layers
+
+    def decoder(h, f):
+        return [("q", h, h), ("k", h, h), ("v", h, h), ("o", h, h), ("gate", f, h), ("up", f, h), ("down", h, f)]
+
+    def run_stack(layers, h, f, batch, nl):
+        x = torch.from_numpy(si.activations(batch, h, si.seed_for(5, 40))).cuda()
+        hb = [torch.empty(batch, h, dtype=torch.float16, device="cuda") for _ in range(5)]     # q k v o + layer output
+        fb = [torch.empty(batch, f, dtype=torch.float16, device="cuda") for _ in range(2)]
+        steps, cur = [], x
+        for l in range(nl):
+            q, k, v, o, gate, up, down = [lay for _, lay, _ in layers[7 * l: 7 * l + 7]]
+            steps += [(q, cur, hb[0]), (k, cur, hb[1]), (v, cur, hb[2]), (o, hb[0], hb[3]), (gate, hb[3], fb[0]),
+                      (up, hb[3], fb[1]), (down, fb[0], hb[4])]
+            cur = hb[4]      # (the data flow of attention / activation functions is not part of this path)
+        arr = stb.make_steps(steps)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        fn = lambda: stb.layer_stack(None, dev_status=status, marshalled=arr)
+        g = capture(torch, [fn])
+        us = time_graph(torch, g, 1, min_calls=20 if nl > 1 else 200)
+        assert int(status.item()) == 0
+        return us
+
+    # 13B block, 5:8, batch 1
+    l13 = build(decoder(5120, 13824), [5] * 7)
+    b13 = sum(b for _, _, b in l13)
+    us = run_stack(l13, 5120, 13824, 1, 1)
+    out.append({"stack": "LLaMA-2-13B decoder block, 7 linears, 5:8, batch 1", "us": round(us, 1), "packed_MB": round(b13 / 1e6, 1),
+                "GBps": round(b13 / us / 1e3, 1), "frac_of_measured_hbm": round(b13 / us / 1e3 / pk["hbm_gbs"], 4)})
+    del l13
+    torch.cuda.empty_cache()
+    # 32-layer 7B stack, N per decoder layer
+    rng = np.random.default_rng(si.seed_for(5, 0))
+    Nl = [int(v) for v in rng.choice([4, 5, 6], size=32)]
+    shapes, Ns = [], []
+    for l in range(32):
+        shapes += decoder(4096, 11008)
+        Ns += [Nl[l]] * 7
+    l7 = build(shapes, Ns)
+    b7 = sum(b for _, _, b in l7)
+    for batch in (1, 8, 64):
+        us = run_stack(l7, 4096, 11008, batch, 32)
+        out.append({"stack": "LLaMA-2-7B, 32 decoder layers x 7 linears, N per layer from {4,5,6} (%d/%d/%d layers)" % (
+                        Nl.count(4), Nl.count(5), Nl.count(6)), "batch": batch, "us": round(us, 1),
+                    "packed_GB": round(b7 / 1e9, 3), "GBps": round(b7 / us / 1e3, 1),
+                    "frac_of_measured_hbm": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "us_per_linear": round(us / 224, 2)})
+    del l7
+    torch.cuda.empty_cache()
+    return out
+
+
 def pack_timing(stb, torch, wl):
     """stb_pack (two launches) on the gate layer: logical bytes read + packed bytes written per second."""
     d = wl.logical[0]
@@ -515,6 +584,7 @@ def cuda_arm(args):
         line["dense_context"] = ctx
         line["gemm_prefill"] = gemm_table(stb, torch, pk)
         line["pack"] = pack_timing(stb, torch, wl)
+        line["decode_stacks"] = stack_tables(stb, torch, pk)
         line["paper_context"] = ("paper's own kernel (2:4 1-bit GEMM, RTX 4090): up to 17.85x over ABQ-LLM 2-bit, "
                                  "263.45 TFLOPS = 79.74% of that GPU's sparse tensor-core peak at sequence length 8192")
     if world == 1 and not args.no_cpu:

@@ -112,7 +112,7 @@ int stb_packed_info(const void *packed, stb_info *info, void *stream);
 int stb_dequant(const void *packed, int n, int m, int N, void *W, stb_dtype dt, size_t ldw,
                 void *stream);
 
-/* Decode GEMV, batch 1..16:  y[t][i] = sum_j W^[i][j] * x[t][j],  fp32 accumulation.
+/* Decode GEMV, batch 1..64:  y[t][i] = sum_j W^[i][j] * x[t][j],  fp32 accumulation.
  * x: fp16 [batch][ldx] (ldx >= m, ldx a multiple of 8, x 16-byte aligned); y: [batch][ldy]
  * (ldy >= n) in fp32 (ydt = STB_F32) or fp16 (STB_F16: the fp32 sum rounded to nearest even,
  * for chaining layers).  The memory-bound case of the paper's Appendix C.2 (decoding stage,

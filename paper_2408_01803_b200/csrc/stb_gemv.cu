@@ -1,4 +1,4 @@
-// stb_gemv: decode GEMV  y[t][i] = sum_j W^[i][j] x[t][j],  batch 1..16, fp32 accumulation.
+// stb_gemv: decode GEMV  y[t][i] = sum_j W^[i][j] x[t][j],  batch 1..64, fp32 accumulation.
 // The memory-bound decoding stage of Appendix C.2: every packed byte is read once.
 #include <cooperative_groups.h>
 #include <cuda_fp16.h>
@@ -16,7 +16,7 @@ namespace cg = cooperative_groups;
 namespace stb {
 
 // ------------------------------------------------------------------------------------------
-// Tensor-core GEMV, N = 4, 5, 6, batch <= 8 NB.
+// Tensor-core GEMV, N = 4, 5, 6, batch <= 8 NB (NB = 1, 2, 4, 8).
 //
 // Grid: one thread-block cluster of `ksplit` CTAs per row tile (32 rows); CTA k of the cluster
 // takes the k-th slice of the 128-column blocks and its warps take contiguous runs of that
@@ -47,7 +47,9 @@ __host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int ksplit, int 
   s.bars = kPosTableEntries * 8;                     // the position table comes first
   s.ring = (s.bars + (uint32_t)(warps * kDepth * 8) + 127u) & ~127u;
   s.tile_stride = (kChunk * tile_bytes(N) + 127u) & ~127u;      // one ring slot = one chunk of tiles
-  s.part = s.ring + (uint32_t)(warps * kDepth) * s.tile_stride;
+  // the ring is reused for the per-warp partial sums (warps x 32 rows x 8 NB floats) after the main loop
+  const uint32_t ring_bytes = (uint32_t)(warps * kDepth) * s.tile_stride, red_bytes = (uint32_t)warps * 32u * 8u * (uint32_t)NB * 4u;
+  s.part = s.ring + (ring_bytes > red_bytes ? ring_bytes : red_bytes);
   s.total = s.part + (uint32_t)ksplit * 32u * 8u * (uint32_t)NB * 4u;
   return s;
 }
@@ -71,7 +73,7 @@ struct GemvLayers {
 #define STB_GEMV_MINBLOCKS 2
 #endif
 template <int N, int NB>
-__global__ void __launch_bounds__(256, STB_GEMV_MINBLOCKS)
+__global__ void __launch_bounds__(256, NB <= 2 ? STB_GEMV_MINBLOCKS : 1)
 gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* __restrict__ x, int batch,
                 size_t ldx, int* dev_status, int lg_ksplit, int bpp) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -191,20 +193,30 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
 #pragma unroll
       for (int j = 0; j < 4; ++j) fr.high(j, 0, XL[j], XH[j]);
     }
-    // all table lookups and activation loads of the tile are issued up front
+    // all table lookups (and, for up to 16 batch rows, activation loads) of the tile are issued up front
     uint2 P[16];
 #pragma unroll
     for (int u = 0; u < 16; ++u) P[u] = ptab[keep_index_of(lt.mask, u >> 2, u & 3)];
-    uint4 xf[4][NB];
+    constexpr int XS = NB <= 2 ? 4 : 1;          // activation fragments held at a time: all four steps, or one
+    uint4 xf[XS][NB];
+    if (NB <= 2) {
 #pragma unroll
-    for (int s = 0; s < 4; ++s)
+      for (int s = 0; s < 4; ++s)
 #pragma unroll
-      for (int c = 0; c < NB; ++c) {
-        xf[s][c] = make_uint4(0, 0, 0, 0);
-        if (xrow[c]) xf[s][c] = ldg_nc_v4(xrow[c] + (size_t)b * kBlock + s * 32);
-      }
+        for (int c = 0; c < NB; ++c) {
+          xf[s % XS][c] = make_uint4(0, 0, 0, 0);
+          if (xrow[c]) xf[s % XS][c] = ldg_nc_v4(xrow[c] + (size_t)b * kBlock + s * 32);
+        }
+    }
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
+      if (NB > 2) {
+#pragma unroll
+        for (int c = 0; c < NB; ++c) {
+          xf[0][c] = make_uint4(0, 0, 0, 0);
+          if (xrow[c]) xf[0][c] = ldg_nc_v4(xrow[c] + (size_t)b * kBlock + s * 32);
+        }
+      }
       uint32_t f[4][4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -215,8 +227,9 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
       for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
         for (int c = 0; c < NB; ++c) {
-          mma16816(acc[mt][c], f[2 * mt][0], f[2 * mt + 1][0], f[2 * mt][1], f[2 * mt + 1][1], xf[s][c].x, xf[s][c].y);
-          mma16816(acc[mt][c], f[2 * mt][2], f[2 * mt + 1][2], f[2 * mt][3], f[2 * mt + 1][3], xf[s][c].z, xf[s][c].w);
+          const uint4 xv = xf[s % XS][c];
+          mma16816(acc[mt][c], f[2 * mt][0], f[2 * mt + 1][0], f[2 * mt][1], f[2 * mt + 1][1], xv.x, xv.y);
+          mma16816(acc[mt][c], f[2 * mt][2], f[2 * mt + 1][2], f[2 * mt][3], f[2 * mt + 1][3], xv.z, xv.w);
         }
     }
 
@@ -375,6 +388,15 @@ static cudaError_t launch_mma_n(int N, const GemvLayers& layers, int m, const __
   return launch_mma<6, NB>(layers, m, x, batch, ldx, dev_status, s, chained);
 }
 
+// batch -> number of 8-row batch groups (1, 2, 4 or 8)
+static cudaError_t launch_mma_b(int batch, int N, const GemvLayers& layers, int m, const __half* x, size_t ldx,
+                                int* dev_status, cudaStream_t s, bool chained) {
+  if (batch <= 8) return launch_mma_n<1>(N, layers, m, x, batch, ldx, dev_status, s, chained);
+  if (batch <= 16) return launch_mma_n<2>(N, layers, m, x, batch, ldx, dev_status, s, chained);
+  if (batch <= 32) return launch_mma_n<4>(N, layers, m, x, batch, ldx, dev_status, s, chained);
+  return launch_mma_n<8>(N, layers, m, x, batch, ldx, dev_status, s, chained);
+}
+
 // ------------------------------------------------------------------------------------------
 // General kernel: any N in 1..8, batch <= BT.  One CTA per row tile (32 rows), 8 warps split
 // the blocks, lane = (g, t); plain position-order decode and fp32 multiply-adds, x read
@@ -505,7 +527,7 @@ static int gemv_impl(const void* packed, int n, int m, int N, const void* x, int
   if (!packed || !x || !y) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
-  if (batch < 1 || batch > 16) return STB_ERR_SIZE;
+  if (batch < 1 || batch > 64) return STB_ERR_SIZE;
   if (ydt != STB_F32 && ydt != STB_F16) return STB_ERR_UNSUPPORTED;
   const int y_f16 = ydt == STB_F16;
   if (ldx < (size_t)m || ldy < (size_t)n || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(x) & 15u)) return STB_ERR_ARG;
@@ -518,19 +540,25 @@ static int gemv_impl(const void* packed, int n, int m, int N, const void* x, int
     stb::GemvLayers layers = {};
     layers.packed[0] = p; layers.y[0] = y; layers.ldy[0] = ldy; layers.n[0] = n; layers.y_f16[0] = y_f16;
     layers.tile_start[0] = 0; layers.tile_start[1] = (n + stb::kTileRows - 1) / stb::kTileRows; layers.count = 1;
-    e = batch <= 8 ? stb::launch_mma_n<1>(N, layers, m, xh, batch, ldx, dev_status, s, chained)
-                   : stb::launch_mma_n<2>(N, layers, m, xh, batch, ldx, dev_status, s, chained);
+    e = stb::launch_mma_b(batch, N, layers, m, xh, ldx, dev_status, s, chained);
     return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
   }
-  switch (N) {
-    case 1: e = stb::launch_general<1>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
-    case 2: e = stb::launch_general<2>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
-    case 3: e = stb::launch_general<3>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
-    case 4: e = stb::launch_general<4>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
-    case 5: e = stb::launch_general<5>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
-    case 6: e = stb::launch_general<6>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
-    case 7: e = stb::launch_general<7>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
-    case 8: e = stb::launch_general<8>(p, n, m, xh, batch, ldx, y, y_f16, ldy, dev_status, s); break;
+  // the general kernel takes up to 16 batch rows per launch
+  for (int t0 = 0; t0 < batch && e == cudaSuccess; t0 += 16) {
+    const int bt = batch - t0 < 16 ? batch - t0 : 16;
+    const __half* xc = xh + (size_t)t0 * ldx;
+    void* yc = y_f16 ? static_cast<void*>(static_cast<__half*>(y) + (size_t)t0 * ldy)
+                     : static_cast<void*>(static_cast<float*>(y) + (size_t)t0 * ldy);
+    switch (N) {
+      case 1: e = stb::launch_general<1>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+      case 2: e = stb::launch_general<2>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+      case 3: e = stb::launch_general<3>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+      case 4: e = stb::launch_general<4>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+      case 5: e = stb::launch_general<5>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+      case 6: e = stb::launch_general<6>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+      case 7: e = stb::launch_general<7>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+      case 8: e = stb::launch_general<8>(p, n, m, xc, bt, ldx, yc, y_f16, ldy, dev_status, s); break;
+    }
   }
   return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
 }
@@ -568,7 +596,7 @@ extern "C" int stb_layer_stack(const stb_step* steps, int count, int* dev_status
       // validate the first step like stb_gemv does; can_fuse has checked what differs in the others
       if (!st.packed || !st.in || !st.out) return STB_ERR_ARG;
       if (st.n < 1 || st.m < stb::kBlock || st.m % stb::kBlock != 0) return STB_ERR_SHAPE;
-      if (st.batch < 1 || st.batch > 16) return STB_ERR_SIZE;
+      if (st.batch < 1 || st.batch > 64) return STB_ERR_SIZE;
       if (st.odt != STB_F32 && st.odt != STB_F16) return STB_ERR_UNSUPPORTED;
       if (st.ldin < (size_t)st.m || st.ldout < (size_t)st.n || (st.ldin % 8) != 0 || (reinterpret_cast<uintptr_t>(st.in) & 15u))
         return STB_ERR_ARG;
@@ -583,8 +611,7 @@ extern "C" int stb_layer_stack(const stb_step* steps, int count, int* dev_status
       }
       cudaStream_t s = static_cast<cudaStream_t>(stream);
       const __half* xh = static_cast<const __half*>(st.in);
-      cudaError_t e = st.batch <= 8 ? stb::launch_mma_n<1>(st.N, layers, st.m, xh, st.batch, st.ldin, dev_status, s, chained)
-                                    : stb::launch_mma_n<2>(st.N, layers, st.m, xh, st.batch, st.ldin, dev_status, s, chained);
+      cudaError_t e = stb::launch_mma_b(st.batch, st.N, layers, st.m, xh, st.ldin, dev_status, s, chained);
       if (e != cudaSuccess) return STB_ERR_CUDA;
     }
     i = j;

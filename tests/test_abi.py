@@ -59,7 +59,7 @@ def test_host_side_argument_checks_launch_nothing(stb):
     assert lib.stb_pack(C.byref(L), one, 1 << 20, null, null) == stb.STB_ERR_ARG      # misaligned
     assert lib.stb_gemv(null, 32, 128, 4, one, 1, 128, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_ARG
     assert lib.stb_gemv(one, 32, 128, 4, one, 0, 128, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_SIZE
-    assert lib.stb_gemv(one, 32, 128, 4, one, 17, 128, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_SIZE
+    assert lib.stb_gemv(one, 32, 128, 4, one, 65, 128, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_SIZE
     assert lib.stb_gemv(one, 32, 128, 4, one, 1, 64, one, stb.STB_F32, 32, null, null) == stb.STB_ERR_ARG
     assert lib.stb_gemv(one, 32, 128, 4, one, 1, 128, one, stb.STB_BF16, 32, null, null) == stb.STB_ERR_UNSUPPORTED
     assert lib.stb_dequant(one, 32, 128, 4, one, 7, 128, null) == stb.STB_ERR_UNSUPPORTED

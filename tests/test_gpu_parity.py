@@ -67,7 +67,7 @@ def test_quantized_layer_dequant_bit_exact_and_gemv(stb, N, n, m):
         g16 = stb.dequant(layer, dtype=dt).float().cpu().numpy()
         want = torch.from_numpy(What).to(dt).float().numpy()
         assert np.array_equal(g16, want)
-    for batch in (1, 3, 4, 7, 16):
+    for batch in (1, 3, 4, 7, 16, 17, 33, 64):
         _check_gemv(stb, layer, What, m, batch, 7 + batch)
     _check_gemv(stb, layer, What, m, 2, 99, out_dtype=torch.float16)
 
@@ -90,7 +90,7 @@ def test_full_size_layers_sampled_rows(stb, N, n, m):
     rows = np.sort(g.choice(n, size=192, replace=False)).astype(np.int32)
     rows[:4] = [0, 1, n - 2, n - 1]
     rows = np.unique(rows)
-    for batch in (1, 4, 16):
+    for batch in (1, 4, 16, 64):
         x = si.activations(batch, m, si.seed_for(2, 8 + batch))
         y_ref = oracle.layer_rows(L, rows, x.astype(np.float64))
         y = stb.gemv(layer, torch.from_numpy(x).cuda())
