@@ -6,7 +6,7 @@
 //   build_lane_words            logical fields of the lane's 16 slots -> packed words (pack)
 //   plain_slot                  position-order decode of one slot, bit by bit (dequant, general
 //                               GEMV): the plain definition, any N
-//   FastRows / fast_slot        N = 4, 5, 6: byte-permute decode of one slot into 8 half
+//   FastRows                    N = 4, 5, 6: byte-permute decode of one slot into 8 half
 //                               precision weights (4 registers), the form the tensor-core paths
 //                               consume.  Works on whatever 16-bit scale bytes it is given
 //                               (fp16 for the GEMV, bf16 for the GEMM).
@@ -64,12 +64,27 @@ STB_HD void load_planes(const uint8_t* tile, uint32_t base, uint32_t* w, int lan
   if (NW & 1) w[NW - 1] = *reinterpret_cast<const uint32_t*>(tile + o + lane * 4);
 }
 
-// `tile` may point to global or to shared memory (16-byte aligned).
+// `tile` may point to global or to shared memory (16-byte aligned).  With pair fields in the
+// mask plane (N = 6) the lane's keep-mask indices are gathered from the quad's fields unless
+// `raw_mask` asks for the lane's 16 bytes as they are.
 template <int N>
-STB_HD void load_lane_tile(const uint8_t* tile, int lane, LaneTile<N>& t) {
+STB_HD void load_lane_tile(const uint8_t* tile, int lane, LaneTile<N>& t, bool raw_mask = false) {
   const int g = lane >> 2;
-  const uint4 mk = *reinterpret_cast<const uint4*>(tile + lane * 16);
-  t.mask[0] = mk.x; t.mask[1] = mk.y; t.mask[2] = mk.z; t.mask[3] = mk.w;
+  if (mask_pairs(N) && !raw_mask) {
+    const int tq = lane & 3;
+    t.mask[0] = t.mask[1] = t.mask[2] = t.mask[3] = 0;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int sidx = 0; sidx < 4; ++sidx) {
+        const uint32_t f = *reinterpret_cast<const uint16_t*>(tile + pair_field_off(g, mt, sidx, tq));
+        t.mask[2 * mt] |= pair_field_index(f, 0) << (8 * sidx);
+        t.mask[2 * mt + 1] |= pair_field_index(f, 1) << (8 * sidx);
+      }
+  } else {
+    const uint4 mk = *reinterpret_cast<const uint4*>(tile + lane * 16);
+    t.mask[0] = mk.x; t.mask[1] = mk.y; t.mask[2] = mk.z; t.mask[3] = mk.w;
+  }
   load_planes<N>(tile, off_region(N), t.R, lane);
   load_planes<LaneTile<N>::kFull>(tile, off_sign(N), t.S, lane);
   t.half = 0;
@@ -228,7 +243,54 @@ struct FastRows {
     f[2] = prmt(pl1, ph1, 0x5140u);
     f[3] = prmt(pl1, ph1, 0x7362u);
   }
+  // N = 6, rank order: slot (j, s) -> r[i] = the 16-bit values of ranks 2 i, 2 i + 1 (low half =
+  // lower rank); XL / XH from high(j, s >> 1).  Nothing is moved to column positions: the sparse
+  // tensor-core instruction does that with the metadata of meta6_nibble.
+  STB_HD void pairs(int j, int s, uint32_t XL, uint32_t XH, uint32_t (&r)[3]) const {
+    const uint32_t sel = ((s & 2) ? o[j] : e[j]) >> (16 * (s & 1));
+    const uint32_t lo0 = prmt(A[j], A[j], sel), hi0 = prmt(Bp[j], Bn[j], sel);
+    r[0] = prmt(lo0, hi0, 0x5140u);
+    r[1] = prmt(lo0, hi0, 0x7362u);
+    r[2] = prmt(XL, XH, (s & 1) ? 0x7362u : 0x5140u);
+  }
 };
+
+// ------------------------------------------------------------------------------------------
+// N = 6 through the 2:4 sparse tensor-core instruction (mma.sp m16n8k32).  With 6 of 8 columns
+// kept, rank 2 i sits in column 2 i .. 2 i + 2 and rank 2 i + 1 in column 2 i + 1 .. 2 i + 3, so
+// the pair (2 i, 2 i + 1) is a 2-of-4 selection from columns 2 i .. 2 i + 3: every group is three
+// "chunks" of the instruction, whose operand holds the pair in rank order and whose activations
+// are x[8 G + 2 i .. 8 G + 2 i + 3].  Metadata nibble of chunk i = idx0 | idx1 << 2 with
+// idx = column - 2 i of the two ranks (idx0 < idx1).
+STB_HD constexpr uint32_t meta6_nibble(uint32_t keep_byte, int i) {
+  uint32_t col[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  int r = 0;
+  for (int c = 0; c < 8; ++c)
+    if ((keep_byte >> c) & 1u) col[r++ & 7] = (uint32_t)c;
+  return ((col[2 * i] - 2u * (uint32_t)i) & 3u) | (((col[2 * i + 1] - 2u * (uint32_t)i) & 3u) << 2);
+}
+// Table keyed by the keep-mask index: byte i = nibble of chunk i.  Entries past the 28 masks hold a valid pattern.
+constexpr int kMeta6Entries = 64;
+struct Meta6Table { uint32_t v[kMeta6Entries]; };
+constexpr Meta6Table make_meta6_table() {
+  Meta6Table t{};
+  for (int e = 0; e < kMeta6Entries; ++e) {
+    t.v[e] = 0;
+    for (int i = 0; i < 3; ++i) t.v[e] |= (e < 28 ? meta6_nibble(kMaskTables.mask[6][e], i) : 0x4u) << (8 * i);
+  }
+  return t;
+}
+// The six metadata words of a lane from the table entries en[rp][tq] (row g + 16 mt + 8 rp, lane tq of the quad)
+// of one of its two slots: word i has the nibble of lane tq at bit 4 tq (row rp = 0) and 16 + 4 tq (rp = 1).
+STB_HD void meta6_words(const uint32_t (&en)[2][4], uint32_t (&E)[3]) {
+  const uint32_t z01a = en[0][0] + (en[0][1] << 4), z23a = en[0][2] + (en[0][3] << 4);
+  const uint32_t z01b = en[1][0] + (en[1][1] << 4), z23b = en[1][2] + (en[1][3] << 4);
+  const uint32_t wa = prmt(z01a, z23a, 0x5140u), wb = prmt(z01b, z23b, 0x5140u);
+  const uint32_t wc = prmt(z01a, z23a, 0x7362u), wd = prmt(z01b, z23b, 0x7362u);
+  E[0] = prmt(wa, wb, 0x5410u);
+  E[1] = prmt(wa, wb, 0x7632u);
+  E[2] = prmt(wc, wd, 0x5410u);
+}
 
 // position selector of a keep byte: nibble c = rank of column c among the kept columns, 7 for a
 // dropped column (byte 7 of the rank-ordered bytes is zero for N <= 7)

@@ -15,6 +15,8 @@ namespace cg = cooperative_groups;
 
 namespace stb {
 
+__device__ const Meta6Table g_meta6 = make_meta6_table();
+
 // ------------------------------------------------------------------------------------------
 // Tensor-core GEMV, N = 4, 5, 6, batch <= 8 NB (NB = 1, 2, 4, 8).
 //
@@ -129,13 +131,18 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
       bulk_g2s(smem_u32(ring + (size_t)i * L.tile_stride), rtbase + (size_t)(wb0 + i * kChunk) * tbytes, bytes, bar0 + 8u * i);
     }
   }
-  for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x) reinterpret_cast<uint2*>(smem)[i] = g_pos_table.v[N][i];
+  if (N == 6 && NB == 1) {   // metadata by keep-mask index (256 bytes: an index byte of the tile cannot point past it)
+    for (int i = threadIdx.x; i < kMeta6Entries; i += blockDim.x) reinterpret_cast<uint32_t*>(smem)[i] = g_meta6.v[i];
+  } else {
+    for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x) reinterpret_cast<uint2*>(smem)[i] = g_pos_table.v[N][i];
+  }
 
   // Everything below reads the activations (the previous layer's output) or writes y: wait for the
   // previous grid of the stream to have completed (no-op without a programmatic launch), then let
   // the next grid start its own weight stream.
   grid_dependency_wait();
   grid_launch_dependents();
+  x = after_dependency_wait(x);
   __syncthreads();
 
   float acc[2][NB][4];
@@ -159,6 +166,10 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   const __half* xrow[NB];
 #pragma unroll
   for (int c = 0; c < NB; ++c) xrow[c] = g + 8 * c < batch ? x + (size_t)(g + 8 * c) * ldx + t * 8 : nullptr;
+  // N = 6: the lane's activation pairs of a chunk start at column 8 (t >> 1) + 2 (t & 1) of a 32-column step
+  const __half* xsp[NB];
+#pragma unroll
+  for (int c = 0; c < NB; ++c) xsp[c] = xrow[c] ? xrow[c] - t * 8 + 8 * (t >> 1) + 2 * (t & 1) : nullptr;
 
   for (int it = 0; it < cnt; ++it) {
     const int ch = it / kChunk, kin = it - ch * kChunk;     // chunk and tile inside the chunk
@@ -175,20 +186,98 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
     // all lanes poll; the verdict is made warp-uniform so that nobody is left at a __syncwarp
     if (kin == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(ch / kDepth) & 1u, kWaitLimit))) { failed = true; break; }
     const uint8_t* tile = ring + (size_t)slot * L.tile_stride + (size_t)kin * tbytes;
+    // release of the ring slot: once the whole chunk is in registers or consumed, refill it
+    auto refill = [&]() {
+      if (kin == kChunk - 1 || it == cnt - 1) {
+        __syncwarp();
+        const int nxt = (ch + kDepth) * kChunk;      // first tile of the chunk that reuses this slot
+        if (lane == 0 && nxt < cnt) {
+          const uint32_t bytes = (uint32_t)min(kChunk, cnt - nxt) * tbytes;
+          fence_async_smem();
+          mbar_expect_tx(bar, bytes);
+          bulk_g2s(smem_u32(ring + (size_t)slot * L.tile_stride), rtbase + (size_t)(wb0 + nxt) * tbytes, bytes, bar);
+        }
+      }
+    };
+    if constexpr (N == 6 && NB == 1) {
+      // Rank order through the sparse instruction.  This lane's metadata: rows g + 16 (t >> 1) and + 8, the chunks
+      // of operand registers 2 h, 2 h + 1 (h = t & 1) of the quad's four lanes, i.e. their slots 2 h and 2 h + 1.
+      LaneTile<N> lt;
+      load_lane_tile<N>(tile, lane, lt, true);
+      if (mine) { rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1]; }
+      refill();
+      FastRows<N> fr;
+      fr.init(lt, lt.A, lt.B);
+      uint32_t E[2][3];
+#pragma unroll
+      for (int bb = 0; bb < 2; ++bb) {
+        uint32_t en[2][4];
+#pragma unroll
+        for (int tq = 0; tq < 4; ++tq)
+#pragma unroll
+          for (int rp = 0; rp < 2; ++rp) {
+            const uint32_t off = prmt(lt.mask[2 * bb + (tq >> 1)], 0u, 0x4440u + (uint32_t)(2 * (tq & 1) + rp));
+            en[rp][tq] = *reinterpret_cast<const uint32_t*>(smem + off);
+          }
+        meta6_words(en, E[bb]);
+      }
+      uint32_t XL6[4][2], XH6[4][2];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int sp = 0; sp < 2; ++sp) fr.high(j, sp, XL6[j][sp], XH6[j][sp]);
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl) {
+        uint32_t R[4][2][3];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) fr.pairs(j, 2 * h + sl, XL6[j][h], XH6[j][h], R[j][h]);
+        // Activations of chunk i of a step: columns 2 i + 2 (t & 1) + {0, 1} of the group's eight.  Up to two batch
+        // rows: one 4-byte load per register (few lanes are active); more: the group's 16 bytes, then a select.
+        if (batch <= 2) {
+#pragma unroll
+          for (int i = 0; i < 3; ++i) {
+#pragma unroll
+            for (int c = 0; c < NB; ++c) {
+              uint32_t bx[4] = {0, 0, 0, 0};
+              if (xsp[c]) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                  bx[u] = ldg_nc_u32(xsp[c] + (size_t)b * kBlock + 64 * (u >> 1) + 16 * (u & 1) + 32 * sl + 2 * i);
+              }
+              mma_sp16832<0>(acc[0][c], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx[0], bx[1], bx[2], bx[3], E[sl][i]);
+              mma_sp16832<1>(acc[1][c], R[2][0][i], R[3][0][i], R[2][1][i], R[3][1][i], bx[0], bx[1], bx[2], bx[3], E[sl][i]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < NB; ++c) {
+            uint4 xw[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              xw[u] = make_uint4(0, 0, 0, 0);
+              if (xsp[c]) xw[u] = ldg_nc_v4(xsp[c] - 2 * (t & 1) + (size_t)b * kBlock + 64 * (u >> 1) + 16 * (u & 1) + 32 * sl);
+            }
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+              uint32_t bx[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const uint32_t w0 = i == 0 ? xw[u].x : (i == 1 ? xw[u].y : xw[u].z), w1 = i == 0 ? xw[u].y : (i == 1 ? xw[u].z : xw[u].w);
+                bx[u] = (t & 1) ? w1 : w0;
+              }
+              mma_sp16832<0>(acc[0][c], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx[0], bx[1], bx[2], bx[3], E[sl][i]);
+              mma_sp16832<1>(acc[1][c], R[2][0][i], R[3][0][i], R[2][1][i], R[3][1][i], bx[0], bx[1], bx[2], bx[3], E[sl][i]);
+            }
+          }
+        }
+      }
+    } else {
     LaneTile<N> lt;
     load_lane_tile<N>(tile, lane, lt);
     if (mine) { rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1]; }
-    if (kin == kChunk - 1 || it == cnt - 1) {      // the whole chunk is in registers or consumed
-      __syncwarp();
-      const int nxt = (ch + kDepth) * kChunk;      // first tile of the chunk that reuses this slot
-      if (lane == 0 && nxt < cnt) {
-        const uint32_t bytes = (uint32_t)min(kChunk, cnt - nxt) * tbytes;
-        fence_async_smem();
-        mbar_expect_tx(bar, bytes);
-        bulk_g2s(smem_u32(ring + (size_t)slot * L.tile_stride), rtbase + (size_t)(wb0 + nxt) * tbytes, bytes, bar);
-      }
-    }
-
+    refill();
     FastRows<N> fr;
     fr.init(lt, lt.A, lt.B);
     uint32_t XL[4] = {0, 0, 0, 0}, XH[4] = {0, 0, 0, 0};
@@ -234,6 +323,7 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
           mma16816(acc[mt][c], f[2 * mt][0], f[2 * mt + 1][0], f[2 * mt][1], f[2 * mt + 1][1], xv.x, xv.y);
           mma16816(acc[mt][c], f[2 * mt][2], f[2 * mt + 1][2], f[2 * mt][3], f[2 * mt + 1][3], xv.z, xv.w);
         }
+    }
     }
 
     // residual term: once the salient slots of 16 / SPB blocks are collected (or at the end)

@@ -20,6 +20,14 @@
 //                               numeric order): the same 8 bits, but a lookup table keyed by it
 //                               has at most 70 entries, which keeps shared-memory lookups by the
 //                               32 lanes of a warp nearly free of bank conflicts
+//                               N = 6 stores the same bytes in another order (mask_pairs): the
+//                               GEMV multiplies rank-ordered weights with the sparse tensor-core
+//                               instruction, whose selection metadata for rows g + 16 mt and
+//                               g + 16 mt + 8 comes from lanes 2 mt and 2 mt + 1 of the quad.  So
+//                               lane (g, t) holds, at byte 8 b + 2 tq + rp, four times the
+//                               keep-mask index of group 4 (2 (t & 1) + b) + tq of row
+//                               g + 16 (t >> 1) + 8 rp (four times: the byte offset into a table
+//                               of 4-byte entries).
 //   region  N words per lane    two-bit region codes, 16 per word, of the lane's 16 N kept
 //                               weights: first the "low" part (ranks k < min(N, 4) of every
 //                               slot, weight number wl = u NL + k), then the "high" part
@@ -101,6 +109,16 @@ STB_HD constexpr uint32_t tiles_offset(int nblk) {
 }
 STB_HD constexpr int spb_for(int max_nsal) {
   return max_nsal == 0 ? 0 : (max_nsal <= 4 ? 4 : (max_nsal <= 8 ? 8 : (max_nsal <= 16 ? 16 : 32)));
+}
+// N = 6: the mask plane is ordered for the metadata of the sparse instruction (see the layout comment)
+STB_HD constexpr bool mask_pairs(int N) { return N == 6; }
+// byte offset, inside the tile, of the two bytes (row g + 16 mt, then row g + 16 mt + 8) of group 4 s + tq
+STB_HD constexpr uint32_t pair_field_off(int g, int mt, int s, int tq) {
+  return 16u * (uint32_t)(4 * g + 2 * mt + (s >> 1)) + 8u * (uint32_t)(s & 1) + 2u * (uint32_t)tq;
+}
+STB_HD constexpr uint32_t pair_field(uint32_t i0, uint32_t i1) { return (4u * i0) | ((4u * i1) << 8); }
+STB_HD constexpr uint32_t pair_field_index(uint32_t field, int upper_row) {
+  return upper_row ? ((field >> 10) & 63u) : ((field >> 2) & 63u);
 }
 STB_HD constexpr uint32_t off_region(int) { return 512u; }
 STB_HD constexpr uint32_t off_sign(int N) { return 512u + 128u * (uint32_t)N; }

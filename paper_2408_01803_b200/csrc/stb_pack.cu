@@ -207,6 +207,20 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
   }
   LaneWords<N> w;
   build_lane_words<N>(sgn, reg, true, w);
+  if (mask_pairs(N)) {
+    // this lane's 16 bytes cover rows g + 16 mt, g + 16 mt + 8 and slots 2 h, 2 h + 1 of all four lanes
+    const int mt = t >> 1, h = t & 1;
+#pragma unroll
+    for (int wq = 0; wq < 4; ++wq) {
+      maskw[wq] = 0;
+#pragma unroll
+      for (int hw = 0; hw < 2; ++hw) {
+        const int sidx = 2 * h + (wq >> 1), tq = 2 * (wq & 1) + hw, grp = 4 * sidx + tq;
+        const uint32_t i0 = mask_index(N, sm_keep[wib][g + 16 * mt][grp]), i1 = mask_index(N, sm_keep[wib][g + 16 * mt + 8][grp]);
+        maskw[wq] |= pair_field(i0, i1) << (16 * hw);
+      }
+    }
+  }
   *reinterpret_cast<uint4*>(tile + lane * 16) = make_uint4(maskw[0], maskw[1], maskw[2], maskw[3]);
   store_planes<N>(tile, off_region(N), w.R, lane);
   store_planes<LaneTile<N>::kFull>(tile, off_sign(N), w.S, lane);

@@ -4,6 +4,8 @@
 //   * plain_slot returns every kept weight's region code and sign at the right column,
 //   * FastRows::slot (N = 4, 5, 6) returns, for every column, the 16-bit pattern of the signed
 //     scale of the weight's region, or zero for a dropped column,
+//   * for N = 6 the rank-order operand pairs and the metadata table of the sparse tensor-core path
+//     rebuild the same 16-bit patterns, and the pair fields return the keep-mask indices,
 //   * the residual selectors return the stored two-bit codes.
 // Expected values come from the logical fields directly (the definition of the format), not
 // from any packed-side code.
@@ -65,6 +67,16 @@ static int check(int trials, int spb) {
       }
       LaneWords<N> w;
       build_lane_words<N>(sg, rg, true, w);
+      if (mask_pairs(N)) {
+        // pair fields: lane (g, t) holds rows g + 16 (t >> 1), + 8 and slots 2 (t & 1), 2 (t & 1) + 1 of the four lanes
+        for (int wq = 0; wq < 4; ++wq) {
+          maskw[wq] = 0;
+          for (int hw = 0; hw < 2; ++hw) {
+            const int s = 2 * (t & 1) + (wq >> 1), tq = 2 * (wq & 1) + hw, grp = 4 * s + tq, r0 = g + 16 * (t >> 1);
+            maskw[wq] |= pair_field(mask_index(N, keep[r0][grp]), mask_index(N, keep[r0 + 8][grp])) << (16 * hw);
+          }
+        }
+      }
       for (int j = 0; j < 4; ++j) put32(lane * 16 + 4 * j, maskw[j]);
       for (int i = 0; i < N; ++i) put32(region_word_off(N, i, lane), w.R[i]);
       for (int i = 0; i < sign_full_words(N); ++i) put32(sign_word_off(N, i, lane), w.S[i]);
@@ -119,6 +131,67 @@ static int check(int trials, int spb) {
           std::memcpy(&word, &resid[resid_word_off(spb, g, q >> 2)], 4);
           if (resid_code(word, j, q & 3) != rcode[r][q]) { if (++errors < 10) std::printf("resid code N=%d\n", N); }
           if (((resid_selector(word, j) >> (4 * (q & 3))) & 0xFu) != rcode[r][q]) { if (++errors < 10) std::printf("resid selector N=%d\n", N); }
+        }
+      }
+      if constexpr (N == 6) {
+        // rank-order operands and metadata of the sparse tensor-core path: rebuilding the row from them
+        // (value of rank k lands on column 2 i + idx) must give the position-order weights
+        static const Meta6Table meta = make_meta6_table();
+        LaneTile<N> raw;
+        load_lane_tile<N>(tile.data(), lane, raw, true);
+        FastRows<N> fr;
+        fr.init(lt, lt.A, lt.B);
+        for (int j = 0; j < 4; ++j)
+          for (int s = 0; s < 4; ++s) {
+            uint32_t XL, XH, rr[3];
+            fr.high(j, s >> 1, XL, XH);
+            fr.pairs(j, s, XL, XH, rr);
+            const int r = g + 8 * j, grp = 4 * s + t;
+            // the lane that supplies this chunk's metadata: (g, 2 (j >> 1) + (s >> 1)), field halfword 4 (s & 1) + t
+            uint16_t field;
+            std::memcpy(&field, &tile[pair_field_off(g, j >> 1, s, t)], 2);
+            if (pair_field_index(field, j & 1) != mask_index(N, keep[r][grp])) { if (++errors < 10) std::printf("pair field N=%d\n", N); }
+            uint32_t row[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            for (int i = 0; i < 3; ++i) {
+              const uint32_t nib = (meta.v[pair_field_index(field, j & 1)] >> (8 * i)) & 0xFu;
+              if ((nib & 3u) >= (nib >> 2)) { if (++errors < 10) std::printf("metadata order N=%d\n", N); }
+              row[2 * i + (nib & 3u)] = rr[i] & 0xFFFFu;
+              row[2 * i + (nib >> 2)] = rr[i] >> 16;
+            }
+            int k = 0;
+            for (int c = 0; c < 8; ++c) {
+              uint32_t want = 0;
+              if ((keep[r][grp] >> c) & 1) {
+                const uint32_t code = (region[r][grp] >> (2 * k)) & 3u;
+                const uint32_t ng = ((sign[r][grp] >> k) & 1u) ^ 1u;
+                want = scale[r][code] ^ (ng << 15);
+                ++k;
+              }
+              if (row[c] != want) { if (++errors < 10) std::printf("sparse N=%d lane %d j %d s %d c %d: got %04x want %04x\n", N, lane, j, s, c, row[c], want); }
+            }
+          }
+      }
+      if constexpr (N == 6) {
+        // the metadata words this lane hands to the instruction: rows g + 16 (t >> 1) + 8 rp, slots 2 (t & 1) + bb
+        // of the four lanes tq; nibble of lane tq at bit 4 tq + 16 rp of word i
+        static const Meta6Table meta = make_meta6_table();
+        LaneTile<N> raw;
+        load_lane_tile<N>(tile.data(), lane, raw, true);
+        for (int bb = 0; bb < 2; ++bb) {
+          uint32_t en[2][4], E[3];
+          for (int tq = 0; tq < 4; ++tq)
+            for (int rp = 0; rp < 2; ++rp) {
+              const uint32_t off = prmt(raw.mask[2 * bb + (tq >> 1)], 0u, 0x4440u + (uint32_t)(2 * (tq & 1) + rp));
+              if (off % 4 != 0 || off / 4 >= 28) { ++errors; continue; }
+              en[rp][tq] = meta.v[off / 4];
+            }
+          meta6_words(en, E);
+          for (int i = 0; i < 3; ++i)
+            for (int tq = 0; tq < 4; ++tq)
+              for (int rp = 0; rp < 2; ++rp) {
+                const int r = g + 16 * (t >> 1) + 8 * rp, grp = 4 * (2 * (t & 1) + bb) + tq;
+                if (((E[i] >> (4 * tq + 16 * rp)) & 0xFu) != meta6_nibble(keep[r][grp], i)) { if (++errors < 10) std::printf("metadata word N=%d\n", N); }
+              }
         }
       }
       if constexpr (N >= 4 && N <= 6) {
