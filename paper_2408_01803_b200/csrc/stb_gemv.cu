@@ -41,10 +41,19 @@ constexpr int kChunk = STB_GEMV_CHUNK;     // tiles per bulk copy (consecutive b
 constexpr long long kWaitLimit = 2000000000ll;     // about a second of SM clocks
 
 struct GemvSmem {
-  uint32_t bars, ring, part, total;                 // byte offsets
+  uint32_t bars, ring, part, ximg, total;           // byte offsets
   uint32_t tile_stride;
 };
-__host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int ksplit, int NB) {
+// N = 6, up to two batch rows: the CTA's slice of the activations is kept in shared memory in the order the lanes
+// consume it: per block and batch row 96 words, word ((t * 2 + sl) * 3 + i) * 4 + u = operand register u of chunk i
+// of step sl of lane t (two fp16 each).
+constexpr uint32_t kImgWords = 96;
+constexpr uint32_t kImgMaxBytes = 20 * 1024;
+__host__ __device__ inline uint32_t gemv_image_bytes(int N, int NB, int batch, int bpp) {
+  const uint32_t bytes = (uint32_t)batch * (uint32_t)bpp * kImgWords * 4u;
+  return (N == 6 && NB == 1 && batch <= 2 && bytes <= kImgMaxBytes) ? bytes : 0u;
+}
+__host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int ksplit, int NB, uint32_t image_bytes) {
   GemvSmem s;
   s.bars = kPosTableEntries * 8;                     // the position table comes first
   s.ring = (s.bars + (uint32_t)(warps * kDepth * 8) + 127u) & ~127u;
@@ -52,7 +61,8 @@ __host__ __device__ inline GemvSmem gemv_smem(int N, int warps, int ksplit, int 
   // the ring is reused for the per-warp partial sums (warps x 32 rows x 8 NB floats) after the main loop
   const uint32_t ring_bytes = (uint32_t)(warps * kDepth) * s.tile_stride, red_bytes = (uint32_t)warps * 32u * 8u * (uint32_t)NB * 4u;
   s.part = s.ring + (ring_bytes > red_bytes ? ring_bytes : red_bytes);
-  s.total = s.part + (uint32_t)ksplit * 32u * 8u * (uint32_t)NB * 4u;
+  s.ximg = s.part + (uint32_t)ksplit * 32u * 8u * (uint32_t)NB * 4u;
+  s.total = s.ximg + image_bytes;
   return s;
 }
 
@@ -109,7 +119,8 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)hdr->ntile +
                             (size_t)rt * nblk * resid_tile_bytes(spb);
-  const GemvSmem L = gemv_smem(N, warps, ksplit, NB);
+  const uint32_t image_bytes = gemv_image_bytes(N, NB, batch, bpp);
+  const GemvSmem L = gemv_smem(N, warps, ksplit, NB, image_bytes);
 
   const uint2* ptab = reinterpret_cast<const uint2*>(smem);
   uint8_t* ring = smem + L.ring + (size_t)warp * kDepth * L.tile_stride;
@@ -143,6 +154,37 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   grid_dependency_wait();
   grid_launch_dependents();
   x = after_dependency_wait(x);
+  const uint32_t* ximg = reinterpret_cast<const uint32_t*>(smem + L.ximg);
+  const uint32_t img_row_words = (uint32_t)bpp * kImgWords;
+  if (N == 6 && NB == 1 && image_bytes != 0u) {
+    // one item = the 8 activations of one group of one block of one batch row: a 16-byte load, six 4-byte stores
+    // (lanes t = 2 (G & 1) + p read word i + p of group G as chunk i: words 0..2 for p = 0, words 1..3 for p = 1)
+    uint32_t* img = reinterpret_cast<uint32_t*>(smem + L.ximg);
+    const int items = batch * nbp * 16;
+    for (int base = 0; base < items; base += 4 * (int)blockDim.x) {
+      uint4 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int it = base + k * (int)blockDim.x + (int)threadIdx.x;
+        v[k] = make_uint4(0, 0, 0, 0);
+        if (it < items) {
+          const int r = it / (nbp * 16), q = it - r * nbp * 16;
+          v[k] = ldg_nc_v4(x + (size_t)r * ldx + (size_t)b0 * kBlock + (size_t)q * 8);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int it = base + k * (int)blockDim.x + (int)threadIdx.x;
+        if (it < items) {
+          const int r = it / (nbp * 16), q = it - r * nbp * 16, blk = q >> 4, G = q & 15;
+          uint32_t* d = img + (uint32_t)r * img_row_words + (uint32_t)blk * kImgWords +
+                        (uint32_t)((4 * (G & 1) + ((G >> 2) & 1)) * 12 + 2 * (G >> 3) + ((G >> 1) & 1));
+          d[0] = v[k].x; d[4] = v[k].y; d[8] = v[k].z;
+          d[24] = v[k].y; d[28] = v[k].z; d[32] = v[k].w;
+        }
+      }
+    }
+  }
   __syncthreads();
 
   float acc[2][NB][4];
@@ -234,8 +276,18 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
 #pragma unroll
           for (int h = 0; h < 2; ++h) fr.pairs(j, 2 * h + sl, XL6[j][h], XH6[j][h], R[j][h]);
         // Activations of chunk i of a step: columns 2 i + 2 (t & 1) + {0, 1} of the group's eight.  Up to two batch
-        // rows: one 4-byte load per register (few lanes are active); more: the group's 16 bytes, then a select.
-        if (batch <= 2) {
+        // rows: from the CTA's image in shared memory (or, when the slice is too long for it, one 4-byte load per
+        // register: few lanes are active); more: the group's 16 bytes through L1, then a select.
+        if (image_bytes != 0u) {
+          const uint32_t* xi = ximg + (uint32_t)g * img_row_words + (uint32_t)(b - b0) * kImgWords + (uint32_t)((t * 2 + sl) * 12);
+#pragma unroll
+          for (int i = 0; i < 3; ++i) {
+            uint4 bx = make_uint4(0, 0, 0, 0);
+            if (g < batch) bx = *reinterpret_cast<const uint4*>(xi + 4 * i);
+            mma_sp16832<0>(acc[0][0], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
+            mma_sp16832<1>(acc[1][0], R[2][0][i], R[3][0][i], R[2][1][i], R[3][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
+          }
+        } else if (batch <= 2) {
 #pragma unroll
           for (int i = 0; i < 3; ++i) {
 #pragma unroll
@@ -442,7 +494,7 @@ static cudaError_t launch_mma(const GemvLayers& layers, int m, const __half* x, 
   int ksplit, warps;
   gemv_shape(ntile * kTileRows, m, ksplit, warps);
   const int bpp = (nblk + ksplit - 1) / ksplit;
-  const GemvSmem L = gemv_smem(N, warps, ksplit, NB);
+  const GemvSmem L = gemv_smem(N, warps, ksplit, NB, gemv_image_bytes(N, NB, batch, bpp));
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(gemv_mma_kernel<N, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
