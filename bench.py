@@ -568,16 +568,16 @@ def cuda_arm(args):
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": round(achieved / pk["hbm_gbs"], 4),
                      # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of this
-                     # workload (44.42 MB for gate+up, 22.25 MB for down; mean of the two launches of a step)
+                     # workload (44.43 MB for gate+up, 22.25 MB for down; mean of the two launches of a step)
                      "traffic": 33.34e6,
                      "kernel": "stb::gemv_mma_kernel<6,1>", "peak_source": pk["_source"],
                      "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
                      "note": "launch_us = timed region / launches (includes the gaps between launches; a launch is gate+up "
                              "(44.4 MB) or down (22.2 MB), bytes_per_launch is their mean); 6:8 multiplies rank-ordered "
-                             "weights with mma.sp, 264 integer-pipe instructions per 32x128 tile (2 warp-instructions/clk/SM) "
-                             "of 463 in all: the pipe alone allows 0.66 of HBM peak, the kernel issues on 46 % of the cycles",
-                     "alu_bound": {"int_lane_ops_per_s": 148 * 64 * 1.965e9, "int_instr_per_tile": 264,
-                                   "floor_us_per_layer": 5.1}},
+                             "weights with mma.sp, 283 integer-pipe instructions per 32x128 tile (2 warp-instructions/clk/SM) "
+                             "of 497 in all: the pipe alone allows 0.62 of HBM peak, the kernel issues on 45 % of the cycles",
+                     "alu_bound": {"int_lane_ops_per_s": 148 * 64 * 1.965e9, "int_instr_per_tile": 283,
+                                   "floor_us_per_layer": 5.4}},
     }
     if world == 1 and not args.no_extras:
         tab, ctx = gemv_table(stb, torch, wl, pk)

@@ -57,7 +57,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                     print(log)
     if todo or not os.path.exists(LIB):
         tmp = LIB + ".tmp%d" % os.getpid()
-        subprocess.check_call([nvcc(), "-shared", "-o", tmp] + objs + ["-lcuda"])
+        subprocess.check_call([nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs + ["-lcuda"])
         os.replace(tmp, LIB)
     return LIB
 
