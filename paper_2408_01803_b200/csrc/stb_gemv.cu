@@ -263,6 +263,34 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
           }
         meta6_words(en, E[bb]);
       }
+      if (image_bytes != 0u) {
+        // activations from the CTA's image in shared memory: two rows of the lane at a time (fewer live registers;
+        // the 16-byte operand loads are cheap enough to be issued once per row pair)
+        const uint32_t* xi0 = ximg + (uint32_t)g * img_row_words + (uint32_t)(b - b0) * kImgWords + (uint32_t)(t * 24);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          uint32_t XLh[2][2], XHh[2][2];
+#pragma unroll
+          for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+            for (int sp = 0; sp < 2; ++sp) fr.high(2 * mt + jj, sp, XLh[jj][sp], XHh[jj][sp]);
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl) {
+            uint32_t R[2][2][3];
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+              for (int h = 0; h < 2; ++h) fr.pairs(2 * mt + jj, 2 * h + sl, XLh[jj][h], XHh[jj][h], R[jj][h]);
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+              uint4 bx = make_uint4(0, 0, 0, 0);
+              if (g < batch) bx = *reinterpret_cast<const uint4*>(xi0 + sl * 12 + 4 * i);
+              if (mt == 0) mma_sp16832<0>(acc[0][0], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
+              else mma_sp16832<1>(acc[1][0], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
+            }
+          }
+        }
+      } else {
       uint32_t XL6[4][2], XH6[4][2];
 #pragma unroll
       for (int j = 0; j < 4; ++j)
@@ -276,18 +304,9 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
 #pragma unroll
           for (int h = 0; h < 2; ++h) fr.pairs(j, 2 * h + sl, XL6[j][h], XH6[j][h], R[j][h]);
         // Activations of chunk i of a step: columns 2 i + 2 (t & 1) + {0, 1} of the group's eight.  Up to two batch
-        // rows: from the CTA's image in shared memory (or, when the slice is too long for it, one 4-byte load per
-        // register: few lanes are active); more: the group's 16 bytes through L1, then a select.
-        if (image_bytes != 0u) {
-          const uint32_t* xi = ximg + (uint32_t)g * img_row_words + (uint32_t)(b - b0) * kImgWords + (uint32_t)((t * 2 + sl) * 12);
-#pragma unroll
-          for (int i = 0; i < 3; ++i) {
-            uint4 bx = make_uint4(0, 0, 0, 0);
-            if (g < batch) bx = *reinterpret_cast<const uint4*>(xi + 4 * i);
-            mma_sp16832<0>(acc[0][0], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
-            mma_sp16832<1>(acc[1][0], R[2][0][i], R[3][0][i], R[2][1][i], R[3][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
-          }
-        } else if (batch <= 2) {
+        // rows whose slice is too long for the image: one 4-byte load per register (few lanes are active); more
+        // batch rows: the group's 16 bytes through L1, then a select.
+        if (batch <= 2) {
 #pragma unroll
           for (int i = 0; i < 3; ++i) {
 #pragma unroll
@@ -324,6 +343,7 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
             }
           }
         }
+      }
       }
     } else {
     LaneTile<N> lt;
