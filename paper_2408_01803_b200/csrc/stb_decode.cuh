@@ -292,6 +292,96 @@ STB_HD void meta6_words(const uint32_t (&en)[2][4], uint32_t (&E)[3]) {
   E[2] = prmt(wc, wd, 0x5410u);
 }
 
+// ------------------------------------------------------------------------------------------
+// The same fast decode for ONE of the lane's four rows, the row index j a run-time value (the
+// prefill GEMM gives each of four warps one row of a row tile: one copy of the code serves all).
+struct RowWords {
+  uint32_t mask;            // byte s = keep-mask index of group 4 s + t
+  uint32_t Rlo, Rhi;        // region words: ranks 0..3 of the row's four slots / the word holding its ranks 4..
+  uint32_t Slo, Shi;        // sign words: the one holding ranks 0..3 / ranks 4.. (N = 5: the half word, lower-lane form)
+  uint32_t A, B;            // low / high bytes of the four main scales
+  uint32_t sal2;            // a_sal2 (16 bits)
+};
+template <int N>
+STB_HD void load_row_words(const uint8_t* tile, int lane, int j, RowWords& w) {
+  static_assert(N >= 4 && N <= 6, "fast decode covers N = 4, 5, 6");
+  const int g = lane >> 2, t = lane & 3;
+  if (mask_pairs(N)) {
+    w.mask = 0;
+#pragma unroll
+    for (int sidx = 0; sidx < 4; ++sidx) {
+      const uint32_t f = *reinterpret_cast<const uint16_t*>(tile + pair_field_off(g, j >> 1, sidx, t));
+      w.mask |= pair_field_index(f, j & 1) << (8 * sidx);
+    }
+  } else {
+    w.mask = *reinterpret_cast<const uint32_t*>(tile + lane * 16 + 4 * j);
+  }
+  w.Rlo = *reinterpret_cast<const uint32_t*>(tile + region_word_off(N, j, lane));
+  w.Slo = *reinterpret_cast<const uint32_t*>(tile + sign_word_off(N, j >> 1, lane));
+  w.Rhi = 0; w.Shi = 0;
+  if (N == 6) {
+    w.Rhi = *reinterpret_cast<const uint32_t*>(tile + region_word_off(N, 4 + (j >> 1), lane));
+    w.Shi = *reinterpret_cast<const uint32_t*>(tile + sign_word_off(N, 2, lane));
+  } else if (N == 5) {
+    w.Rhi = *reinterpret_cast<const uint32_t*>(tile + region_word_off(N, 4, lane));
+    const uint32_t h = *reinterpret_cast<const uint32_t*>(tile + sign_half_off(N, lane));
+    w.Shi = lane < 16 ? (h & 0x66666666u) : half_from_upper(h & 0x99999999u);
+  }
+  const uint2 sc = *reinterpret_cast<const uint2*>(tile + scale_off(N, g, j));
+  w.A = sc.x; w.B = sc.y;
+  w.sal2 = *reinterpret_cast<const uint16_t*>(tile + sal2_off(N, g, j));
+}
+
+template <int N>
+struct OneRow {
+  static_assert(N >= 4 && N <= 6, "fast decode covers N = 4, 5, 6");
+  uint32_t A, Bp, Bn, e, o, hs, XL, XH;
+
+  // A_, B_: low / high bytes of the four main scales in the 16-bit format wanted
+  STB_HD void init(const RowWords& w, int j, uint32_t A_, uint32_t B_) {
+    A = A_; Bp = B_; Bn = B_ ^ 0x80808080u;
+    const uint32_t se = w.Slo >> (j & 1), so = w.Slo << (1 + (j & 1));
+    e = (w.Rlo & 0x33333333u) | (se & 0x44444444u);
+    o = ((w.Rlo >> 2) & 0x33333333u) | (so & 0x44444444u);
+    hs = 0; XL = 0; XH = 0;
+    if (N == 6) {
+      const uint32_t sg = j == 0 ? w.Shi : (j == 1 ? (w.Shi << 1) : (j == 2 ? (w.Shi >> 1) : (w.Shi << 2)));
+      hs = ((w.Rhi >> (2 * (j & 1))) & 0x33333333u) | (sg & 0x44444444u);
+    } else if (N == 5) {
+      const uint32_t sel = (j & 2) ? (((w.Rhi >> 2) & 0x33333333u) | ((w.Shi << 1) & 0x44444444u))
+                                   : ((w.Rhi & 0x33333333u) | (w.Shi & 0x44444444u));
+      hs = sel >> (16 * (j & 1));
+      XL = prmt(A, A, hs);
+      XH = prmt(Bp, Bn, hs);
+    }
+  }
+  // N = 6: ranks 4, 5 of slots 2 sp, 2 sp + 1 (call before slot(2 sp, ..) and slot(2 sp + 1, ..))
+  STB_HD void high(int sp) {
+    const uint32_t sel = hs >> (16 * sp);
+    XL = prmt(A, A, sel);
+    XH = prmt(Bp, Bn, sel);
+  }
+  // slot s -> f[0..3]: columns (0,1), (2,3), (4,5), (6,7) as 16-bit pairs; P0 / P1 = position selectors of columns 0..3 / 4..7
+  STB_HD void slot(int s, uint32_t P0, uint32_t P1, uint32_t (&f)[4]) const {
+    const uint32_t sel = ((s & 2) ? o : e) >> (16 * (s & 1));
+    const uint32_t lo0 = prmt(A, A, sel), hi0 = prmt(Bp, Bn, sel);
+    uint32_t lo1 = 0, hi1 = 0;
+    if (N == 6) {
+      lo1 = (s & 1) ? (XL >> 16) : (XL & 0xFFFFu);
+      hi1 = (s & 1) ? (XH >> 16) : (XH & 0xFFFFu);
+    } else if (N == 5) {
+      lo1 = prmt(XL, 0u, 0x4440u + (uint32_t)s);
+      hi1 = prmt(XH, 0u, 0x4440u + (uint32_t)s);
+    }
+    const uint32_t pl0 = prmt(lo0, lo1, P0), pl1 = prmt(lo0, lo1, P1);
+    const uint32_t ph0 = prmt(hi0, hi1, P0), ph1 = prmt(hi0, hi1, P1);
+    f[0] = prmt(pl0, ph0, 0x5140u);
+    f[1] = prmt(pl0, ph0, 0x7362u);
+    f[2] = prmt(pl1, ph1, 0x5140u);
+    f[3] = prmt(pl1, ph1, 0x7362u);
+  }
+};
+
 // position selector of a keep byte: nibble c = rank of column c among the kept columns, 7 for a
 // dropped column (byte 7 of the rank-ordered bytes is zero for N <= 7)
 STB_HD uint32_t position_selector(uint32_t keep_byte) {

@@ -44,10 +44,7 @@ constexpr int kAcc = STB_GEMM_ACC;              // accumulators per CTA: a decod
 constexpr int kTok = kBN * kAcc;                // tokens per CTA
 constexpr int kBK = 64;           // K per stage: one 128-byte swizzle row of bf16
 constexpr int kStages = kAcc == 1 ? 4 : 2;
-#ifndef STB_GEMM_GROUPS
-#define STB_GEMM_GROUPS 4
-#endif
-constexpr int kGroups = STB_GEMM_GROUPS;                // decode warps per 32-row quarter: 1, 2 or 4
+constexpr int kGroups = 4;                              // decode warps per 32-row quarter: one per row of a lane
 constexpr int kGemmThreads = 64 + 128 * kGroups;
 constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
 constexpr uint32_t kStageB = kTok * kBK * 2;     // 32 KB per accumulator
@@ -132,190 +129,121 @@ struct DecodeArgs {
   int mt, b0, b1, nblk, ntile, q, lane;
 };
 
-// Decode role of one warp: rows J0 .. J0 + NJ - 1 (of the four rows g + 8 j each lane owns) of
-// packed row tile 4 mt + q, for every block of the CTA's K range, written into the A stages.
-template <int N, int J0, int NJ>
-__device__ __forceinline__ void decode_rows(const DecodeArgs& da) {
+// Decode role of one warp: row j (of the four rows g + 8 j each lane owns) of packed row tile 4 mt + q, for
+// every block of the CTA's K range, written into the A stages.  j is a run-time value: the four warps of a
+// row tile run the same code.
+template <int N>
+__device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
   const uint8_t* packed = da.packed;
   const Header* hdr = da.hdr;
   uint8_t* smem = da.smem;
   volatile int* abort_flag = da.abort_flag;
   const uint32_t bar_full = da.bar_full, bar_empty = da.bar_empty;
   const int mt = da.mt, b0 = da.b0, b1 = da.b1, nblk = da.nblk, ntile = da.ntile, q = da.q;
-    // The lane plays the part of packed-layout lane 4 g + t with g = lane % 8, t = lane / 8: the eight
-    // lanes of a quarter-warp then hold eight different rows g and their 16-byte stores into the
-    // swizzled stage fall on eight different 16-byte bank groups (no conflict); loads of the
-    // lane-major planes stay coalesced, they are only permuted inside the warp.
-    const int g = da.lane & 7, t = da.lane >> 3;
-    const int lane = 4 * g + t;
-    const int rtile = mt * 4 + q;                 // packed row tile
-    const bool live = rtile < ntile;
-    const uint32_t* ptab = reinterpret_cast<const uint32_t*>(smem + kGemmTab);     // low half: columns 0..3, high half: 4..7
-    const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
-    const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
-    const int spb = (int)hdr->spb;
-    const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                              (size_t)rtile * nblk * resid_tile_bytes(spb);
-    constexpr uint32_t tbytes = tile_bytes(N);
-    LaneTile<N> cur = {}, nxt = {};
-    // salient metadata of a block, fetched one block ahead like the tile: the count, and for the
-    // lane's slots t, t + 4 (slots beyond 8 are fetched on demand) the column bytes and residual words
-    struct Sal { int nsal; uint32_t cw[2], rw[2]; };
-    auto load_sal = [&](int b, Sal& z) {
-      z.nsal = (int)__ldg(&binfo[b].nsal);
-      z.cw[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols));
-      z.cw[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + 1);
-      const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb);
-      z.rw[0] = spb > 0 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 0))) : 0x55555555u;
-      z.rw[1] = spb > 4 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 1))) : 0x55555555u;
-    };
-    Sal csal = {0, {0, 0}, {0, 0}}, nsalv = {0, {0, 0}, {0, 0}};
-    if (live && b0 < b1) { load_lane_tile<N>(rtbase + (size_t)b0 * tbytes, lane, cur); load_sal(b0, csal); }
-    bool ok = true;
-    for (int b = b0; b < b1 && ok; ++b) {
-      if (live && b + 1 < b1) { load_lane_tile<N>(rtbase + (size_t)(b + 1) * tbytes, lane, nxt); load_sal(b + 1, nsalv); }
-      // bf16 scale bytes of the lane's four rows
-      uint32_t A16[4] = {0, 0, 0, 0}, B16[4] = {0, 0, 0, 0};
-      float a1f[4] = {0.f, 0.f, 0.f, 0.f}, a2f[4] = {0.f, 0.f, 0.f, 0.f};
+  // The lane plays the part of packed-layout lane 4 g + t with g = lane % 8, t = lane / 8: the eight
+  // lanes of a quarter-warp then hold eight different rows g and their 16-byte stores into the
+  // swizzled stage fall on eight different 16-byte bank groups (no conflict); loads of the
+  // lane-major planes stay coalesced, they are only permuted inside the warp.
+  const int g = da.lane & 7, t = da.lane >> 3;
+  const int lane = 4 * g + t;
+  const int rtile = mt * 4 + q;                 // packed row tile
+  const bool live = rtile < ntile;
+  const uint32_t* ptab = reinterpret_cast<const uint32_t*>(smem + kGemmTab);     // low half: columns 0..3, high half: 4..7
+  const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+  const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
+  const int spb = (int)hdr->spb;
+  const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
+                            (size_t)rtile * nblk * resid_tile_bytes(spb);
+  constexpr uint32_t tbytes = tile_bytes(N);
+  RowWords cur = {}, nxt = {};
+  // salient metadata of a block, fetched one block ahead like the row's words: the count, and for the
+  // lane's slots t, t + 4 (slots beyond 8 are fetched on demand) the column bytes and residual words
+  struct Sal { int nsal; uint32_t cw[2], rw[2]; };
+  auto load_sal = [&](int b, Sal& z) {
+    z.nsal = (int)__ldg(&binfo[b].nsal);
+    z.cw[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols));
+    z.cw[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + 1);
+    const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb);
+    z.rw[0] = spb > 0 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 0))) : 0x55555555u;
+    z.rw[1] = spb > 4 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 1))) : 0x55555555u;
+  };
+  Sal csal = {0, {0, 0}, {0, 0}}, nsalv = {0, {0, 0}, {0, 0}};
+  if (live && b0 < b1) { load_row_words<N>(rtbase + (size_t)b0 * tbytes, lane, j, cur); load_sal(b0, csal); }
+  bool ok = true;
+  for (int b = b0; b < b1 && ok; ++b) {
+    if (live && b + 1 < b1) { load_row_words<N>(rtbase + (size_t)(b + 1) * tbytes, lane, j, nxt); load_sal(b + 1, nsalv); }
+    // bf16 scale bytes of the row
+    uint32_t A16 = 0, B16 = 0;
+    float a1f = 0.f, a2f = 0.f;
+    if (live) {
 #pragma unroll
-      for (int j = J0; j < J0 + NJ; ++j) {
-        uint32_t lo = 0, hi = 0;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t v = live ? bf16_bits(scale_bits<N>(cur, j, c)) : 0u;
-          lo |= (v & 0xFFu) << (8 * c);
-          hi |= (v >> 8) << (8 * c);
-        }
-        A16[j] = lo; B16[j] = hi;
-        a1f[j] = live ? __half2float(__ushort_as_half((unsigned short)scale_bits<N>(cur, j, 3))) : 0.f;
-        a2f[j] = live ? __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(cur, j))) : 0.f;
+      for (int c = 0; c < 4; ++c) {
+        const uint32_t h16 = ((cur.A >> (8 * c)) & 0xFFu) | (((cur.B >> (8 * c)) & 0xFFu) << 8);
+        const uint32_t v = bf16_bits(h16);
+        A16 |= (v & 0xFFu) << (8 * c);
+        B16 |= (v >> 8) << (8 * c);
+        if (c == 3) a1f = __half2float(__ushort_as_half((unsigned short)h16));
       }
-      FastRows<N> fr;
-      fr.init(cur, A16, B16);
-      uint32_t XL[4] = {0, 0, 0, 0}, XH[4] = {0, 0, 0, 0};
-      if (N == 5) {
+      a2f = __half2float(__ushort_as_half((unsigned short)cur.sal2));
+    }
+    OneRow<N> row;
+    row.init(cur, j, A16, B16);
+    const int nsal = live ? csal.nsal : 0;
+    // position selectors of the row's slots of this block, looked up before the stage waits
+    uint32_t P[4];
 #pragma unroll
-        for (int j = J0; j < J0 + NJ; ++j) fr.high(j, 0, XL[j], XH[j]);
-      }
-      const int nsal = live ? csal.nsal : 0;
-      // position selectors of the warp's slots of this block, looked up before the stage waits
-      uint32_t P[4][4];
+    for (int sidx = 0; sidx < 4; ++sidx) P[sidx] = live ? ptab[(cur.mask >> (8 * sidx)) & 0xFFu] : 0u;
+    // Salient patches of this block: one per salient slot sq, dealt to the four lanes t of a lane
+    // group; the first one per lane is prepared here.
+    int pc0 = -1; uint32_t prc0 = 1u;          // column and residual code of patch t
+    if (t < nsal) {
+      const int sq = t;
+      pc0 = (int)((csal.cw[0] >> (8 * (sq & 3))) & 0xFFu);
+      prc0 = resid_code(csal.rw[0], j, sq & 3);
+    }
 #pragma unroll
-      for (int j = J0; j < J0 + NJ; ++j)
+    for (int h = 0; h < 2; ++h) {
+      const int it = 2 * (b - b0) + h, st = it % kStages;
+      if (!gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      uint8_t* As = smem + kGemmA + st * kStageA;
+      uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
+      if (N == 6 && live) row.high(h);
 #pragma unroll
-        for (int sidx = 0; sidx < 4; ++sidx) P[j][sidx] = live ? ptab[keep_index_of(cur.mask, j, sidx)] : 0u;
-      // Salient patches of this block: (salient slot sq, row j) pairs, nsal * NJ of them, dealt to
-      // the four lanes t of a lane group; the first one per lane is prepared here.
-      const int np = nsal * NJ;
-      int pc0 = -1, pj0 = J0; uint32_t prc0 = 1u;          // column, row, residual code of patch t
-      if (t < np) {
-        const int sq = t / NJ;
-        pj0 = J0 + t % NJ;
-        const uint32_t cwd = sq < 4 ? csal.cw[0] : (sq < 8 ? csal.cw[1] : __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + (sq >> 2)));
-        pc0 = (int)((cwd >> (8 * (sq & 3))) & 0xFFu);
-        const uint32_t word = sq < 4 ? csal.rw[0] : (sq < 8 ? csal.rw[1] :
-            __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2))));
-        prc0 = resid_code(word, pj0, sq & 3);
-      }
-      if constexpr (kStages >= 4) {
-      // both 64-column halves of the block go out together: two consecutive stages
-      const int it0 = 2 * (b - b0), s0 = it0 % kStages, s1 = (it0 + 1) % kStages;
-      if (!gemm_wait(bar_empty + 8 * s0, ((uint32_t)(it0 / kStages) & 1u) ^ 1u, abort_flag) ||
-          !gemm_wait(bar_empty + 8 * s1, ((uint32_t)((it0 + 1) / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-      uint8_t* Ah[2] = {smem + kGemmA + s0 * kStageA, smem + kGemmA + s1 * kStageA};
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-#pragma unroll
-        for (int j = J0; j < J0 + NJ; ++j) {
-          uint8_t* rowp = Ah[h] + (size_t)(4 * q + j) * 1024 + g * 128;
-#pragma unroll
-          for (int sl = 0; sl < 2; ++sl) {
-            const int sidx = 2 * h + sl;                       // slot s of the block, group 4 sidx + t
-            uint32_t f[4] = {0, 0, 0, 0};
-            if (live) {
-              if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
-              fr.slot2(j, sidx, P[j][sidx], P[j][sidx] >> 16, XL[j], XH[j], f);
-            }
-            const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
-            *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
-          }
-        }
+      for (int sl = 0; sl < 2; ++sl) {
+        const int sidx = 2 * h + sl;                       // slot s of the block, group 4 sidx + t
+        uint32_t f[4] = {0, 0, 0, 0};
+        if (live) row.slot(sidx, P[sidx], P[sidx] >> 16, f);
+        const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
+        *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
       }
       // salient columns: bf16( fl32( s1 a_sal1 + s2 a_sal2 ) ) replaces the value the main decode
       // wrote (whose sign is s1); patch p = t + 4 i of the block's list belongs to lane t
       if (nsal > 0) {
         __syncwarp();
-        for (int p = t; p < np; p += 4) {
-          int c = pc0, j = pj0; uint32_t rc = prc0;
+        for (int p = t; p < nsal; p += 4) {
+          int c = pc0; uint32_t rc = prc0;
           if (p >= 4) {
-            const int sq = p / NJ;
-            j = J0 + p % NJ;
+            const int sq = p;
             c = binfo[b].cols[sq];
-            rc = resid_code(__ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2))), j, sq & 3);
+            const uint32_t word = sq < 8 ? csal.rw[1] :
+                __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2)));
+            rc = resid_code(word, j, sq & 3);
           }
-          if (rc == 1u) continue;
+          if ((c >> 6) != h || rc == 1u) continue;
           const int c64 = c & 63;
-          unsigned short* pv = reinterpret_cast<unsigned short*>(Ah[c >> 6] + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
+          unsigned short* pv = reinterpret_cast<unsigned short*>(rowp + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
           const bool neg1 = (*pv & 0x8000u) != 0;
-          const float a1 = j == 0 ? a1f[0] : (j == 1 ? a1f[1] : (j == 2 ? a1f[2] : a1f[3]));
-          const float a2 = j == 0 ? a2f[0] : (j == 1 ? a2f[1] : (j == 2 ? a2f[2] : a2f[3]));
-          const float v = __fadd_rn(neg1 ? -a1 : a1, rc == 0u ? a2 : -a2);
+          const float v = __fadd_rn(neg1 ? -a1f : a1f, rc == 0u ? a2f : -a2f);
           *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
         }
       }
       fence_async_smem();          // generic-proxy writes -> visible to the tensor core
       __syncwarp();
-      if (lane == 0) { mbar_arrive(bar_full + 8 * s0); mbar_arrive(bar_full + 8 * s1); }
-      } else {
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int it = 2 * (b - b0) + h, st = it % kStages;
-        if (!gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-        uint8_t* As = smem + kGemmA + st * kStageA;
-#pragma unroll
-        for (int j = J0; j < J0 + NJ; ++j) {
-          uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
-#pragma unroll
-          for (int sl = 0; sl < 2; ++sl) {
-            const int sidx = 2 * h + sl;
-            uint32_t f[4] = {0, 0, 0, 0};
-            if (live) {
-              if (N == 6 && sl == 0) fr.high(j, h, XL[j], XH[j]);
-              fr.slot2(j, sidx, P[j][sidx], P[j][sidx] >> 16, XL[j], XH[j], f);
-            }
-            const int chunk = 4 * sl + t;
-            *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
-          }
-        }
-        if (nsal > 0) {
-          __syncwarp();
-          for (int p = t; p < np; p += 4) {
-            int c = pc0, j = pj0; uint32_t rc = prc0;
-            if (p >= 4) {
-              const int sq = p / NJ;
-              j = J0 + p % NJ;
-              c = binfo[b].cols[sq];
-              rc = resid_code(__ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2))), j, sq & 3);
-            }
-            if ((c >> 6) != h || rc == 1u) continue;
-            const int c64 = c & 63;
-            unsigned short* pv = reinterpret_cast<unsigned short*>(As + (size_t)(4 * q + j) * 1024 + g * 128 + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
-            const bool neg1 = (*pv & 0x8000u) != 0;
-            const float a1 = j == 0 ? a1f[0] : (j == 1 ? a1f[1] : (j == 2 ? a1f[2] : a1f[3]));
-            const float a2 = j == 0 ? a2f[0] : (j == 1 ? a2f[1] : (j == 2 ? a2f[2] : a2f[3]));
-            const float v = __fadd_rn(neg1 ? -a1 : a1, rc == 0u ? a2 : -a2);
-            *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-          }
-        }
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_full + 8 * st);
-      }
-      }
-      if (!ok) break;
-      if (live && b + 1 < b1) { cur = nxt; csal = nsalv; }
+      if (lane == 0) mbar_arrive(bar_full + 8 * st);
     }
-
+    if (!ok) break;
+    if (live && b + 1 < b1) { cur = nxt; csal = nsalv; }
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -398,14 +326,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     da.packed = packed; da.hdr = hdr; da.smem = smem; da.abort_flag = abort_flag;
     da.bar_full = bar_full; da.bar_empty = bar_empty;
     da.mt = mt; da.b0 = b0; da.b1 = b1; da.nblk = nblk; da.ntile = ntile; da.q = warp & 3; da.lane = lane;
-    if (kGroups == 1) decode_rows<N, 0, 4>(da);
-    else if (kGroups == 2) { if (gi == 0) decode_rows<N, 0, 2>(da); else decode_rows<N, 2, 2>(da); }
-    else {
-      if (gi == 0) decode_rows<N, 0, 1>(da);
-      else if (gi == 1) decode_rows<N, 1, 1>(da);
-      else if (gi == 2) decode_rows<N, 2, 1>(da);
-      else decode_rows<N, 3, 1>(da);
-    }
+    decode_row<N>(da, gi);
 
     // ---------------- epilogue: TMEM -> registers -> Y ----------------
     const int q = warp & 3;                        // TMEM lane quarter of this warp

@@ -207,6 +207,19 @@ static int check(int trials, int spb) {
             if (kb != keep[r][grp]) { if (++errors < 10) std::printf("keep byte N=%d\n", N); }
             uint32_t f[4];
             fr.slot(j, s, position_selector(kb), XL, XH, f);
+            {   // the one-row form with a run-time row index must give the same registers
+              RowWords rw;
+              load_row_words<N>(tile.data(), lane, j, rw);
+              OneRow<N> orow;
+              orow.init(rw, j, rw.A, rw.B);
+              if (N == 6) orow.high(s >> 1);
+              uint32_t f1[4];
+              const uint32_t pp = position_selector(mask_from_index(N, (rw.mask >> (8 * s)) & 0xFFu));
+              orow.slot(s, pp & 0xFFFFu, pp >> 16, f1);
+              if (f1[0] != f[0] || f1[1] != f[1] || f1[2] != f[2] || f1[3] != f[3] || rw.sal2 != sal2_bits<N>(lt, j)) {
+                if (++errors < 10) std::printf("one row N=%d lane %d j %d s %d\n", N, lane, j, s);
+              }
+            }
             int k = 0;
             for (int c = 0; c < 8; ++c) {
               uint32_t want = 0;
