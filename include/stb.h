@@ -120,14 +120,18 @@ int stb_dequant(const void *packed, int n, int m, int N, void *W, stb_dtype dt, 
 int stb_gemv(const void *packed, int n, int m, int N, const void *x, int batch, size_t ldx,
              void *y, stb_dtype ydt, size_t ldy, int *dev_status, void *stream);
 
-/* Bytes of workspace stb_gemm needs for T tokens (0 if none).  HOST result. */
+/* Bytes of workspace stb_gemm wants for T tokens (0 if none).  HOST result.  Two cases ask for one:
+ * few output tiles (every tile is then split along K and the partial tiles are summed afterwards:
+ * the workspace is required), and many output tiles whose last wave of 148 would be small (only
+ * that wave's tiles are split: the workspace is optional, without it those tiles run unsplit). */
 int stb_gemm_workspace(int n, int m, int N, int T, size_t *bytes);
 
 /* Prefill GEMM:  Y[t][i] = sum_j W^[i][j] * X[t][j]  on the tensor cores (tcgen05, fp32
  * accumulation in tensor memory); W^ is decoded tile by tile to bf16 (RN-even).
  * X: bf16 [T][ldx]; Y: fp32 or bf16 [T][ldy] (ydt).  The compute-bound case of Appendix C.2
  * (prefilling stage, N = sequence length x batch).  ws / ws_bytes: caller-owned workspace of
- * stb_gemm_workspace bytes (may be NULL when that is 0). */
+ * stb_gemm_workspace bytes (may be NULL when that is 0).  A smaller or missing workspace gives
+ * STB_ERR_SIZE when the split is required and the unsplit launch when it is optional. */
 int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size_t ldx, void *Y,
              stb_dtype ydt, size_t ldy, void *ws, size_t ws_bytes, int *dev_status,
              void *stream);
@@ -139,8 +143,9 @@ int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size
  * is forbidden.  For them the split-K partial sums go into a fixed 8 MiB array that is part of
  * the library image: every GPU that loads the library holds these 8 MiB until the process
  * exits.  Same arguments, results and errors as stb_gemm, except:
- *   - a call whose stb_gemm_workspace() exceeds 8 MiB returns STB_ERR_SIZE and launches
- *     nothing (use stb_gemm with your own workspace for it);
+ *   - a call whose required workspace (see stb_gemm_workspace) exceeds 8 MiB returns
+ *     STB_ERR_SIZE and launches nothing (use stb_gemm with your own workspace for it); an
+ *     optional split is used only if its partial tiles fit the array;
  *   - the first call on each device looks the array's device address up (with that device
  *     current); make that first call outside any stream capture;
  *   - all calls share the one array.  It keeps whatever the last call left there; nothing in

@@ -250,8 +250,8 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
 template <int N>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict__ packed, int n, int m, int T,
-            void* __restrict__ Y, int y_bf16, size_t ldy, float* __restrict__ ws, int ksplit, int bps,
-            uint32_t box_bytes, int* dev_status) {
+            void* __restrict__ Y, int y_bf16, size_t ldy, float* __restrict__ ws, int full_tiles, int ksplit, int bps,
+            int ttiles, uint32_t box_bytes, int* dev_status) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const Header* hdr = reinterpret_cast<const Header*>(packed);
   if (!header_matches(hdr, n, m, N)) {
@@ -260,8 +260,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
   }
   const int nblk = m / kBlock, ntile = hdr->ntile;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tt = blockIdx.x, mt = blockIdx.y, kz = blockIdx.z;
-  const int b0 = kz * bps, b1 = min(nblk, b0 + bps);
+  // CTAs 0 .. full_tiles - 1 compute one output tile each over the whole K; the rest come in groups of `ksplit`
+  // per tile, each with `bps` blocks of K, and leave fp32 partial tiles in the workspace
+  const int cta = (int)blockIdx.x;
+  const bool split = cta >= full_tiles;
+  const int tile = split ? full_tiles + (cta - full_tiles) / ksplit : cta;
+  const int kz = split ? (cta - full_tiles) % ksplit : 0;
+  const int tt = tile % ttiles, mt = tile / ttiles;
+  const int b0 = split ? kz * bps : 0, b1 = split ? min(nblk, b0 + bps) : nblk;
   const int nstage = 2 * max(b1 - b0, 0);              // 64-column stages of this CTA
 
   const uint32_t sbase = smem_u32(smem);
@@ -333,7 +339,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     if (gemm_wait(bar_accum, 0u, abort_flag) && nstage > 0) {
       tc_fence_after();
       const int row = mt * kBM + 32 * q + lane;                // output feature (row of W^)
-      float* wsz = ws ? ws + (size_t)kz * (size_t)T * (size_t)n : nullptr;
+      float* wsz = split ? ws + ((size_t)(tile - full_tiles) * ksplit + kz) * (size_t)(kBM * kTok) : nullptr;
 #pragma unroll 1
       for (int cc = gi; cc < kTok / 32; cc += kGroups) {       // the groups share the column chunks
         uint32_t r[32];
@@ -344,7 +350,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
             const int tok = tt * kTok + 32 * cc + i;
             if (tok < T) {
               const float v = __uint_as_float(r[i]);
-              if (wsz) wsz[(size_t)tok * n + row] = v;
+              if (wsz) wsz[(size_t)(32 * cc + i) * kBM + 32 * q + lane] = v;
               else if (y_bf16) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(v);
               else static_cast<float*>(Y)[(size_t)tok * ldy + row] = v;
             }
@@ -362,16 +368,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
   if (threadIdx.x == 0 && *abort_flag && dev_status) *dev_status = STB_ERR_TIMEOUT;
 }
 
-// Split-K reduction: Y[t][i] = sum_z ws[z][t][i], in z order.
-__global__ void gemm_reduce_kernel(const float* __restrict__ ws, int ksplit, int n, int T, void* __restrict__ Y,
-                                   int y_bf16, size_t ldy) {
-  const size_t total = (size_t)T * n;
+// Split-K reduction of the tiles that were computed in parts: partial tile z of split tile u is
+// ws[(u ksplit + z)][token 0..kTok-1][row 0..kBM-1]; summed in z order.
+__global__ void gemm_reduce_kernel(const float* __restrict__ ws, int first_tile, int split_tiles, int ksplit, int ttiles,
+                                   int n, int T, void* __restrict__ Y, int y_bf16, size_t ldy) {
+  const size_t per = (size_t)kBM * kTok, total = (size_t)split_tiles * per;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    float s = 0.0f;
-    for (int z = 0; z < ksplit; ++z) s += ws[(size_t)z * total + i];
-    const size_t tok = i / n, row = i % n;
-    if (y_bf16) static_cast<__nv_bfloat16*>(Y)[tok * ldy + row] = __float2bfloat16_rn(s);
-    else static_cast<float*>(Y)[tok * ldy + row] = s;
+    const size_t u = i / per, r = i % per;
+    const int tile = first_tile + (int)u, tt = tile % ttiles, mt = tile / ttiles;
+    const int tok = tt * kTok + (int)(r / kBM), row = mt * kBM + (int)(r % kBM);
+    if (tok >= T || row >= n) continue;
+    float acc = 0.0f;
+    for (int z = 0; z < ksplit; ++z) acc += ws[(u * ksplit + z) * per + r];
+    if (y_bf16) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(acc);
+    else static_cast<float*>(Y)[(size_t)tok * ldy + row] = acc;
   }
 }
 
@@ -388,6 +398,46 @@ static int gemm_ksplit(int n, int m, int T) {
   if (ks < 1) ks = 1;
   const int bps = (nblk + ks - 1) / ks;          // blocks per split; every split gets at least one
   return (nblk + bps - 1) / bps;
+}
+
+// How a call is laid out on the 148 SMs (one CTA per SM at a time).
+//   few output tiles:   every tile is split along K (`ksplit` parts) into the workspace: mandatory
+//   many output tiles:  whole waves of 148 tiles run unsplit; a small last wave (at most half the SMs) would leave
+//                       the machine idle for a whole tile time, so its tiles are split along K as well, if the
+//                       caller's workspace holds their partial tiles: optional
+struct GemmPlan {
+  int ttiles, tiles, full_tiles, split_tiles, ksplit, bps;
+  size_t mandatory_bytes, preferred_bytes;
+};
+static GemmPlan gemm_plan(int n, int m, int T, size_t ws_bytes, bool have_ws) {
+  GemmPlan p;
+  const int nblk = m / kBlock;
+  p.ttiles = (T + kTok - 1) / kTok;
+  p.tiles = ((n + kBM - 1) / kBM) * p.ttiles;
+  const size_t per = (size_t)kBM * kTok * sizeof(float);
+  const int ks = gemm_ksplit(n, m, T);
+  p.full_tiles = p.tiles; p.split_tiles = 0; p.ksplit = 1; p.bps = nblk;
+  p.mandatory_bytes = 0; p.preferred_bytes = 0;
+  if (ks > 1) {
+    p.full_tiles = 0; p.split_tiles = p.tiles; p.ksplit = ks; p.bps = (nblk + ks - 1) / ks;
+    p.mandatory_bytes = p.preferred_bytes = (size_t)p.tiles * ks * per;
+    return p;
+  }
+  const int tail = p.tiles % 148;
+  if (p.tiles > 148 && tail > 0 && tail <= 74) {
+    int kt = 148 / tail;
+    if (kt > 16) kt = 16;
+    while (kt > 1 && nblk / kt < 4) --kt;
+    if (kt > 1) {
+      const int bps = (nblk + kt - 1) / kt;
+      kt = (nblk + bps - 1) / bps;
+      p.preferred_bytes = (size_t)tail * kt * per;
+      if (have_ws && ws_bytes >= p.preferred_bytes) {
+        p.full_tiles = p.tiles - tail; p.split_tiles = tail; p.ksplit = kt; p.bps = bps;
+      }
+    }
+  }
+  return p;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -407,8 +457,8 @@ static EncodeTiledFn encode_tiled_fn() {
 template <int N>
 static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T, size_t ldx, void* Y, int y_bf16,
                        size_t ldy, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t s) {
-  const int ks = gemm_ksplit(n, m, T);
-  if (ks > 1 && (!ws || ws_bytes < (size_t)ks * T * n * sizeof(float))) return STB_ERR_SIZE;
+  const GemmPlan plan = gemm_plan(n, m, T, ws_bytes, ws != nullptr);
+  if (plan.mandatory_bytes > 0 && (!ws || ws_bytes < plan.mandatory_bytes)) return STB_ERR_SIZE;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return STB_ERR_CUDA;
   CUtensorMap map;
@@ -426,13 +476,13 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
     if (cudaFuncSetAttribute(gemm_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem) != cudaSuccess) return STB_ERR_CUDA;
     attr_done = true;
   }
-  const int nblk = m / kBlock, bps = (nblk + ks - 1) / ks;
-  dim3 grid((unsigned)((T + kTok - 1) / kTok), (unsigned)((n + kBM - 1) / kBM), (unsigned)ks);
-  gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, ks > 1 ? static_cast<float*>(ws) : nullptr,
-                                              ks, bps, box_rows * kBK * 2, dev_status);
+  const unsigned grid = (unsigned)(plan.full_tiles + plan.split_tiles * plan.ksplit);
+  gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, static_cast<float*>(ws), plan.full_tiles,
+                                              plan.ksplit, plan.bps, plan.ttiles, box_rows * kBK * 2, dev_status);
   if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
-  if (ks > 1) {
-    gemm_reduce_kernel<<<148 * 4, 256, 0, s>>>(static_cast<const float*>(ws), ks, n, T, Y, y_bf16, ldy);
+  if (plan.split_tiles > 0) {
+    gemm_reduce_kernel<<<148 * 4, 256, 0, s>>>(static_cast<const float*>(ws), plan.full_tiles, plan.split_tiles, plan.ksplit,
+                                               plan.ttiles, n, T, Y, y_bf16, ldy);
     if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   }
   return STB_OK;
@@ -444,8 +494,7 @@ extern "C" int stb_gemm_workspace(int n, int m, int N, int T, size_t* bytes) {
   if (!bytes) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0 || T < 1) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
-  const int ks = stb::gemm_ksplit(n, m, T);
-  *bytes = ks > 1 ? (size_t)ks * (size_t)T * (size_t)n * sizeof(float) : 0;
+  *bytes = stb::gemm_plan(n, m, T, 0, false).preferred_bytes;
   return STB_OK;
 }
 
@@ -484,10 +533,8 @@ extern "C" int stb_gemm_noalloc(const void* packed, int n, int m, int N, const v
   if (N < 4 || N > 6) return STB_ERR_UNSUPPORTED;
   if (ydt != STB_F32 && ydt != STB_BF16) return STB_ERR_UNSUPPORTED;
   if (ldx < (size_t)m || ldy < (size_t)n || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u)) return STB_ERR_ARG;
-  size_t need = 0;
-  const int rc = stb_gemm_workspace(n, m, N, T, &need);
-  if (rc != STB_OK) return rc;
-  if (need > stb::kNoAllocScratchBytes) return STB_ERR_SIZE;           // this shape needs the caller-workspace entry point
+  // this shape needs the caller-workspace entry point if the partial sums it cannot do without do not fit
+  if (stb::gemm_plan(n, m, T, 0, false).mandatory_bytes > stb::kNoAllocScratchBytes) return STB_ERR_SIZE;
   // The array's name is only a host-side handle: ask the runtime for its address on the current
   // device, once per device, and give the kernels that address.
   static float* scratch_of_device[64] = {nullptr};

@@ -277,6 +277,32 @@ def test_gemm_split_k_uses_the_workspace(stb):
     assert e.value.status == stb.STB_ERR_SIZE
 
 
+def test_gemm_splits_the_tiles_of_a_small_last_wave(stb):
+    """150 output tiles on 148 SMs: the two tiles of the last wave are split along K when the caller gives the
+    workspace stb_gemm_workspace asks for, and run unsplit without it; both must match the oracle (sampled
+    rows, among them rows of the last two tiles) and each other."""
+    import torch
+    n, m, N, T = 150 * 128 - 5, 1024, 5, 100
+    d = si.logical_layer(n, m, N, 612)
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    need = stb.gemm_workspace(n, m, N, T)
+    assert need == 2 * 2 * 128 * 512 * 4                       # two tiles, two parts each, fp32 partial tiles
+    g = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 148 * 128 - 1, 148 * 128, 149 * 128 + 7, n - 1], g.choice(n, 64, replace=False)])).astype(np.int32)
+    toks = np.arange(T)
+    _check_gemm(stb, layer, L, T, 31, rows=rows, toks=toks)
+    x = torch.from_numpy(si.activations(T, m, 31, "bf16")).cuda().to(torch.bfloat16)
+    y_split = stb.gemm(layer, x)
+    y_whole = torch.empty(T, n, device="cuda")
+    stb._check(stb._lib.stb_gemm(stb._ptr(layer.buf), n, m, N, stb._ptr(x), T, m, stb._ptr(y_whole), stb.STB_F32, n,
+                                 None, 0, stb._ptr(layer.dev_status), stb._stream()), "stb_gemm")
+    torch.cuda.synchronize()
+    assert int(layer.dev_status.item()) == 0
+    a, b = y_split.double().cpu().numpy(), y_whole.double().cpu().numpy()
+    assert np.abs(a - b).max() <= 1e-4 * np.abs(b).max()       # the same bf16 products, another fp32 summation order
+
+
 @pytest.mark.parametrize("n,m", [(8192, 8192), (1024, 8192)])
 def test_gemm_full_size_sampled(stb, n, m):
     """LLaMA-2-70B prefill shapes at 4:8, 2048 tokens: sampled (token, row) pairs against the oracle."""
