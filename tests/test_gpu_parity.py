@@ -192,7 +192,7 @@ def test_layer_stack_chains_layers_with_per_layer_N(stb):
         assert np.abs(got - y_ref).max() <= tol
 
 
-@pytest.mark.parametrize("batch", [1, 5, 16])
+@pytest.mark.parametrize("batch", [1, 2, 5, 16])
 def test_layer_stack_runs_same_input_layers_as_one_grid(stb, batch):
     """An MLP-shaped stack: gate and up read the same input (one fused launch, different row counts and
     output types), down reads gate's fp16 output; every layer is checked against the oracle fed the
