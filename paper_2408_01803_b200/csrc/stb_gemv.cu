@@ -202,8 +202,6 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   const int bpr_mask = (1 << lg_bpr) - 1;
   const int my_pos = t >> lg_wpb, my_wq = t & ((1 << lg_wpb) - 1);
   const uint32_t my_resid_off = spb > 0 ? resid_word_off(spb, g, my_wq) : 0u;
-  uint32_t rword = 0x55555555u, rword2 = 0x55555555u, rsal0 = 0, rsal1 = 0;
-  int rblk = b0;
   bool failed = false;
   const __half* xrow[NB];
 #pragma unroll
@@ -213,18 +211,31 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
 #pragma unroll
   for (int c = 0; c < NB; ++c) xsp[c] = xrow[c] ? xrow[c] - t * 8 + 8 * (t >> 1) + 2 * (t & 1) : nullptr;
 
+  struct ResidWords { uint32_t rw[2], cols[2]; uint2 a2; };
+  auto fetch = [&](int gi, ResidWords& w) {
+    w.rw[0] = w.rw[1] = 0x55555555u; w.cols[0] = w.cols[1] = 0u; w.a2 = make_uint2(0u, 0u);
+    const int bi = (gi << lg_bpr) + my_pos;
+    if (bi < cnt) {
+      const int b = wb0 + bi;
+      const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb) + my_resid_off;
+      w.rw[0] = __ldg(reinterpret_cast<const uint32_t*>(rp));
+      w.cols[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols + 4 * my_wq));
+      if (spb == 32) {
+        w.rw[1] = __ldg(reinterpret_cast<const uint32_t*>(rp + 16));
+        w.cols[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols + 4 * (my_wq + 4)));
+      }
+      w.a2 = __ldg(reinterpret_cast<const uint2*>(rtbase + (size_t)b * tbytes + sal2_off(N, g, 0)));
+    }
+  };
+  ResidWords rfirst;
+  rfirst.rw[0] = rfirst.rw[1] = 0x55555555u; rfirst.cols[0] = rfirst.cols[1] = 0u; rfirst.a2 = make_uint2(0u, 0u);
+  if (spb > 0) fetch(0, rfirst);      // in flight during the main loop
+
   for (int it = 0; it < cnt; ++it) {
     const int ch = it / kChunk, kin = it - ch * kChunk;     // chunk and tile inside the chunk
     const int slot = ch % kDepth;
     const uint32_t bar = bar0 + 8u * slot;
     const int b = wb0 + it;
-    const bool mine = spb > 0 && (it & bpr_mask) == my_pos;
-    if (mine) {
-      const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb) + my_resid_off;
-      rword = __ldg(reinterpret_cast<const uint32_t*>(rp));
-      if (spb == 32) rword2 = __ldg(reinterpret_cast<const uint32_t*>(rp + 16));
-      rblk = b;
-    }
     // all lanes poll; the verdict is made warp-uniform so that nobody is left at a __syncwarp
     if (kin == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(ch / kDepth) & 1u, kWaitLimit))) { failed = true; break; }
     const uint8_t* tile = ring + (size_t)slot * L.tile_stride + (size_t)kin * tbytes;
@@ -246,7 +257,6 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
       // of operand registers 2 h, 2 h + 1 (h = t & 1) of the quad's four lanes, i.e. their slots 2 h and 2 h + 1.
       LaneTile<N> lt;
       load_lane_tile<N>(tile, lane, lt, true);
-      if (mine) { rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1]; }
       refill();
       FastRows<N> fr;
       fr.init(lt, lt.A, lt.B);
@@ -348,7 +358,6 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
     } else {
     LaneTile<N> lt;
     load_lane_tile<N>(tile, lane, lt);
-    if (mine) { rsal0 = lt.sal2[0]; rsal1 = lt.sal2[1]; }
     refill();
     FastRows<N> fr;
     fr.init(lt, lt.A, lt.B);
@@ -398,15 +407,26 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
     }
     }
 
-    // residual term: once the salient slots of 16 / SPB blocks are collected (or at the end)
-    if (spb > 0 && ((it & bpr_mask) == bpr_mask || it == cnt - 1)) {
+  }
+
+  // Residual term of the salient columns, after the main stream (its registers and loads stay out of the main
+  // loop): per group of 16 / SPB blocks one tensor-core step with the salient slots as K.  The lane's words of a
+  // group (residual codes, a_sal2 of its rows, the salient columns) are fetched one group ahead.
+  if (spb > 0 && !failed) {
+    const int ngroup = (cnt + bpr_mask) >> lg_bpr;
+    ResidWords cur = rfirst, nxt;
+#pragma unroll 1
+    for (int gi = 0; gi < ngroup; ++gi) {
+      fetch(gi + 1, nxt);
+      const int bi = (gi << lg_bpr) + my_pos;
+      const size_t xoff = (size_t)(wb0 + (bi < cnt ? bi : 0)) * kBlock;
 #pragma unroll 1
       for (int pass = 0; pass < (spb == 32 ? 2 : 1); ++pass) {
-        const uint32_t rw = pass ? rword2 : rword;
+        const uint32_t rw = pass ? cur.rw[1] : cur.rw[0];
         uint32_t fa[4][2];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const uint32_t h = (((j & 2) ? rsal1 : rsal0) >> (16 * (j & 1))) & 0xFFFFu;
+          const uint32_t h = (((j & 2) ? cur.a2.y : cur.a2.x) >> (16 * (j & 1))) & 0xFFFFu;
           const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
           const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
           const uint32_t sel = resid_selector(rw, j);
@@ -415,12 +435,12 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
           fa[j][1] = prmt(lo4, hi4, 0x7362u);
         }
         // the four salient columns behind this lane's residual word
-        const uint32_t cw = __ldg(reinterpret_cast<const uint32_t*>(binfo[rblk].cols + 4 * (my_wq + 4 * pass)));
+        const uint32_t cw = pass ? cur.cols[1] : cur.cols[0];
 #pragma unroll
         for (int c = 0; c < NB; ++c) {
           uint2 xr = make_uint2(0, 0);
           if (xrow[c]) {
-            const unsigned short* xq = reinterpret_cast<const unsigned short*>(xrow[c] - t * 8 + (size_t)rblk * kBlock);
+            const unsigned short* xq = reinterpret_cast<const unsigned short*>(xrow[c] - t * 8 + xoff);
             xr.x = (uint32_t)__ldg(xq + (cw & 0xFFu)) | ((uint32_t)__ldg(xq + ((cw >> 8) & 0xFFu)) << 16);
             xr.y = (uint32_t)__ldg(xq + ((cw >> 16) & 0xFFu)) | ((uint32_t)__ldg(xq + (cw >> 24)) << 16);
           }
@@ -428,7 +448,7 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
           mma16816(acc[1][c], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
         }
       }
-      rword = 0x55555555u; rword2 = 0x55555555u;
+      cur = nxt;
     }
   }
 
