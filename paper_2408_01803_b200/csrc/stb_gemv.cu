@@ -23,13 +23,20 @@ __device__ const Meta6Table g_meta6 = make_meta6_table();
 // Grid: one thread-block cluster of `ksplit` CTAs per row tile (32 rows); CTA k of the cluster
 // takes the k-th slice of the 128-column blocks and its warps take contiguous runs of that
 // slice.  Each warp streams its tiles from HBM into a private ring in shared memory with 1-D
-// bulk copies (kChunk tiles per copy, kDepth copies in flight), reads a tile into registers, decodes it slot by slot
-// into fp16 operand registers (stb_decode.cuh) and multiplies with m16n8k16 tensor-core
-// instructions: A = 16 rows x 16 columns of W^, B = the activations (8 batch rows), read
-// through L1 (they are shared by every CTA of the SM), fp32 accumulators in registers for the
-// whole run.  The residual term of the salient columns goes through the same instruction, with
-// the salient slots of 16 / SPB blocks as its K dimension.  Partial sums: warps through shared
-// memory, CTAs of the cluster through distributed shared memory, both in a fixed order.
+// bulk copies (kChunk tiles per copy, kDepth copies in flight), reads a tile into registers,
+// decodes it into fp16 operand registers (stb_decode.cuh) and multiplies on the tensor cores,
+// fp32 accumulators in registers for the whole run:
+//   N = 4, 5, and N = 6 beyond 8 batch rows: position-order decode, m16n8k16 (A = 16 rows x 16
+//     columns of W^, B = the activations of 8 batch rows read through L1);
+//   N = 6 up to 8 batch rows: the weights stay in rank order and the 2:4 sparse instruction
+//     (m16n8k32) places them: every pair of kept weights is a 2-of-4 selection from a window of
+//     four columns, three overlapping windows per group of 8 (stb_decode.cuh, meta6_nibble);
+//     the activations are read three halves wide, for up to two batch rows from a copy of the
+//     CTA's slice that is laid out in operand order in shared memory once per CTA.
+// The residual term of the salient columns goes through the dense instruction with the salient
+// slots of 16 / SPB blocks as its K dimension, after the weight stream.  Partial sums: warps
+// through shared memory, CTAs of the cluster through distributed shared memory, both in a fixed
+// order.
 #ifndef STB_GEMV_DEPTH
 #define STB_GEMV_DEPTH 4
 #endif
