@@ -13,12 +13,16 @@
 //   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage, tcgen05.commit frees
 //               and accumulator, tcgen05.commit frees the stage; also allocates / frees TMEM
 //   warps 2..   decode: warp w works on rows 32 (w % 4) .. +31 of the tile = one packed row tile;
-//               kGroups warps share a row tile, each taking 4 / kGroups of the four rows a lane
-//               owns (one warp alone per scheduler would be bound by instruction latency);
-//               per 128-column block it loads the lane's words (prefetching the next block),
-//               converts the four fp16 scales of its rows to bf16 (RN-even) and writes the two
-//               64-column halves of the block into two stages; afterwards the same warps read
-//               the accumulator (TMEM lanes 32 (w % 4) ..) and store Y.
+//               four warps share a row tile, each taking one of the four rows a lane owns (the row
+//               index is a run-time value: one copy of the code; one warp alone per scheduler
+//               would be bound by instruction latency); per 128-column block it loads its row's
+//               words (prefetching the next block), converts the four fp16 scales to bf16
+//               (RN-even) and writes the two 64-column halves of the block into two stages;
+//               afterwards the same warps read the accumulator (TMEM lanes 32 (w % 4) ..) and
+//               store Y.
+// One CTA fits an SM, so the grid runs in waves of 148 output tiles; tiles of a small last wave
+// (and all tiles when there are few) are split along K into fp32 partial tiles in the caller's
+// workspace and summed by a second kernel.
 // Every wait on an mbarrier is bounded; a wait that runs out sets an abort flag (all roles then
 // leave their loops), reports STB_ERR_TIMEOUT through dev_status and the CTA still frees TMEM.
 #include <cuda.h>
