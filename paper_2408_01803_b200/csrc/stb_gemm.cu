@@ -10,8 +10,8 @@
 //       divides the decode work per flop by kAcc,
 // in a ring of kStages stages over K.  Warp roles:
 //   warp 0      TMA producer (one lane): X slices
-//   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage, tcgen05.commit frees
-//               and accumulator, tcgen05.commit frees the stage; also allocates / frees TMEM
+//   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage and accumulator,
+//               tcgen05.commit frees the stage; also allocates / frees TMEM
 //   warps 2..   decode: warp w works on rows 32 (w % 4) .. +31 of the tile = one packed row tile;
 //               four warps share a row tile, each taking one of the four rows a lane owns (the row
 //               index is a run-time value: one copy of the code; one warp alone per scheduler
