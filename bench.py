@@ -603,6 +603,11 @@ def cuda_arm(args):
         line["cpu_baseline"] = {"value": wl.bytes_step * reps / t / 1e9, "unit": UNIT, "cores": oracle.hardware_threads(),
                                 "kind": "oracle", "sample": "all output rows of gate, up and down, batch 1, %d passes (%.1f s)" % (reps, t),
                                 "us_per_layer": round(1e6 * t / reps / 3, 1)}
+        # the same oracle on one core, on every 8th output row (scaled to all rows)
+        rows8 = [r[::8] for r in rows]
+        t1 = min(oracle_pass(Ls, xs, rows8, threads=1) for _ in range(2)) * 8.0
+        line["cpu_baseline"]["one_core"] = {"value": wl.bytes_step / t1 / 1e9, "unit": UNIT, "us_per_layer": round(1e6 * t1 / 3, 1),
+                                            "sample": "every 8th output row, one thread, time scaled by 8"}
     print(json.dumps(line))
     if world > 1:
         dist.barrier()
