@@ -267,7 +267,8 @@ def gemv_table(stb, torch, wl, pk):
             us = time_graph(torch, g, len(fns))
             out.append({"layer": name, "n": n, "m": m, "N": N, "batch": b, "us_per_layer": round(us, 3),
                         "packed_MB": round(sbytes / 1e6, 3), "GBps": round(sbytes / us / 1e3, 1),
-                        "frac_of_measured_hbm": round(sbytes / us / 1e3 / pk["hbm_gbs"], 4)})
+                        "frac_of_measured_hbm": round(sbytes / us / 1e3 / pk["hbm_gbs"], 4),
+                        "frac_of_nominal_hbm_8TBps": round(sbytes / us / 1e3 / 8000.0, 4)})
             del g
 
     ncopy = len(wl.layers)
@@ -360,6 +361,7 @@ def gemm_table(stb, torch, pk):
         fl = 2.0 * n * m * T
         out.append({"layer": name, "n": n, "m": m, "tokens": T, "N": N, "us": round(us, 1), "dense_TFLOPs": round(fl / us / 1e6, 1),
                     "frac_of_measured_bf16_burst": round(fl / us / 1e6 / pk["bf16_tflops"], 4),
+                    "frac_of_nominal_bf16_2250TF": round(fl / us / 1e6 / 2250.0, 4),
                     "frac_of_measured_bf16_sustained": round(fl / us / 1e6 / pk["bf16_tflops_sustained"], 4),
                     "useful_TFLOPs": round(fl * N / 8 / us / 1e6, 1), "split_k_workspace_MB": round(need / 1e6, 1),
                     "cublas_bf16_us": round(usd, 1), "cublas_bf16_TFLOPs": round(fl / usd / 1e6, 1)})
