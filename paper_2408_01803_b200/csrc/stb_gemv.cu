@@ -38,10 +38,10 @@ __device__ const Meta6Table g_meta6 = make_meta6_table();
 // through shared memory, CTAs of the cluster through distributed shared memory, both in a fixed
 // order.
 #ifndef STB_GEMV_DEPTH
-#define STB_GEMV_DEPTH 4
+#define STB_GEMV_DEPTH 2
 #endif
 #ifndef STB_GEMV_CHUNK
-#define STB_GEMV_CHUNK 1
+#define STB_GEMV_CHUNK 2
 #endif
 constexpr int kDepth = STB_GEMV_DEPTH;     // ring slots per warp
 constexpr int kChunk = STB_GEMV_CHUNK;     // tiles per bulk copy (consecutive blocks of a row tile are contiguous)
