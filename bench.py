@@ -576,10 +576,10 @@ def cuda_arm(args):
                      "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
                      "note": "launch_us = timed region / launches (includes the gaps between launches; a launch is gate+up "
                              "(44.4 MB) or down (22.2 MB), bytes_per_launch is their mean); 6:8 multiplies rank-ordered "
-                             "weights with mma.sp, 286 integer-pipe instructions per 32x128 tile (2 warp-instructions/clk/SM) "
-                             "of 486 in all: the pipe alone allows 0.61 of HBM peak, the kernel issues on 46 % of the cycles",
-                     "alu_bound": {"int_lane_ops_per_s": 148 * 64 * 1.965e9, "int_instr_per_tile": 286,
-                                   "floor_us_per_layer": 5.5}},
+                             "weights with mma.sp, 282 integer-pipe instructions per 32x128 tile (2 warp-instructions/clk/SM) "
+                             "of 493 in all: the pipe alone allows 0.62 of HBM peak, the kernel issues on 48 % of the cycles",
+                     "alu_bound": {"int_lane_ops_per_s": 148 * 64 * 1.965e9, "int_instr_per_tile": 282,
+                                   "floor_us_per_layer": 5.4}},
     }
     if world == 1 and not args.no_extras:
         tab, ctx = gemv_table(stb, torch, wl, pk)
