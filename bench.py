@@ -1,11 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the N:M structured-binary linear layer on B200.
 
-One step = one decode pass (batch 1) over the three MLP linears of a LLaMA-2-7B decoder layer at
+One pass = one decode pass (batch 1) over the three MLP linears of a LLaMA-2-7B decoder layer at
 6:8: gate 11008x4096 and up 11008x4096 read the same fp16 input, down 4096x11008 reads gate's
-fp16 output; the three GEMVs are queued by stb_layer_stack on one stream.  The headline value is
-the effective HBM bandwidth: bytes of packed weights streamed per second.  Weights are resident
-in HBM; every step reads another copy of the packed layers so that no byte comes from L2.
+fp16 output; the three GEMVs are queued by stb_layer_stack on one stream.  The layers are the
+workload's own: dense synthetic weights put through the method's quantizer (the CPU oracle's, run
+here to PREPARE the inputs; it is never on the timed path).  The headline value is the effective
+HBM bandwidth: bytes of packed weights streamed per second.  Weights are resident in HBM; every
+pass reads another copy of the packed layers so that no byte comes from L2.  A "step" of
+--steps is as many passes as it takes for the timed region to last a quarter of a second.
 
   python bench.py [--gpus N] [--steps K] [--warmup W]          CUDA path, one JSON line
   python bench.py --impl reference ...                         the CPU oracle on the host cores
@@ -16,6 +19,7 @@ replica of the same workload: the layer is not sharded, there is no data-path co
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import sys
@@ -32,11 +36,14 @@ import stb_inputs as si
 
 METRIC = "gemv_packed_weight_bandwidth"
 UNIT = "GB/s"
-WORKLOAD = "llama2-7b-mlp gate/up 11008x4096 + down 4096x11008, 6:8, block 128, batch-1 decode GEMV"
-MLP = [("gate", 11008, 4096), ("up", 11008, 4096), ("down", 4096, 11008)]
-MLP_N = 6
+WORKLOAD = ("llama2-7b-mlp gate/up 11008x4096 + down 4096x11008, 6:8, block 128, batch-1 decode GEMV, "
+            "layers made by the oracle's quantizer from the dense synthetic weights")
+MLP = ("gate", "up", "down")
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+MIN_TIMED_S = 0.25
+KERNEL_SOURCES = ("stb_gemv.cu", "stb_decode.cuh", "stb_layout.cuh", "stb_ptx.cuh")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic_gemv_llama7b_mlp_6of8_batch1.txt")
 
 
 def peaks():
@@ -50,9 +57,41 @@ def peaks():
     return d
 
 
-def mlp_logical(k: int) -> dict:
-    name, n, m = MLP[k]
-    return si.logical_layer(n, m, MLP_N, si.seed_for(2, k))
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        h.update(open(os.path.join(ROOT, "paper_2408_01803_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def captured_traffic():
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMV on this workload, from the ncu summary
+    under profiles/ -- or None (with the reason) when there is none or the kernel's sources changed since."""
+    if not os.path.exists(TRAFFIC_FILE):
+        return None, "no capture on file"
+    kv = {}
+    for line in open(TRAFFIC_FILE):
+        if "=" in line and not line.lstrip().startswith("#"):
+            k, v = line.split("=", 1)
+            kv[k.strip()] = v.split("#")[0].strip()
+    if kv.get("source_sha256") != kernel_source_hash():
+        return None, "kernel sources changed since the capture (%s)" % os.path.basename(TRAFFIC_FILE)
+    return float(kv["dram_bytes_per_launch"]), os.path.basename(TRAFFIC_FILE)
+
+
+def quantized(config, name, N=0, verbose=True):
+    """The workload's layer as the method makes it (oracle quantizer, cached on disk): input preparation."""
+    import oracle.workloads as wl
+    n, m, NN, seed = si.workload_layer(config, name, N)
+    return wl.quantized_layer(n, m, NN, seed, verbose=verbose)
+
+
+def salient_histogram(d):
+    import oracle.workloads as wl
+    c = wl.salient_counts(d)
+    return {"mean": round(float(c.mean()), 2), "max": int(c.max()),
+            "blocks_by_count": {"1-4": int(((c >= 1) & (c <= 4)).sum()), "5-8": int(((c >= 5) & (c <= 8)).sum()),
+                                "9-16": int(((c >= 9) & (c <= 16)).sum()), "17-32": int((c >= 17).sum()), "0": int((c == 0).sum())}}
 
 
 # ------------------------------------------------------------------------------------------
@@ -126,16 +165,6 @@ def oracle_pass(Ls, xs, rows, threads=0):
     return time.perf_counter() - t0
 
 
-def stream_bytes_of(d: dict) -> int:
-    """Bytes one GEMV pass streams for a logical layer: 16 + 6N + 10 bytes per row and block plus
-    two residual bits for each of the 0 / 4 / 8 / 16 / 32 salient-column slots of a block (the
-    smallest count that holds the layer's largest block); rows are padded to tiles of 32."""
-    n, m, N = d["n"], d["m"], d["N"]
-    most = max(bin(int(a) | (int(b) << 64)).count("1") for a, b in d["salient"])
-    spb = 0 if most == 0 else 4 if most <= 4 else 8 if most <= 8 else 16 if most <= 16 else 32
-    return -(-n // 32) * 32 * (26 + 6 * N + spb // 4) * (m // 128)
-
-
 def reference_arm(args):
     """The CPU oracle, as it stands, on the host cores: same workload, metric and unit.  Each step
     is a bounded sample of output rows so that the run ends within minutes."""
@@ -143,9 +172,10 @@ def reference_arm(args):
     if rank != 0:
         return
     import oracle
+    import oracle.workloads as wl
     oracle.build()
-    ds = [mlp_logical(k) for k in range(3)]
-    Ls = [oracle.Logical(**d) for d in ds]
+    ds = [quantized(2, name, verbose=False) for name in MLP]
+    Ls = [wl.as_logical(d) for d in ds]
     x0 = si.activations(1, 4096, si.seed_for(2, 8)).astype(np.float64)
     x1 = si.activations(1, 11008, si.seed_for(2, 9)).astype(np.float64)     # stands in for gate's output
     xs = [x0, x0, x1]
@@ -158,7 +188,7 @@ def reference_arm(args):
     frac = min(1.0, frac_probe * budget / max(tp, 1e-6))
     stride = max(1, int(np.ceil(1.0 / frac)))
     rows = [np.arange(0, d["n"], stride, dtype=np.int32) for d in ds]
-    bytes_step = sum(stream_bytes_of(d) * len(r) / (-(-d["n"] // 32) * 32) for d, r in zip(ds, rows))
+    bytes_step = sum(wl.stream_bytes(d) * len(r) / (-(-d["n"] // 32) * 32) for d, r in zip(ds, rows))
     for _ in range(args.warmup):
         oracle_pass(Ls, xs, rows)
     t = 0.0
@@ -178,12 +208,16 @@ def reference_arm(args):
 
 
 # ------------------------------------------------------------------------------------------
+def clone_layer(stb, lay, used):
+    return stb.PackedLayer(lay.n, lay.m, lay.N, lay.buf[:used].clone(), lay.dev_status)
+
+
 class Workload:
     """The MLP layers packed on the device, `copies` times each at distinct addresses."""
 
     def __init__(self, stb, torch, copies):
         self.stb, self.torch = stb, torch
-        self.logical = [mlp_logical(k) for k in range(3)]
+        self.logical = [quantized(2, name) for name in MLP]
         self.layers = []          # [copy][k]
         first = [stb.pack_numpy(d) for d in self.logical]
         torch.cuda.synchronize()
@@ -191,11 +225,7 @@ class Workload:
             assert int(lay.dev_status.item()) == 0
         self.infos = [lay.info() for lay in first]
         for c in range(copies):
-            if c == 0:
-                self.layers.append(first)
-            else:
-                self.layers.append([stb.PackedLayer(l.n, l.m, l.N, l.buf[: self.infos[k]["used_bytes"]].clone(),
-                                                    l.dev_status) for k, l in enumerate(first)])
+            self.layers.append(first if c == 0 else [clone_layer(stb, l, self.infos[k]["used_bytes"]) for k, l in enumerate(first)])
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.x_np = si.activations(1, 4096, si.seed_for(2, 8))
         self.x = torch.from_numpy(self.x_np).cuda()
@@ -205,12 +235,13 @@ class Workload:
         self.steps = [stb.make_steps([(ls[0], self.x, self.h_gate), (ls[1], self.x, self.h_up),
                                       (ls[2], self.h_gate, self.y)]) for ls in self.layers]
         self.bytes_step = sum(i["stream_bytes"] for i in self.infos)
+        self.launches_per_pass = 2          # gate and up read the same input and run as one grid; down is the second launch
 
     def step(self, c):
         self.stb.layer_stack(None, dev_status=self.status, marshalled=self.steps[c % len(self.steps)])
 
     def run_steps(self, first, count):
-        """`count` consecutive steps (copies first, first + 1, ...) as ONE stb_layer_stack call, the way a
+        """`count` consecutive passes (copies first, first + 1, ...) as ONE stb_layer_stack call, the way a
         model's whole stack of linears is queued: every layer after the first is chained to its
         predecessor by a programmatic dependent launch."""
         trip = []
@@ -252,10 +283,16 @@ def time_graph(torch, g, calls_per_replay, min_calls=2000, warm=3):
     return 1e3 * e0.elapsed_time(e1) / (reps * calls_per_replay)
 
 
+def rotating_copies(stb, lay, min_bytes=3 * L2_BYTES, lo=4, hi=48):
+    info = lay.info()
+    k = max(lo, min(hi, -(-min_bytes // info["stream_bytes"])))
+    return [lay] + [clone_layer(stb, lay, info["used_bytes"]) for _ in range(k - 1)], info
+
+
 def gemv_table(stb, torch, wl, pk):
     """Isolated per-layer GEMV timings, cold L2 (rotating over distinct packed copies), for the
-    decode batches of the workload; plus the other decode shapes and a dense bf16 cuBLAS GEMV
-    (torch.matmul) of the same shape as context."""
+    decode batches of the workload; plus the other decode shapes (quantizer-made layers as well) and a
+    dense bf16 cuBLAS GEMV (torch.matmul) of the same shape as context."""
     out = []
 
     def one(name, copies, n, m, N, sbytes, batches):
@@ -272,20 +309,17 @@ def gemv_table(stb, torch, wl, pk):
             del g
 
     ncopy = len(wl.layers)
-    one("gate/up 11008x4096", [wl.layers[c][k] for c in range(ncopy) for k in (0, 1)], 11008, 4096, MLP_N,
+    one("gate/up 11008x4096 (isolated launches)", [wl.layers[c][k] for c in range(ncopy) for k in (0, 1)], 11008, 4096, 6,
         wl.infos[0]["stream_bytes"], (1, 4, 8, 16))
-    one("down 4096x11008", [wl.layers[c][2] for c in range(ncopy)], 4096, 11008, MLP_N,
+    one("down 4096x11008 (isolated launches)", [wl.layers[c][2] for c in range(ncopy)], 4096, 11008, 6,
         wl.infos[2]["stream_bytes"], (1, 4, 8, 16))
-    # other decode shapes of the workload list (batch 1): 7B attention at 4:8, 13B block at 5:8
-    for name, n, m, N, item in (("7B q_proj 4096x4096", 4096, 4096, 4, 0), ("13B q 5120x5120", 5120, 5120, 5, 1),
-                                ("13B gate 13824x5120", 13824, 5120, 5, 2), ("13B down 5120x13824", 5120, 13824, 5, 3)):
-        d = si.logical_layer(n, m, N, si.seed_for(3, item))
+    # other decode shapes of the workload list (batch 1): 7B attention at 4:8, 13B block shapes at 5:8
+    for label, config, name in (("7B q_proj 4096x4096", 1, "q"), ("13B q 5120x5120", 3, "q"),
+                                ("13B gate 13824x5120", 3, "gate"), ("13B down 5120x13824", 3, "down")):
+        d = quantized(config, name)
         lay = stb.pack_numpy(d)
-        used = lay.info()["used_bytes"]
-        sb = lay.info()["stream_bytes"]
-        k = max(4, min(48, -(-3 * L2_BYTES // sb)))
-        copies = [lay] + [stb.PackedLayer(n, m, N, lay.buf[:used].clone(), lay.dev_status) for _ in range(k - 1)]
-        one(name, copies, n, m, N, sb, (1,))
+        copies, info = rotating_copies(stb, lay)
+        one(label, copies, d["n"], d["m"], d["N"], info["stream_bytes"], (1,))
         del copies, lay
         torch.cuda.empty_cache()
     # dense bf16 context
@@ -304,20 +338,19 @@ def gemv_table(stb, torch, wl, pk):
     return out, ctx
 
 
-def gemm_table(stb, torch, pk):
+def gemm_table(stb, torch, pk, real_ffn):
     """Prefill GEMM (stb_gemm, tcgen05) on the LLaMA-2-70B linear shapes at 4:8, 2048 bf16 tokens, with a
-    dense bf16 cuBLAS GEMM (torch.matmul) of the same shape beside it.  The two tall / wide FFN layers
-    are built on the device by repeating the rows / column blocks of the 8192 x 8192 logical layer
-    (valid layers of the same format; the kernel's work does not depend on the values)."""
+    dense bf16 cuBLAS GEMM (torch.matmul) of the same shape beside it.  q/o and k/v are quantizer-made.  The
+    two tall / wide FFN layers take the CPU quantizer minutes, so by default they are built on the device by
+    repeating the rows / column blocks of the quantizer-made 8192 x 8192 layer (valid layers with the same
+    salient-column statistics; --real-ffn quantizes the real ones, as tests/ do)."""
     T, N = 2048, 4
-    base = si.logical_layer(8192, 8192, N, si.seed_for(4, 0))
-    kv = si.logical_layer(1024, 8192, N, si.seed_for(4, 1))
     views = {"keep": np.uint8, "sign": np.uint8, "region": np.int16, "sign2": np.int32, "salient": np.int64, "scale": np.int16}
 
     def up(d):
         return {k: torch.from_numpy(np.ascontiguousarray(d[k]).view(v)).cuda() for k, v in views.items()}
 
-    def rows_x(t, times):      # 28672 = 3.5 x 8192 rows
+    def rows_x(t):             # 28672 = 3.5 x 8192 rows
         return {k: (v if k == "salient" else torch.cat([v] * 3 + [v[:4096]], 0).contiguous()) for k, v in t.items()}
 
     def cols_x(t):             # 28672 = 3.5 x 8192 columns (whole 128-column blocks)
@@ -330,11 +363,20 @@ def gemm_table(stb, torch, pk):
                 out[k] = torch.cat([v] * 3 + [v[:, :half]], 1).contiguous()
         return out
 
-    b = up(base)
-    cases = [("q/o 8192x8192", 8192, 8192, b), ("k/v 1024x8192", 1024, 8192, up(kv)),
-             ("gate/up 28672x8192", 28672, 8192, rows_x(b, 3.5)), ("down 8192x28672", 8192, 28672, cols_x(b))]
+    dq = quantized(4, "q")
+    b = up(dq)
+    cases = [("q/o 8192x8192", 8192, 8192, b, "oracle-quantized", salient_histogram(dq))]
+    dk = quantized(4, "k")
+    cases.append(("k/v 1024x8192", 1024, 8192, up(dk), "oracle-quantized", salient_histogram(dk)))
+    if real_ffn:
+        dg, dd = quantized(4, "gate"), quantized(4, "down")
+        cases += [("gate/up 28672x8192", 28672, 8192, up(dg), "oracle-quantized", salient_histogram(dg)),
+                  ("down 8192x28672", 8192, 28672, up(dd), "oracle-quantized", salient_histogram(dd))]
+    else:
+        cases += [("gate/up 28672x8192", 28672, 8192, rows_x(b), "rows of the quantized q layer repeated 3.5 times", None),
+                  ("down 8192x28672", 8192, 28672, cols_x(b), "column blocks of the quantized q layer repeated 3.5 times", None)]
     out = []
-    for name, n, m, t in cases:
+    for name, n, m, t, how, hist in cases:
         lay = stb.pack(n, m, N, t["keep"], t["sign"], t["region"], t["sign2"], t["salient"], t["scale"])
         torch.cuda.synchronize()
         assert int(lay.dev_status.item()) == 0, name
@@ -359,81 +401,92 @@ def gemm_table(stb, torch, pk):
         W = torch.randn(n, m, device="cuda").to(torch.bfloat16)
         usd = timed(lambda: torch.matmul(x, W.t(), out=y))
         fl = 2.0 * n * m * T
-        out.append({"layer": name, "n": n, "m": m, "tokens": T, "N": N, "us": round(us, 1), "dense_TFLOPs": round(fl / us / 1e6, 1),
-                    "frac_of_measured_bf16_burst": round(fl / us / 1e6 / pk["bf16_tflops"], 4),
-                    "frac_of_nominal_bf16_2250TF": round(fl / us / 1e6 / 2250.0, 4),
-                    "frac_of_measured_bf16_sustained": round(fl / us / 1e6 / pk["bf16_tflops_sustained"], 4),
-                    "useful_TFLOPs": round(fl * N / 8 / us / 1e6, 1), "split_k_workspace_MB": round(need / 1e6, 1),
-                    "cublas_bf16_us": round(usd, 1), "cublas_bf16_TFLOPs": round(fl / usd / 1e6, 1)})
+        row = {"layer": name, "n": n, "m": m, "tokens": T, "N": N, "inputs": how, "us": round(us, 1), "dense_TFLOPs": round(fl / us / 1e6, 1),
+               "frac_of_measured_bf16_burst": round(fl / us / 1e6 / pk["bf16_tflops"], 4),
+               "frac_of_nominal_bf16_2250TF": round(fl / us / 1e6 / 2250.0, 4),
+               "frac_of_measured_bf16_sustained": round(fl / us / 1e6 / pk["bf16_tflops_sustained"], 4),
+               "useful_TFLOPs": round(fl * N / 8 / us / 1e6, 1), "split_k_workspace_MB": round(need / 1e6, 1),
+               "cublas_bf16_us": round(usd, 1), "cublas_bf16_TFLOPs": round(fl / usd / 1e6, 1)}
+        if hist:
+            row["salient_columns_per_block"] = hist
+        out.append(row)
         del lay, W, x, y, ws, flush
         torch.cuda.empty_cache()
     return out
+
+
+def decoder(h, f):
+    return [("q", h, h), ("k", h, h), ("v", h, h), ("o", h, h), ("gate", f, h), ("up", f, h), ("down", h, f)]
+
+
+def build_stack(stb, config, names_N):
+    """Packed layers of a stack, every one at its own address; one quantizer-made layer per (shape, N) family."""
+    cache, layers = {}, []
+    for name, N in names_N:
+        n, m, NN, seed = si.workload_layer(config, name, N)
+        key = (n, m, NN)
+        if key not in cache:
+            fam = {"k": "q", "v": "q", "o": "q", "up": "gate"}.get(name, name)
+            base = stb.pack_numpy(quantized(config, fam, N))
+            cache[key] = (base, base.info())
+        base, info = cache[key]
+        layers.append((name, clone_layer(stb, base, info["used_bytes"]), info["stream_bytes"]))
+    return layers
+
+
+def run_stack(stb, torch, layers, h, f, batch, nl, min_calls):
+    """All linears of `nl` decoder layers as ONE stb_layer_stack call in a CUDA graph; microseconds per call."""
+    x = torch.from_numpy(si.activations(batch, h, si.seed_for(5, 40))).cuda()
+    hb = [torch.empty(batch, h, dtype=torch.float16, device="cuda") for _ in range(5)]     # q k v o + layer output
+    fb = [torch.empty(batch, f, dtype=torch.float16, device="cuda") for _ in range(2)]
+    steps, cur = [], x
+    for l in range(nl):
+        q, k, v, o, gate, up, down = [lay for _, lay, _ in layers[7 * l: 7 * l + 7]]
+        steps += [(q, cur, hb[0]), (k, cur, hb[1]), (v, cur, hb[2]), (o, hb[0], hb[3]), (gate, hb[3], fb[0]),
+                  (up, hb[3], fb[1]), (down, fb[0], hb[4])]
+        cur = hb[4]      # (the data flow of attention / activation functions is not part of this path)
+    arr = stb.make_steps(steps)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fn = lambda: stb.layer_stack(None, dev_status=status, marshalled=arr)
+    g = capture(torch, [fn])
+    us = time_graph(torch, g, 1, min_calls=min_calls)
+    assert int(status.item()) == 0
+    return us
 
 
 def stack_tables(stb, torch, pk):
     """Whole decoder stacks as single stb_layer_stack calls (the other decode workloads):
       * one LLaMA-2-13B decoder block at 5:8, batch 1 (q/k/v, o, gate/up, down chained on one stream);
       * all 224 linears of a 32-layer LLaMA-2-7B stack with N drawn per decoder layer from {4, 5, 6}
-        (seeded), batch 1, 8 and 64.
-    One logical layer is drawn per (shape, N) and packed once per use at its own address (the kernels'
-    work does not depend on the values), so that the 2.5-3.1 GB of a 7B stack are all distinct memory."""
+        (seeded), batch 1, 8 and 64 -- the largest decode workload; its batch-1 line carries its own roofline.
+    One layer is quantized per (shape, N) family and packed once per use at its own address (the kernels'
+    work does not depend on which layer of a family it is), so that the 2.5-3.1 GB of a 7B stack are all
+    distinct memory."""
     out = []
-
-    def build(shapes, Ns):
-        cache, layers = {}, []
-        for (name, n, m), N in zip(shapes, Ns):
-            key = (n, m, N)
-            if key not in cache:
-                cache[key] = stb.pack_numpy(si.logical_layer(n, m, N, si.seed_for(5, len(cache))))
-            base = cache[key]
-            used = base.info()["used_bytes"]
-            layers.append((name, stb.PackedLayer(n, m, N, base.buf[:used].clone(), base.dev_status), base.info()["stream_bytes"]))
-        return layers
-
-    def decoder(h, f):
-        return [("q", h, h), ("k", h, h), ("v", h, h), ("o", h, h), ("gate", f, h), ("up", f, h), ("down", h, f)]
-
-    def run_stack(layers, h, f, batch, nl):
-        x = torch.from_numpy(si.activations(batch, h, si.seed_for(5, 40))).cuda()
-        hb = [torch.empty(batch, h, dtype=torch.float16, device="cuda") for _ in range(5)]     # q k v o + layer output
-        fb = [torch.empty(batch, f, dtype=torch.float16, device="cuda") for _ in range(2)]
-        steps, cur = [], x
-        for l in range(nl):
-            q, k, v, o, gate, up, down = [lay for _, lay, _ in layers[7 * l: 7 * l + 7]]
-            steps += [(q, cur, hb[0]), (k, cur, hb[1]), (v, cur, hb[2]), (o, hb[0], hb[3]), (gate, hb[3], fb[0]),
-                      (up, hb[3], fb[1]), (down, fb[0], hb[4])]
-            cur = hb[4]      # (the data flow of attention / activation functions is not part of this path)
-        arr = stb.make_steps(steps)
-        status = torch.zeros(1, dtype=torch.int32, device="cuda")
-        fn = lambda: stb.layer_stack(None, dev_status=status, marshalled=arr)
-        g = capture(torch, [fn])
-        us = time_graph(torch, g, 1, min_calls=20 if nl > 1 else 200)
-        assert int(status.item()) == 0
-        return us
-
-    # 13B block, 5:8, batch 1
-    l13 = build(decoder(5120, 13824), [5] * 7)
+    l13 = build_stack(stb, 3, [(nm, 5) for nm, _, _ in decoder(5120, 13824)])
     b13 = sum(b for _, _, b in l13)
-    us = run_stack(l13, 5120, 13824, 1, 1)
+    us = run_stack(stb, torch, l13, 5120, 13824, 1, 1, 200)
     out.append({"stack": "LLaMA-2-13B decoder block, 7 linears, 5:8, batch 1", "us": round(us, 1), "packed_MB": round(b13 / 1e6, 1),
                 "GBps": round(b13 / us / 1e3, 1), "frac_of_measured_hbm": round(b13 / us / 1e3 / pk["hbm_gbs"], 4)})
     del l13
     torch.cuda.empty_cache()
-    # 32-layer 7B stack, N per decoder layer
-    rng = np.random.default_rng(si.seed_for(5, 0))
-    Nl = [int(v) for v in rng.choice([4, 5, 6], size=32)]
-    shapes, Ns = [], []
-    for l in range(32):
-        shapes += decoder(4096, 11008)
-        Ns += [Nl[l]] * 7
-    l7 = build(shapes, Ns)
+    Nl = si.stack_N_per_layer(32)
+    names_N = [(nm, Nl[l]) for l in range(32) for nm, _, _ in decoder(4096, 11008)]
+    l7 = build_stack(stb, 5, names_N)
     b7 = sum(b for _, _, b in l7)
+    launches = 32 * 4                 # q/k/v as one grid, o, gate/up as one grid, down
     for batch in (1, 8, 64):
-        us = run_stack(l7, 4096, 11008, batch, 32)
-        out.append({"stack": "LLaMA-2-7B, 32 decoder layers x 7 linears, N per layer from {4,5,6} (%d/%d/%d layers)" % (
-                        Nl.count(4), Nl.count(5), Nl.count(6)), "batch": batch, "us": round(us, 1),
-                    "packed_GB": round(b7 / 1e9, 3), "GBps": round(b7 / us / 1e3, 1),
-                    "frac_of_measured_hbm": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "us_per_linear": round(us / 224, 2)})
+        us = run_stack(stb, torch, l7, 4096, 11008, batch, 32, 20)
+        row = {"stack": "LLaMA-2-7B, 32 decoder layers x 7 linears, N per layer from {4,5,6} (%d/%d/%d layers)" % (
+                   Nl.count(4), Nl.count(5), Nl.count(6)), "batch": batch, "us": round(us, 1),
+               "packed_GB": round(b7 / 1e9, 3), "GBps": round(b7 / us / 1e3, 1),
+               "frac_of_measured_hbm": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "us_per_linear": round(us / 224, 2)}
+        if batch == 1:
+            row["roofline"] = {"bound": "hbm", "achieved": round(b7 / us / 1e3, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
+                               "frac": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "traffic": None,
+                               "bytes_per_launch": round(b7 / launches), "launch_us": round(us / launches, 3),
+                               "launches": launches, "peak_source": pk["_source"]}
+        out.append(row)
     del l7
     torch.cuda.empty_cache()
     return out
@@ -479,18 +532,26 @@ def cuda_arm(args):
     import paper_2408_01803_b200 as stb
     pk = peaks()
 
-    copies = 12          # 12 x 65.5 MB per rotation: more than 6 x L2
+    copies = 12          # 12 distinct copies of the three layers per rotation: more than 6 x L2
+    if world > 1 and rank != 0:
+        dist.barrier()   # rank 0 quantizes (and caches) the layers first
     wl = Workload(stb, torch, copies)
+    if world > 1 and rank == 0:
+        dist.barrier()
     K, W = args.steps, args.warmup
 
-    # graph of `copies` consecutive steps (every step another copy of the weights) + remainder
+    # one graph = `copies` consecutive passes (every pass another copy of the weights)
     g_full = capture(torch, [lambda: wl.run_steps(0, copies)])
-    rem = K % copies
-    g_rem = capture(torch, [lambda: wl.run_steps(0, rem)]) if rem else None
     for i in range(max(W, 3)):
         wl.step(i)
-    g_full.replay()
-    torch.cuda.synchronize()
+    us_pass = time_graph(torch, g_full, copies, min_calls=20 * copies)
+    # a step = `reps` graph replays, sized so that the K steps of the timed region last MIN_TIMED_S
+    reps = max(1, int(np.ceil(MIN_TIMED_S / (K * copies * us_pass * 1e-6))))
+    if world > 1:
+        t = torch.tensor([reps], device="cuda", dtype=torch.int64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        reps = int(t.item())
+    passes = K * reps * copies
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -500,10 +561,8 @@ def cuda_arm(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.perf_counter()
     e0.record()
-    for _ in range(K // copies):
+    for _ in range(K * reps):
         g_full.replay()
-    if g_rem is not None:
-        g_rem.replay()
     e1.record()
     sampler.sample()
     torch.cuda.synchronize()
@@ -517,16 +576,16 @@ def cuda_arm(args):
         t = torch.tensor([ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
-    launches = 2 * K                 # gate and up read the same input and run as one grid; down is the second launch
-    value = world * wl.bytes_step * K / (ms * 1e-3) / 1e9
+    launches = wl.launches_per_pass * passes
+    value = world * wl.bytes_step * passes / (ms * 1e-3) / 1e9
     launch_us = 1e3 * ms / launches
-    per_launch_bytes = wl.bytes_step / 2.0
+    per_launch_bytes = wl.bytes_step / float(wl.launches_per_pass)
     achieved = per_launch_bytes / launch_us / 1e3
 
-    # end to end: x from pinned host memory, y back to the host, every step
+    # end to end: x from pinned host memory, y back to the host, every pass
     xh = torch.from_numpy(wl.x_np.copy()).pin_memory()
     yh = torch.empty(1, 4096, dtype=torch.float32).pin_memory()
-    Ke = min(K, 5000)
+    Ke = max(200, min(passes, 4000))
     for i in range(5):
         stb.layer_stack_host(wl.steps[i % copies], xh, yh, dev_status=wl.status)
         torch.cuda.synchronize()
@@ -551,60 +610,67 @@ def cuda_arm(args):
             dist.destroy_process_group()
         return
 
+    traffic, traffic_note = captured_traffic()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms / passes, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "batch": 1, "layers_per_step": 3, "packed_bytes_per_step": wl.bytes_step,
-                   "us_per_layer": round(1e3 * ms / (3 * K), 3),
+        "config": {"workload": WORKLOAD, "inputs": "oracle-quantized", "batch": 1, "layers_per_step": 3,
+                   "packed_bytes_per_step": wl.bytes_step, "us_per_layer": round(1e3 * ms / (3 * passes), 3),
+                   "step": "ms_per_step is per pass over the three layers; each of the %d steps of the timed region is %d passes "
+                           "(%d graph replays) so that the region lasts >= %.2f s" % (K, reps * copies, reps, MIN_TIMED_S),
+                   "passes_timed": passes, "timed_region_ms": round(ms, 3),
+                   "salient_columns_per_block": {name: salient_histogram(d) for name, d in zip(MLP, wl.logical)},
                    "l2": "cold: %d distinct packed copies of each layer (%.0f MB per rotation, L2 is 126 MB)" % (
                        copies, copies * wl.bytes_step / 1e6),
-                   "launch": "one stb_layer_stack call of %d steps (3 linears each) captured in a CUDA graph and replayed; 2 launches "
-                             "per step (gate+up as one grid, down), chained by programmatic dependent launch" % copies,
+                   "launch": "one stb_layer_stack call of %d passes (3 linears each) captured in a CUDA graph and replayed; %d launches "
+                             "per pass (gate+up as one grid, down), chained by programmatic dependent launch" % (copies, wl.launches_per_pass),
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": xh.numel() * 2, "d2h_bytes_per_step": yh.numel() * 4,
                 "steps": Ke, "us_per_step": round(1e6 * e2e_s / Ke, 2),
-                "call": "stb_layer_stack_host: pinned host x -> device, 3 GEMVs, y -> pinned host, stream sync per step"},
+                "call": "stb_layer_stack_host: pinned host x -> device, 3 GEMVs, y -> pinned host, stream sync per pass"},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
-                     "frac": round(achieved / pk["hbm_gbs"], 4),
-                     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture of this
-                     # workload (44.43 MB for gate+up, 22.25 MB for down; mean of the two launches of a step)
-                     "traffic": 33.34e6,
+                     "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": traffic, "traffic_source": traffic_note,
                      "kernel": "stb::gemv_mma_kernel<6,1>", "peak_source": pk["_source"],
                      "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
-                     "note": "launch_us = timed region / launches (includes the gaps between launches; a launch is gate+up "
-                             "(44.4 MB) or down (22.2 MB), bytes_per_launch is their mean); 6:8 multiplies rank-ordered "
-                             "weights with mma.sp, 282 integer-pipe instructions per 32x128 tile (2 warp-instructions/clk/SM) "
-                             "of 493 in all: the pipe alone allows 0.62 of HBM peak, the kernel issues on 48 % of the cycles",
-                     "alu_bound": {"int_lane_ops_per_s": 148 * 64 * 1.965e9, "int_instr_per_tile": 282,
-                                   "floor_us_per_layer": 5.4}},
+                     "note": "launch_us = timed region / launches (includes the gaps between launches; a launch is gate+up or down, "
+                             "bytes_per_launch is their mean); chained launches of one stb_layer_stack call"},
     }
     if world == 1 and not args.no_extras:
         tab, ctx = gemv_table(stb, torch, wl, pk)
         line["gemv_layers"] = tab
+        iso = [r for r in tab if r["batch"] == 1 and r["N"] == 6]
+        line["roofline"]["isolated_launch_frac"] = round(float(np.mean([r["frac_of_measured_hbm"] for r in iso])), 4)
         line["dense_context"] = ctx
-        line["gemm_prefill"] = gemm_table(stb, torch, pk)
+        line["gemm_prefill"] = gemm_table(stb, torch, pk, args.real_ffn)
+        line["gemm_prefill_note"] = "fractions of the MEASURED cuBLAS bf16 burst peak (%s TFLOP/s) decide the 50 %% target; fractions of the nominal 2250 TFLOP/s are printed beside them" % pk["bf16_tflops"]
         line["pack"] = pack_timing(stb, torch, wl)
-        line["decode_stacks"] = stack_tables(stb, torch, pk)
+        st = stack_tables(stb, torch, pk)
+        line["decode_stacks"] = st
+        big = [r for r in st if r.get("batch") == 1 and "roofline" in r][0]
+        line["largest_decode_workload"] = {"metric": METRIC, "value": big["GBps"], "unit": UNIT, "ms_per_step": big["us"] / 1e3,
+                                           "config": {"workload": big["stack"], "inputs": "oracle-quantized, one layer per (shape, N) family", "batch": 1},
+                                           "roofline": big["roofline"]}
         line["paper_context"] = ("paper's own kernel (2:4 1-bit GEMM, RTX 4090): up to 17.85x over ABQ-LLM 2-bit, "
                                  "263.45 TFLOPS = 79.74% of that GPU's sparse tensor-core peak at sequence length 8192")
     if world == 1 and not args.no_cpu:
         import oracle
+        import oracle.workloads as owl
         oracle.build()
-        Ls = [oracle.Logical(**d) for d in wl.logical]
+        Ls = [owl.as_logical(d) for d in wl.logical]
         x0 = wl.x_np.astype(np.float64)
         x1 = wl.h_gate.double().cpu().numpy()
         xs = [x0, x0, x1]
         rows = [np.arange(d["n"], dtype=np.int32) for d in wl.logical]
-        t, reps = 0.0, 0
-        while t < 10.0 and reps < 50:
+        t, n_pass = 0.0, 0
+        while t < 10.0 and n_pass < 50:
             t += oracle_pass(Ls, xs, rows)
-            reps += 1
-        line["cpu_baseline"] = {"value": wl.bytes_step * reps / t / 1e9, "unit": UNIT, "cores": oracle.hardware_threads(),
-                                "kind": "oracle", "sample": "all output rows of gate, up and down, batch 1, %d passes (%.1f s)" % (reps, t),
-                                "us_per_layer": round(1e6 * t / reps / 3, 1)}
+            n_pass += 1
+        line["cpu_baseline"] = {"value": wl.bytes_step * n_pass / t / 1e9, "unit": UNIT, "cores": oracle.hardware_threads(),
+                                "kind": "oracle", "sample": "all output rows of gate, up and down, batch 1, %d passes (%.1f s)" % (n_pass, t),
+                                "us_per_layer": round(1e6 * t / n_pass / 3, 1)}
         # the same oracle on one core, on every 8th output row (scaled to all rows)
         rows8 = [r[::8] for r in rows]
         t1 = min(oracle_pass(Ls, xs, rows8, threads=1) for _ in range(2)) * 8.0
@@ -619,17 +685,17 @@ def cuda_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None, help="default: 60000 (cuda), 20 (reference)")
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=None, help="default: 20")
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the per-layer table and the dense context")
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-layer tables, the prefill GEMM and the decoder stacks")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--real-ffn", action="store_true", help="prefill GEMM: quantize the real 28672-wide FFN layers (CPU minutes)")
     args = ap.parse_args()
+    args.steps = args.steps or 20
     if args.impl == "reference":
-        args.steps = args.steps or 20
         reference_arm(args)
     else:
-        args.steps = args.steps or 60000
         cuda_arm(args)
 
 

@@ -12,7 +12,11 @@
  * All entry points are asynchronous on the CUDA stream they are given (a cudaStream_t passed
  * as void*; NULL = the default stream) unless stated otherwise.  Every data pointer is a
  * DEVICE pointer owned by the caller unless its comment says HOST.  The library allocates no
- * device memory and keeps no mutable global state.  Argument errors are returned
+ * device memory.  Its global state is: constant lookup tables in device memory; per-process,
+ * per-device caches on the host (which kernels already had their shared-memory limit raised on a
+ * device, the device address of the array below, the driver entry point that encodes tensor maps);
+ * and the one 8 MiB device array of stb_gemm_noalloc, which that entry point alone writes.
+ * Argument errors are returned
  * synchronously and launch nothing; conditions only the device can see (a corrupt logical
  * layer, a bounded wait that ran out) are written to the caller's `dev_status` word (device
  * memory, int32, may be NULL, must be zeroed by the caller) and are read by the caller after
@@ -71,8 +75,10 @@ typedef struct stb_logical {
 typedef struct stb_info {
   int n, m, N;
   int status;             /* what the pack kernels found: STB_OK or STB_ERR_CORRUPT */
-  uint64_t used_bytes;    /* header + per-block table + all tiles */
-  uint64_t stream_bytes;  /* tiles only: the bytes one GEMV pass streams from HBM */
+  uint64_t used_bytes;    /* header + tables + all tiles + residual codes */
+  uint64_t stream_bytes;  /* tiles and residual codes: the bytes one GEMV pass streams from HBM:
+                             26 + 6 N bytes per row and block, plus one byte per four salient
+                             columns (rounded up) of the block; rows padded to a multiple of 32 */
 } stb_info;
 
 /* One step of stb_layer_stack: out[batch][n] = layer(in[batch][m]).  HOST struct. */
@@ -87,8 +93,8 @@ typedef struct stb_step {
 } stb_step;
 
 /* Upper bound of the packed size of an n x m layer at N:8 (the packed size depends on the
- * number of salient columns per block, at most 4 bytes per row and block; this is the size
- * with all of them).  *bytes is HOST memory.  Synchronous, no CUDA call. */
+ * number of salient columns of every block, at most 8 bytes per row and block for 32 of them;
+ * this is the size with all of them).  *bytes is HOST memory.  Synchronous, no CUDA call. */
 int stb_pack_size(int n, int m, int N, size_t *bytes);
 
 /* Fused pack / transpose: logical arrays -> the streaming layout read by stb_gemv and
@@ -119,6 +125,16 @@ int stb_dequant(const void *packed, int n, int m, int N, void *W, stb_dtype dt, 
  * N = batch). */
 int stb_gemv(const void *packed, int n, int m, int N, const void *x, int batch, size_t ldx,
              void *y, stb_dtype ydt, size_t ldy, int *dev_status, void *stream);
+
+/* Self-test of the bounded device-side waits (Appendix C describes no counterpart; this is the
+ * library's failure detection).  Launches the stb_gemv kernel for these arguments (N = 4, 5, 6;
+ * other N give STB_ERR_UNSUPPORTED) with its weight copies switched off and its wait limit cut
+ * to about 50 microseconds: every warp's wait for its first tiles runs out, the kernel returns
+ * normally and *dev_status (required) becomes STB_ERR_TIMEOUT; y receives meaningless values.
+ * Nothing faults or hangs, and the next ordinary call works as usual. */
+int stb_gemv_wait_selftest(const void *packed, int n, int m, int N, const void *x, int batch,
+                           size_t ldx, void *y, stb_dtype ydt, size_t ldy, int *dev_status,
+                           void *stream);
 
 /* Bytes of workspace stb_gemm wants for T tokens (0 if none).  HOST result.  Two cases ask for one:
  * few output tiles (every tile is then split along K and the partial tiles are summed afterwards:

@@ -20,7 +20,7 @@ STB_OK, STB_ERR_ARG, STB_ERR_SHAPE, STB_ERR_NM, STB_ERR_SIZE = 0, 1, 2, 3, 4
 STB_ERR_UNSUPPORTED, STB_ERR_CORRUPT, STB_ERR_TIMEOUT, STB_ERR_CUDA = 5, 6, 7, 8
 STB_F16, STB_BF16, STB_F32 = 0, 1, 2
 
-EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv",
+EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
            "stb_gemm_workspace", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host", "stb_status_str"]
 
 
@@ -58,6 +58,7 @@ def _load():
     lib.stb_packed_info.argtypes = [v, p(_Info), v]
     lib.stb_dequant.argtypes = [v, i, i, i, v, i, z, v]
     lib.stb_gemv.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
+    lib.stb_gemv_wait_selftest.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_gemm_workspace.argtypes = [i, i, i, i, p(z)]
     lib.stb_gemm.argtypes = [v, i, i, i, v, i, z, v, i, z, v, z, v, v]
     lib.stb_gemm_noalloc.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
@@ -177,6 +178,16 @@ def gemv(layer: PackedLayer, x, out=None, out_dtype=None, stream=None):
     _check(_lib.stb_gemv(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(x2), batch, x2.stride(0),
                          _ptr(out), ydt, out.stride(0), _ptr(layer.dev_status), _stream(stream)), "stb_gemv")
     return out if x.dim() == 2 else out[0]
+
+
+def gemv_wait_selftest(layer: PackedLayer, x, out, dev_status, stream=None):
+    """stb_gemv_wait_selftest: the GEMV kernel with its copies off and a short wait limit; dev_status
+    (torch.int32[1], zeroed) becomes STB_ERR_TIMEOUT."""
+    x2 = x if x.dim() == 2 else x.unsqueeze(0)
+    ydt = STB_F32 if out.element_size() == 4 else STB_F16
+    _check(_lib.stb_gemv_wait_selftest(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(x2), x2.shape[0], x2.stride(0),
+                                       _ptr(out), ydt, out.stride(-2) if out.dim() == 2 else layer.n, _ptr(dev_status),
+                                       _stream(stream)), "stb_gemv_wait_selftest")
 
 
 def gemm_workspace(n, m, N, T) -> int:

@@ -30,9 +30,9 @@ dequant_kernel(const uint8_t* __restrict__ packed, int n, int m, T* __restrict__
   const int rt = (int)(warp / nblk), b = (int)(warp % nblk);
   const BlockInfo* bi = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header)) + b;
   const uint8_t* tile = packed + hdr->tiles_offset + ((size_t)rt * nblk + b) * (size_t)hdr->tile_bytes;
-  const int spb = (int)hdr->spb;
+  const int nslot = 4 * (int)bi->nrw;
   const uint8_t* resid = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                         ((size_t)rt * nblk + b) * (size_t)resid_tile_bytes(spb);
+                         (size_t)rt * resid_rt_bytes(hdr->nrw) + resid_word_off(bi->rw_off, 0);
   LaneTile<N> lt;
   load_lane_tile<N>(tile, lane, lt);
   const uint64_t sal[2] = {bi->salient[0], bi->salient[1]};
@@ -57,7 +57,7 @@ dequant_kernel(const uint8_t* __restrict__ packed, int n, int m, T* __restrict__
         const float s1 = neg[c] ? -1.0f : 1.0f;
         if (code[c] == 3u) {
           const int q = qbase + __popc(salb & ((1u << c) - 1u));
-          const uint32_t word = q < spb ? *reinterpret_cast<const uint32_t*>(resid + resid_word_off(spb, g, q >> 2)) : 0x55555555u;
+          const uint32_t word = q < nslot ? *reinterpret_cast<const uint32_t*>(resid + resid_word_off((uint32_t)(q >> 2), g)) : 0x55555555u;
           const uint32_t rc = resid_code(word, j, q & 3);
           const float s2 = rc == 0u ? 1.0f : -1.0f;
           v = __fadd_rn(s1 * alpha[3], s2 * alpha[4]);

@@ -30,7 +30,6 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <stdlib.h>
 
 #include "../../include/stb.h"
 #include "stb_decode.cuh"
@@ -41,13 +40,10 @@ namespace stb {
 
 constexpr int kBM = 128;          // rows of W^ per CTA (UMMA M)
 constexpr int kBN = 256;          // tokens per accumulator (UMMA N)
-#ifndef STB_GEMM_ACC
-#define STB_GEMM_ACC 2
-#endif
-constexpr int kAcc = STB_GEMM_ACC;              // accumulators per CTA: a decoded A stage is used kAcc times
+constexpr int kAcc = 2;                         // accumulators per CTA: a decoded A stage is used kAcc times
 constexpr int kTok = kBN * kAcc;                // tokens per CTA
 constexpr int kBK = 64;           // K per stage: one 128-byte swizzle row of bf16
-constexpr int kStages = kAcc == 1 ? 4 : 2;
+constexpr int kStages = 2;
 constexpr int kGroups = 4;                              // decode warps per 32-row quarter: one per row of a lane
 constexpr int kGemmThreads = 64 + 128 * kGroups;
 constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
@@ -155,23 +151,22 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
   const uint32_t* ptab = reinterpret_cast<const uint32_t*>(smem + kGemmTab);     // low half: columns 0..3, high half: 4..7
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
-  const int spb = (int)hdr->spb;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                            (size_t)rtile * nblk * resid_tile_bytes(spb);
+                            (size_t)rtile * resid_rt_bytes(hdr->nrw);
   constexpr uint32_t tbytes = tile_bytes(N);
   RowWords cur = {}, nxt = {};
   // salient metadata of a block, fetched one block ahead like the row's words: the count, and for the
   // lane's slots t, t + 4 (slots beyond 8 are fetched on demand) the column bytes and residual words
-  struct Sal { int nsal; uint32_t cw[2], rw[2]; };
+  struct Sal { int nsal; uint32_t rwo; uint32_t cw[2], rw[2]; };
   auto load_sal = [&](int b, Sal& z) {
     z.nsal = (int)__ldg(&binfo[b].nsal);
+    z.rwo = __ldg(&binfo[b].rw_off);
     z.cw[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols));
     z.cw[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + 1);
-    const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb);
-    z.rw[0] = spb > 0 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 0))) : 0x55555555u;
-    z.rw[1] = spb > 4 ? __ldg(reinterpret_cast<const uint32_t*>(rp + resid_word_off(spb, g, 1))) : 0x55555555u;
+    z.rw[0] = z.nsal > 0 ? __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(z.rwo, g))) : 0x55555555u;
+    z.rw[1] = z.nsal > 4 ? __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(z.rwo + 1u, g))) : 0x55555555u;
   };
-  Sal csal = {0, {0, 0}, {0, 0}}, nsalv = {0, {0, 0}, {0, 0}};
+  Sal csal = {0, 0u, {0, 0}, {0, 0}}, nsalv = {0, 0u, {0, 0}, {0, 0}};
   if (live && b0 < b1) { load_row_words<N>(rtbase + (size_t)b0 * tbytes, lane, j, cur); load_sal(b0, csal); }
   bool ok = true;
   for (int b = b0; b < b1 && ok; ++b) {
@@ -208,7 +203,8 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int it = 2 * (b - b0) + h, st = it % kStages;
-      if (!gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      // the verdict is made warp-uniform: nobody may be left alone at the __syncwarp()s below
+      if (!__all_sync(0xFFFFFFFFu, gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
       uint8_t* As = smem + kGemmA + st * kStageA;
       uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
       if (N == 6 && live) row.high(h);
@@ -230,7 +226,7 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
             const int sq = p;
             c = binfo[b].cols[sq];
             const uint32_t word = sq < 8 ? csal.rw[1] :
-                __ldg(reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, sq >> 2)));
+                __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(csal.rwo + (uint32_t)(sq >> 2), g)));
             rc = resid_code(word, j, sq & 3);
           }
           if ((c >> 6) != h || rc == 1u) continue;
@@ -340,7 +336,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
 
     // ---------------- epilogue: TMEM -> registers -> Y ----------------
     const int q = warp & 3;                        // TMEM lane quarter of this warp
-    if (gemm_wait(bar_accum, 0u, abort_flag) && nstage > 0) {
+    if (__all_sync(0xFFFFFFFFu, gemm_wait(bar_accum, 0u, abort_flag)) && nstage > 0) {
       tc_fence_after();
       const int row = mt * kBM + 32 * q + lane;                // output feature (row of W^)
       float* wsz = split ? ws + ((size_t)(tile - full_tiles) * ksplit + kz) * (size_t)(kBM * kTok) : nullptr;
@@ -364,8 +360,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     }
   }
 
-  // the MMA thread makes sure the tensor core is done with TMEM before it is freed
-  if (warp == 1 && lane == 0) gemm_wait<true>(bar_accum, 0u, abort_flag);
+  // The MMA thread makes sure the tensor core is done with TMEM before it is freed.  Its commit on bar_accum was
+  // issued whether or not the loop above was left early, so this wait ends when the instructions issued so far
+  // have completed; it keeps its own bound and ignores the abort flag.
+  if (warp == 1 && lane == 0) mbar_wait(bar_accum, 0u, kGemmWaitLimit);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_d, kTok);
@@ -391,12 +389,9 @@ __global__ void gemm_reduce_kernel(const float* __restrict__ ws, int first_tile,
 
 // K split: only when the output tiles alone cannot fill the 148 SMs
 static int gemm_ksplit(int n, int m, int T) {
-  static int forced = -1;
-  if (forced < 0) { const char* e = getenv("STB_GEMM_KSPLIT"); forced = e ? atoi(e) : 0; }
   const int tiles = ((n + kBM - 1) / kBM) * ((T + kTok - 1) / kTok), nblk = m / kBlock;
   int ks = 1;
-  if (forced >= 1 && forced <= 16) ks = forced;
-  else if (tiles < 100) ks = 148 / tiles;
+  if (tiles < 100) ks = 148 / tiles;
   if (ks > 16) ks = 16;
   while (ks > 1 && nblk / ks < 4) --ks;
   if (ks < 1) ks = 1;
@@ -475,10 +470,13 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return STB_ERR_ARG;
-  static bool attr_done = false;
-  if (!attr_done) {
+  // the shared-memory limit of a kernel is a per-device setting
+  static bool attr_done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return STB_ERR_CUDA;
+  if (dev < 0 || dev >= 64 || !attr_done[dev]) {
     if (cudaFuncSetAttribute(gemm_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem) != cudaSuccess) return STB_ERR_CUDA;
-    attr_done = true;
+    if (dev >= 0 && dev < 64) attr_done[dev] = true;
   }
   const unsigned grid = (unsigned)(plan.full_tiles + plan.split_tiles * plan.ksplit);
   gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, static_cast<float*>(ws), plan.full_tiles,

@@ -4,7 +4,6 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <stdlib.h>
 
 #include "../../include/stb.h"
 #include "stb_decode.cuh"
@@ -37,15 +36,10 @@ __device__ const Meta6Table g_meta6 = make_meta6_table();
 // slots of 16 / SPB blocks as its K dimension, after the weight stream.  Partial sums: warps
 // through shared memory, CTAs of the cluster through distributed shared memory, both in a fixed
 // order.
-#ifndef STB_GEMV_DEPTH
-#define STB_GEMV_DEPTH 2
-#endif
-#ifndef STB_GEMV_CHUNK
-#define STB_GEMV_CHUNK 2
-#endif
-constexpr int kDepth = STB_GEMV_DEPTH;     // ring slots per warp
-constexpr int kChunk = STB_GEMV_CHUNK;     // tiles per bulk copy (consecutive blocks of a row tile are contiguous)
+constexpr int kDepth = 2;     // ring slots per warp
+constexpr int kChunk = 2;     // tiles per bulk copy (consecutive blocks of a row tile are contiguous)
 constexpr long long kWaitLimit = 2000000000ll;     // about a second of SM clocks
+constexpr long long kSelftestWaitLimit = 100000ll;  // the wait self-test gives up after about 50 microseconds
 
 struct GemvSmem {
   uint32_t bars, ring, part, ximg, total;           // byte offsets
@@ -90,14 +84,12 @@ struct GemvLayers {
 
 // At most 128 threads per CTA, four CTAs per SM for up to 16 batch rows (a bound of five CTAs, 96
 // registers, was measured slower: the spills cost more than the extra resident CTA brings).
-#ifndef STB_GEMV_MINBLOCKS
-#define STB_GEMV_MINBLOCKS 4
-#endif
 constexpr int kGemvMaxThreads = 128;
+constexpr int kMaxDevices = 64;
 template <int N, int NB>
-__global__ void __launch_bounds__(kGemvMaxThreads, NB <= 2 ? STB_GEMV_MINBLOCKS : 1)
+__global__ void __launch_bounds__(kGemvMaxThreads, NB <= 2 ? 4 : 1)
 gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* __restrict__ x, int batch,
-                size_t ldx, int* dev_status, int lg_ksplit, int bpp) {
+                size_t ldx, int* dev_status, int lg_ksplit, int bpp, long long wait_limit, int copies_off) {
   extern __shared__ __align__(128) uint8_t smem[];
   int li = 0, rt_all = (int)(blockIdx.x >> lg_ksplit);
 #pragma unroll
@@ -115,6 +107,9 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   }
   const int nblk = m / kBlock;
   const int ksplit = 1 << lg_ksplit;
+  // A CTA may write into the shared memory of another CTA of its cluster only once that CTA runs: every CTA
+  // arrives here, and waits for the others just before its first remote store (behind the whole weight stream).
+  if (ksplit > 1) cluster_arrive();
   const int warps = (int)(blockDim.x >> 5);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
   const int kpart = (int)(blockIdx.x & (unsigned)(ksplit - 1)), rt = rt_all - layers.tile_start[li];
@@ -122,10 +117,9 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   const int nbp = max(b1 - b0, 0);
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   constexpr uint32_t tbytes = tile_bytes(N);
-  const int spb = (int)hdr->spb;
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)hdr->ntile +
-                            (size_t)rt * nblk * resid_tile_bytes(spb);
+                            (size_t)rt * resid_rt_bytes(hdr->nrw);
   const uint32_t image_bytes = gemv_image_bytes(N, NB, batch, bpp);
   const GemvSmem L = gemv_smem(N, warps, ksplit, NB, image_bytes);
 
@@ -146,7 +140,8 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
     for (int i = 0; i < kDepth && i * kChunk < cnt; ++i) {
       const uint32_t bytes = (uint32_t)min(kChunk, cnt - i * kChunk) * tbytes;
       mbar_expect_tx(bar0 + 8u * i, bytes);
-      bulk_g2s(smem_u32(ring + (size_t)i * L.tile_stride), rtbase + (size_t)(wb0 + i * kChunk) * tbytes, bytes, bar0 + 8u * i);
+      // copies_off (the wait self-test): the barrier is armed but nothing will ever complete it
+      if (!copies_off) bulk_g2s(smem_u32(ring + (size_t)i * L.tile_stride), rtbase + (size_t)(wb0 + i * kChunk) * tbytes, bytes, bar0 + 8u * i);
     }
   }
   if (N == 6 && NB == 1) {   // metadata by keep-mask index (256 bytes: an index byte of the tile cannot point past it)
@@ -202,13 +197,6 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
 #pragma unroll
       for (int d = 0; d < 4; ++d) acc[a][c][d] = 0.0f;
 
-  // Residual bookkeeping: 16 / SPB blocks share one residual instruction (K = 16 salient slots):
-  // lane t keeps the residual word of block (it % bpr) == t / wpb, word t % wpb of that block.
-  const int lg_bpr = spb == 0 || spb >= 16 ? 0 : 4 - ilog2(spb);          // blocks per residual instruction
-  const int lg_wpb = spb >= 16 ? 2 : (spb == 8 ? 1 : 0);                  // words of a block per instruction
-  const int bpr_mask = (1 << lg_bpr) - 1;
-  const int my_pos = t >> lg_wpb, my_wq = t & ((1 << lg_wpb) - 1);
-  const uint32_t my_resid_off = spb > 0 ? resid_word_off(spb, g, my_wq) : 0u;
   bool failed = false;
   const __half* xrow[NB];
 #pragma unroll
@@ -218,25 +206,25 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
 #pragma unroll
   for (int c = 0; c < NB; ++c) xsp[c] = xrow[c] ? xrow[c] - t * 8 + 8 * (t >> 1) + 2 * (t & 1) : nullptr;
 
-  struct ResidWords { uint32_t rw[2], cols[2]; uint2 a2; };
-  auto fetch = [&](int gi, ResidWords& w) {
-    w.rw[0] = w.rw[1] = 0x55555555u; w.cols[0] = w.cols[1] = 0u; w.a2 = make_uint2(0u, 0u);
-    const int bi = (gi << lg_bpr) + my_pos;
-    if (bi < cnt) {
-      const int b = wb0 + bi;
-      const uint8_t* rp = resid_rt + (size_t)b * resid_tile_bytes(spb) + my_resid_off;
-      w.rw[0] = __ldg(reinterpret_cast<const uint32_t*>(rp));
-      w.cols[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols + 4 * my_wq));
-      if (spb == 32) {
-        w.rw[1] = __ldg(reinterpret_cast<const uint32_t*>(rp + 16));
-        w.cols[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols + 4 * (my_wq + 4)));
-      }
-      w.a2 = __ldg(reinterpret_cast<const uint2*>(rtbase + (size_t)b * tbytes + sal2_off(N, g, 0)));
+  // Residual term of the salient columns: the residual words of this warp's run of blocks are numbered
+  // consecutively (stb_layout.cuh); one tensor-core step takes 16 salient slots = four words, lane t the t-th.
+  // A word's table entry names its block and its four salient columns.
+  const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + hdr->rwtab_offset);
+  uint32_t rw0 = 0, rw1 = 0;
+  if (cnt > 0) { rw0 = __ldg(&binfo[wb0].rw_off); rw1 = __ldg(&binfo[wb1 - 1].rw_off) + __ldg(&binfo[wb1 - 1].nrw); }
+  struct ResidWords { uint32_t rw, cols, block; uint2 a2; };
+  auto fetch = [&](uint32_t step, ResidWords& w) {
+    w.rw = 0x55555555u; w.cols = 0u; w.block = (uint32_t)wb0; w.a2 = make_uint2(0u, 0u);
+    const uint32_t wi = rw0 + 4u * step + (uint32_t)t;
+    if (wi < rw1) {
+      const uint2 e = __ldg(reinterpret_cast<const uint2*>(rwt + wi));
+      w.block = e.x; w.cols = e.y;
+      w.rw = __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(wi, g)));
+      w.a2 = __ldg(reinterpret_cast<const uint2*>(rtbase + (size_t)e.x * tbytes + sal2_off(N, g, 0)));
     }
   };
   ResidWords rfirst;
-  rfirst.rw[0] = rfirst.rw[1] = 0x55555555u; rfirst.cols[0] = rfirst.cols[1] = 0u; rfirst.a2 = make_uint2(0u, 0u);
-  if (spb > 0) fetch(0, rfirst);      // in flight during the main loop
+  fetch(0u, rfirst);      // in flight during the main loop
 
   for (int it = 0; it < cnt; ++it) {
     const int ch = it / kChunk, kin = it - ch * kChunk;     // chunk and tile inside the chunk
@@ -244,7 +232,7 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
     const uint32_t bar = bar0 + 8u * slot;
     const int b = wb0 + it;
     // all lanes poll; the verdict is made warp-uniform so that nobody is left at a __syncwarp
-    if (kin == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(ch / kDepth) & 1u, kWaitLimit))) { failed = true; break; }
+    if (kin == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(bar, (uint32_t)(ch / kDepth) & 1u, wait_limit))) { failed = true; break; }
     const uint8_t* tile = ring + (size_t)slot * L.tile_stride + (size_t)kin * tbytes;
     // release of the ring slot: once the whole chunk is in registers or consumed, refill it
     auto refill = [&]() {
@@ -417,43 +405,38 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   }
 
   // Residual term of the salient columns, after the main stream (its registers and loads stay out of the main
-  // loop): per group of 16 / SPB blocks one tensor-core step with the salient slots as K.  The lane's words of a
-  // group (residual codes, a_sal2 of its rows, the salient columns) are fetched one group ahead.
-  if (spb > 0 && !failed) {
-    const int ngroup = (cnt + bpr_mask) >> lg_bpr;
+  // loop): per four residual words one tensor-core step with their 16 salient slots as K.  The lane's word (its
+  // codes, the a_sal2 of its rows in the word's block, the salient columns) is fetched one step ahead.
+  if (rw1 > rw0 && !failed) {
+    const uint32_t nstep = (rw1 - rw0 + 3u) >> 2;
     ResidWords cur = rfirst, nxt;
 #pragma unroll 1
-    for (int gi = 0; gi < ngroup; ++gi) {
-      fetch(gi + 1, nxt);
-      const int bi = (gi << lg_bpr) + my_pos;
-      const size_t xoff = (size_t)(wb0 + (bi < cnt ? bi : 0)) * kBlock;
-#pragma unroll 1
-      for (int pass = 0; pass < (spb == 32 ? 2 : 1); ++pass) {
-        const uint32_t rw = pass ? cur.rw[1] : cur.rw[0];
-        uint32_t fa[4][2];
+    for (uint32_t gi = 0; gi < nstep; ++gi) {
+      fetch(gi + 1u, nxt);
+      const size_t xoff = (size_t)cur.block * kBlock;
+      uint32_t fa[4][2];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t h = (((j & 2) ? cur.a2.y : cur.a2.x) >> (16 * (j & 1))) & 0xFFFFu;
-          const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
-          const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
-          const uint32_t sel = resid_selector(rw, j);
-          const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
-          fa[j][0] = prmt(lo4, hi4, 0x5140u);
-          fa[j][1] = prmt(lo4, hi4, 0x7362u);
-        }
-        // the four salient columns behind this lane's residual word
-        const uint32_t cw = pass ? cur.cols[1] : cur.cols[0];
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t h = (((j & 2) ? cur.a2.y : cur.a2.x) >> (16 * (j & 1))) & 0xFFFFu;
+        const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
+        const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
+        const uint32_t sel = resid_selector(cur.rw, j);
+        const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
+        fa[j][0] = prmt(lo4, hi4, 0x5140u);
+        fa[j][1] = prmt(lo4, hi4, 0x7362u);
+      }
+      // the four salient columns behind this lane's residual word
+      const uint32_t cw = cur.cols;
 #pragma unroll
-        for (int c = 0; c < NB; ++c) {
-          uint2 xr = make_uint2(0, 0);
-          if (xrow[c]) {
-            const unsigned short* xq = reinterpret_cast<const unsigned short*>(xrow[c] - t * 8 + xoff);
-            xr.x = (uint32_t)__ldg(xq + (cw & 0xFFu)) | ((uint32_t)__ldg(xq + ((cw >> 8) & 0xFFu)) << 16);
-            xr.y = (uint32_t)__ldg(xq + ((cw >> 16) & 0xFFu)) | ((uint32_t)__ldg(xq + (cw >> 24)) << 16);
-          }
-          mma16816(acc[0][c], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
-          mma16816(acc[1][c], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
+      for (int c = 0; c < NB; ++c) {
+        uint2 xr = make_uint2(0, 0);
+        if (xrow[c]) {
+          const unsigned short* xq = reinterpret_cast<const unsigned short*>(xrow[c] - t * 8 + xoff);
+          xr.x = (uint32_t)__ldg(xq + (cw & 0xFFu)) | ((uint32_t)__ldg(xq + ((cw >> 8) & 0xFFu)) << 16);
+          xr.y = (uint32_t)__ldg(xq + ((cw >> 16) & 0xFFu)) | ((uint32_t)__ldg(xq + (cw >> 24)) << 16);
         }
+        mma16816(acc[0][c], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
+        mma16816(acc[1][c], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
       }
       cur = nxt;
     }
@@ -481,6 +464,7 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
     }
   __syncthreads();
   float* part = reinterpret_cast<float*>(smem + L.part);       // [ksplit][32][BW], used on cluster rank 0
+  if (ksplit > 1) cluster_wait();
   for (int i = threadIdx.x; i < 32 * BW; i += blockDim.x) {
     float sacc = 0.0f;
     for (int w = 0; w < warps; ++w) sacc += red[(size_t)w * 32 * BW + i];
@@ -510,25 +494,15 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   }
 }
 
-static int env_int(const char* name) {
-  const char* e = getenv(name);
-  return e ? atoi(e) : 0;
-}
-
 // Launch shape: ksplit CTAs per row tile and warps per CTA.  A warp should get a run of several
 // tiles (its ring then streams while it decodes) and the grid should have at least two CTAs per
 // SM while leaving room on the SM for the next layer's CTAs, which start their own weight
 // stream early (programmatic dependent launch).
 static void gemv_shape(int n, int m, int& ksplit, int& warps) {
-  static int f_ks = -1, f_w = -1;
-  if (f_ks < 0) { f_ks = env_int("STB_GEMV_KSPLIT"); f_w = env_int("STB_GEMV_WARPS"); }
   const int ntile = (n + kTileRows - 1) / kTileRows, nblk = m / kBlock;
-  warps = (f_w == 2 || f_w == 4) ? f_w : 4;
+  warps = 4;
   int ks = 1;
-  if (f_ks == 1 || f_ks == 2 || f_ks == 4 || f_ks == 8) ks = f_ks;
-  else
-    while (ks < 8 && ntile * ks < 296 && nblk / (2 * ks * warps) >= 4) ks *= 2;
-  while (ks > 1 && ks > nblk) ks /= 2;
+  while (ks < 8 && ntile * ks < 296 && nblk / (2 * ks * warps) >= 4) ks *= 2;
   ksplit = ks;
 }
 
@@ -536,17 +510,21 @@ static void gemv_shape(int n, int m, int& ksplit, int& warps) {
 // between the GEMVs of one stb_layer_stack call, whose packed layers nobody writes meanwhile).
 template <int N, int NB>
 static cudaError_t launch_mma(const GemvLayers& layers, int m, const __half* x, int batch, size_t ldx,
-                              int* dev_status, cudaStream_t s, bool chained) {
+                              int* dev_status, cudaStream_t s, bool chained, bool wait_selftest = false) {
   const int ntile = layers.tile_start[layers.count], nblk = m / kBlock;
   int ksplit, warps;
   gemv_shape(ntile * kTileRows, m, ksplit, warps);
   const int bpp = (nblk + ksplit - 1) / ksplit;
   const GemvSmem L = gemv_smem(N, warps, ksplit, NB, gemv_image_bytes(N, NB, batch, bpp));
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(gemv_mma_kernel<N, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  // the shared-memory limit of a kernel is a per-device setting
+  static bool attr_done[kMaxDevices] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices || !attr_done[dev]) {
+    e = cudaFuncSetAttribute(gemv_mma_kernel<N, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    if (dev >= 0 && dev < kMaxDevices) attr_done[dev] = true;
   }
   if (L.total > 200 * 1024) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
@@ -569,24 +547,25 @@ static cudaError_t launch_mma(const GemvLayers& layers, int m, const __half* x, 
   cfg.attrs = at; cfg.numAttrs = na;
   int lg = 0;
   while ((1 << lg) < ksplit) ++lg;
-  return cudaLaunchKernelEx(&cfg, gemv_mma_kernel<N, NB>, layers, m, x, batch, ldx, dev_status, lg, bpp);
+  const long long limit = wait_selftest ? kSelftestWaitLimit : kWaitLimit;
+  return cudaLaunchKernelEx(&cfg, gemv_mma_kernel<N, NB>, layers, m, x, batch, ldx, dev_status, lg, bpp, limit, wait_selftest ? 1 : 0);
 }
 
 template <int NB>
 static cudaError_t launch_mma_n(int N, const GemvLayers& layers, int m, const __half* x, int batch, size_t ldx,
-                                int* dev_status, cudaStream_t s, bool chained) {
-  if (N == 4) return launch_mma<4, NB>(layers, m, x, batch, ldx, dev_status, s, chained);
-  if (N == 5) return launch_mma<5, NB>(layers, m, x, batch, ldx, dev_status, s, chained);
-  return launch_mma<6, NB>(layers, m, x, batch, ldx, dev_status, s, chained);
+                                int* dev_status, cudaStream_t s, bool chained, bool selftest) {
+  if (N == 4) return launch_mma<4, NB>(layers, m, x, batch, ldx, dev_status, s, chained, selftest);
+  if (N == 5) return launch_mma<5, NB>(layers, m, x, batch, ldx, dev_status, s, chained, selftest);
+  return launch_mma<6, NB>(layers, m, x, batch, ldx, dev_status, s, chained, selftest);
 }
 
 // batch -> number of 8-row batch groups (1, 2, 4 or 8)
 static cudaError_t launch_mma_b(int batch, int N, const GemvLayers& layers, int m, const __half* x, size_t ldx,
-                                int* dev_status, cudaStream_t s, bool chained) {
-  if (batch <= 8) return launch_mma_n<1>(N, layers, m, x, batch, ldx, dev_status, s, chained);
-  if (batch <= 16) return launch_mma_n<2>(N, layers, m, x, batch, ldx, dev_status, s, chained);
-  if (batch <= 32) return launch_mma_n<4>(N, layers, m, x, batch, ldx, dev_status, s, chained);
-  return launch_mma_n<8>(N, layers, m, x, batch, ldx, dev_status, s, chained);
+                                int* dev_status, cudaStream_t s, bool chained, bool selftest = false) {
+  if (batch <= 8) return launch_mma_n<1>(N, layers, m, x, batch, ldx, dev_status, s, chained, selftest);
+  if (batch <= 16) return launch_mma_n<2>(N, layers, m, x, batch, ldx, dev_status, s, chained, selftest);
+  if (batch <= 32) return launch_mma_n<4>(N, layers, m, x, batch, ldx, dev_status, s, chained, selftest);
+  return launch_mma_n<8>(N, layers, m, x, batch, ldx, dev_status, s, chained, selftest);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -608,9 +587,8 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
   const int rt = blockIdx.x;
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
-  const int spb = (int)hdr->spb;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)hdr->ntile +
-                            (size_t)rt * nblk * resid_tile_bytes(spb);
+                            (size_t)rt * resid_rt_bytes(hdr->nrw);
 
   float acc[4][BT];
 #pragma unroll
@@ -623,6 +601,8 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
     LaneTile<N> lt;
     load_lane_tile<N>(tile, lane, lt);
     const uint64_t sal[2] = {binfo[b].salient[0], binfo[b].salient[1]};
+    const uint32_t rwo = binfo[b].rw_off;
+    const int nslot = 4 * (int)binfo[b].nrw;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       float alpha[5];
@@ -645,7 +625,7 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
             const float s1 = neg[c] ? -1.0f : 1.0f;
             if (code[c] == 3u) {
               const int q = qbase + __popc(salb & ((1u << c) - 1u));
-              const uint32_t word = q < spb ? *reinterpret_cast<const uint32_t*>(resid_rt + (size_t)b * resid_tile_bytes(spb) + resid_word_off(spb, g, q >> 2)) : 0x55555555u;
+              const uint32_t word = q < nslot ? *reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(rwo + (uint32_t)(q >> 2), g)) : 0x55555555u;
               const float s2 = resid_code(word, j, q & 3) == 0u ? 1.0f : -1.0f;
               w = __fadd_rn(s1 * alpha[3], s2 * alpha[4]);
             } else {
@@ -715,7 +695,8 @@ static cudaError_t launch_general(const uint8_t* packed, int n, int m, const __h
 }  // namespace stb
 
 static int gemv_impl(const void* packed, int n, int m, int N, const void* x, int batch, size_t ldx,
-                     void* y, stb_dtype ydt, size_t ldy, int* dev_status, void* stream, bool chained) {
+                     void* y, stb_dtype ydt, size_t ldy, int* dev_status, void* stream, bool chained,
+                     bool wait_selftest = false) {
   if (!packed || !x || !y) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
@@ -727,14 +708,14 @@ static int gemv_impl(const void* packed, int n, int m, int N, const void* x, int
   const uint8_t* p = static_cast<const uint8_t*>(packed);
   const __half* xh = static_cast<const __half*>(x);
   cudaError_t e = cudaSuccess;
-  static const bool force_general = stb::env_int("STB_GEMV_GENERAL") != 0;
-  if (N >= 4 && N <= 6 && !force_general) {
+  if (N >= 4 && N <= 6) {
     stb::GemvLayers layers = {};
     layers.packed[0] = p; layers.y[0] = y; layers.ldy[0] = ldy; layers.n[0] = n; layers.y_f16[0] = y_f16;
     layers.tile_start[0] = 0; layers.tile_start[1] = (n + stb::kTileRows - 1) / stb::kTileRows; layers.count = 1;
-    e = stb::launch_mma_b(batch, N, layers, m, xh, ldx, dev_status, s, chained);
+    e = stb::launch_mma_b(batch, N, layers, m, xh, ldx, dev_status, s, chained, wait_selftest);
     return e == cudaSuccess ? STB_OK : STB_ERR_CUDA;
   }
+  if (wait_selftest) return STB_ERR_UNSUPPORTED;
   // the general kernel takes up to 16 batch rows per launch
   for (int t0 = 0; t0 < batch && e == cudaSuccess; t0 += 16) {
     const int bt = batch - t0 < 16 ? batch - t0 : 16;
@@ -760,6 +741,12 @@ extern "C" int stb_gemv(const void* packed, int n, int m, int N, const void* x, 
   return gemv_impl(packed, n, m, N, x, batch, ldx, y, ydt, ldy, dev_status, stream, false);
 }
 
+extern "C" int stb_gemv_wait_selftest(const void* packed, int n, int m, int N, const void* x, int batch, size_t ldx,
+                                      void* y, stb_dtype ydt, size_t ldy, int* dev_status, void* stream) {
+  if (!dev_status) return STB_ERR_ARG;
+  return gemv_impl(packed, n, m, N, x, batch, ldx, y, ydt, ldy, dev_status, stream, false, true);
+}
+
 // Steps i..j-1 can share one grid when they read the same activations with the same batch, m and N
 // (4, 5 or 6) and none of them writes what another reads: same-input projections of a decoder
 // layer (q / k / v, gate / up).
@@ -770,16 +757,13 @@ static bool can_fuse(const stb_step& a, const stb_step& b) {
 
 extern "C" int stb_layer_stack(const stb_step* steps, int count, int* dev_status, void* stream) {
   if (!steps || count < 0) return STB_ERR_ARG;
-  static const bool no_pdl = stb::env_int("STB_NO_PDL") != 0;
-  static const bool no_fuse = stb::env_int("STB_NO_FUSE") != 0 || stb::env_int("STB_GEMV_GENERAL") != 0;
   int i = 0;
   while (i < count) {
     const stb_step& st = steps[i];
     int j = i + 1;
-    if (!no_fuse)
-      while (j < count && j - i < stb::kMaxFused && can_fuse(st, steps[j])) ++j;
+    while (j < count && j - i < stb::kMaxFused && can_fuse(st, steps[j])) ++j;
     // steps after the first start their weight stream while the previous step drains
-    const bool chained = i > 0 && !no_pdl;
+    const bool chained = i > 0;
     if (j - i == 1) {
       int rc = gemv_impl(st.packed, st.n, st.m, st.N, st.in, st.batch, st.ldin, st.out, st.odt, st.ldout,
                          dev_status, stream, chained);

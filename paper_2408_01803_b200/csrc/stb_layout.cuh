@@ -4,8 +4,9 @@
 //
 // The unit of the layout is a TILE: 32 output rows x one 128-column block; all tiles of a layer
 // have the same size, which depends on N alone, and follow each other in (row tile, block)
-// order after a header and a per-block table.  The residual codes of the salient columns, whose
-// size depends on the layer's salient counts, follow the tiles in the same order.  Inside a tile the work is split the way a warp-level tensor-core
+// order after a header, a per-block table and a table of residual words.  The residual codes of
+// the salient columns, whose size follows each block's own salient count, come after the tiles,
+// one run per row tile.  Inside a tile the work is split the way a warp-level tensor-core
 // instruction (m16n8k16) splits a 16 x 16 operand: lane = 4 g + t  (g = 0..7, t = 0..3) owns
 //     rows    r_j = g + 8 j      (j = 0..3) of the tile and, of each of them,
 //     groups  G_s = 4 s + t      (s = 0..3) of the block (a group = 8 columns),
@@ -45,17 +46,21 @@
 //                               are stored in the order p = 4 (r % 8) + r / 8, so that the
 //                               four rows of a lane are contiguous.
 //   sal2    32 x u16            a_sal2 per row, same row order
-// and, outside the tile, in the residual region (8 SPB bytes per tile):
-//   resid   SPB / 4 words per g residual of the block's salient columns: slot q (the q-th
-//                               salient column, ascending) of row r_j has the two-bit code
-//                               0 = +a_sal2, 2 = -a_sal2, 1 = no term (weight dropped, or
-//                               q >= number of salient columns); word q / 4 of the 8 x SPB/4
-//                               words holds rows r_0..r_3 of g at code_bit(4 j + q % 4).
-//                               SPB (slots per block) is one of 0, 4, 8, 16, 32: the smallest
-//                               that holds the largest salient count of the layer.
+// and, outside the tile, in the residual region (32 bytes per row tile and residual word):
+//   resid   a block with S salient columns owns ceil(S / 4) residual words; the words of all
+//                               blocks are numbered block after block (BlockInfo::rw_off is the
+//                               number of a block's first word, Header::nrw their total).  Word w
+//                               of a row tile is stored once per lane group g (8 x 4 bytes): slot
+//                               q (the q-th salient column of the block, ascending; q / 4 picks
+//                               the word) of row r_j has the two-bit code 0 = +a_sal2,
+//                               2 = -a_sal2, 1 = no term (weight dropped, or q >= S), at
+//                               code_bit(4 j + q % 4).  The residual word table (ResidWord, one
+//                               entry per word, after the block table) names the word's block and
+//                               its four salient columns, so that a reader can walk the words of a
+//                               run of blocks without looking at the blocks.
 //
 // Tile bytes = 512 + 192 N + 320   (50 / 56 / 62 bytes per row and block at N = 4 / 5 / 6),
-// plus 8 SPB bytes per tile (SPB / 4 per row and block) in the residual region.
+// plus ceil(S / 4) bytes per row and block in the residual region.
 #pragma once
 #include <stdint.h>
 
@@ -84,18 +89,28 @@ struct Header {          // 64 bytes at the start of the packed buffer
   uint64_t used_bytes;
   uint32_t status;       // 0 or STB_ERR_CORRUPT
   uint32_t tile_bytes;
-  uint32_t spb;          // residual slots per block: 0, 4, 8, 16 or 32
-  uint32_t pad;          // the residual region starts at tiles_offset + rt_stride * ntile
+  uint32_t nrw;          // residual words per row tile (all blocks); the residual region starts at
+                         // tiles_offset + rt_stride * ntile and holds 32 nrw bytes per row tile
+  uint32_t rwtab_offset; // byte offset of the residual word table
 };
 static_assert(sizeof(Header) == 64, "header is 64 bytes");
 
 struct BlockInfo {       // 64 bytes, one per block, right after the header
   uint64_t salient[2];   // 128-bit salient-column mask
   uint32_t nsal;         // number of salient columns
-  uint32_t pad[3];
+  uint32_t rw_off;       // number of the block's first residual word
+  uint32_t nrw;          // its residual words: ceil(nsal / 4)
+  uint32_t pad;
   uint8_t cols[32];      // the salient columns (0..127) in ascending order; unused entries 0
 };
 static_assert(sizeof(BlockInfo) == 64, "block info is 64 bytes");
+
+struct ResidWord {       // 8 bytes, one per residual word, in word order
+  uint32_t block;        // the block the word belongs to
+  uint8_t cols[4];       // its four salient columns (0..127); 0 for unused slots (their code is "no term")
+};
+static_assert(sizeof(ResidWord) == 8, "residual word entry is 8 bytes");
+constexpr int kMaxResidWords = kMaxSalient / 4;    // per block
 
 STB_HD constexpr int n_lo(int N) { return N < 4 ? N : 4; }
 STB_HD constexpr int n_hi(int N) { return N > 4 ? N - 4 : 0; }
@@ -103,13 +118,15 @@ STB_HD constexpr int sign_full_words(int N) { return (n_lo(N) >> 1) + (n_hi(N) >
 STB_HD constexpr bool sign_has_half(int N) { return (N & 1) != 0; }
 
 STB_HD constexpr uint32_t tile_bytes(int N) { return 512u + 192u * (uint32_t)N + 320u; }
-STB_HD constexpr uint32_t resid_tile_bytes(int spb) { return 8u * (uint32_t)spb; }
+// bytes of the residual codes of one row tile / of one residual word of a row tile
+STB_HD constexpr uint64_t resid_rt_bytes(uint32_t nrw) { return 32ull * nrw; }
+STB_HD constexpr uint32_t rwtab_offset(int nblk) { return (uint32_t)(sizeof(Header) + sizeof(BlockInfo) * (size_t)nblk); }
+// the table is sized for the most residual words a layer can have, so that the tiles start at an offset that
+// depends on the shape alone
 STB_HD constexpr uint32_t tiles_offset(int nblk) {
-  return (uint32_t)((sizeof(Header) + sizeof(BlockInfo) * (size_t)nblk + 255) / 256 * 256);
+  return (uint32_t)((rwtab_offset(nblk) + sizeof(ResidWord) * (size_t)kMaxResidWords * (size_t)nblk + 255) / 256 * 256);
 }
-STB_HD constexpr int spb_for(int max_nsal) {
-  return max_nsal == 0 ? 0 : (max_nsal <= 4 ? 4 : (max_nsal <= 8 ? 8 : (max_nsal <= 16 ? 16 : 32)));
-}
+STB_HD constexpr int resid_words_for(int nsal) { return (nsal + 3) >> 2; }
 // N = 6: the mask plane is ordered for the metadata of the sparse instruction (see the layout comment)
 STB_HD constexpr bool mask_pairs(int N) { return N == 6; }
 // byte offset, inside the tile, of the two bytes (row g + 16 mt, then row g + 16 mt + 8) of group 4 s + tq
@@ -150,10 +167,9 @@ STB_HD constexpr uint32_t sign_half_off(int N, int lane) {
 // scale / sal2 / resid are indexed by the permuted row position p = 4 g + j of row g + 8 j
 STB_HD constexpr uint32_t scale_off(int N, int g, int j) { return off_scale(N) + (uint32_t)(4 * g + j) * 8u; }
 STB_HD constexpr uint32_t sal2_off(int N, int g, int j) { return off_sal2(N) + (uint32_t)(4 * g + j) * 2u; }
-// byte offset of residual word wq of lane group g inside a tile's 8 SPB residual bytes
-STB_HD constexpr uint32_t resid_word_off(int spb, int g, int wq) {
-  return ((uint32_t)g * (uint32_t)(spb >> 2) + (uint32_t)wq) * 4u;
-}
+// byte offset of residual word w (numbered over the whole row tile) of lane group g inside the row tile's
+// residual codes
+STB_HD constexpr uint64_t resid_word_off(uint32_t w, int g) { return ((uint64_t)w * 8u + (uint32_t)g) * 4u; }
 
 // bit position of the two-bit code number i (0..15) of a region word
 STB_HD constexpr int code_bit(int i) {

@@ -2,7 +2,7 @@
 // tile-major streaming layout (stb_layout.cuh), plus the small host-side entry points that
 // need no kernel of their own.  Counterpart of the paper's "matrix compression" and "value
 // compression" steps (Appendix C), generalised to an 8-bit keep mask, N sign bits and 2N region
-// bits per group, five scales per row-block and a two-bit residual code per salient column.
+// bits per group, five scales per row-block and a two-bit residual code per salient column of each block.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -13,14 +13,17 @@
 namespace stb {
 
 // ---------------------------------------------------------------------------------------
-// Header + per-block table.  One CTA; the salient counts give the residual slots per block.
+// Header, per-block table and residual word table.  One CTA; every block gets ceil(S / 4)
+// residual words for its S salient columns, numbered block after block.
 __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ salient,
                               uint8_t* __restrict__ packed, int* dev_status) {
   const int nblk = m / kBlock;
   Header* hdr = reinterpret_cast<Header*>(packed);
   BlockInfo* bi = reinterpret_cast<BlockInfo*>(packed + sizeof(Header));
-  __shared__ int bad, maxsal;
-  if (threadIdx.x == 0) { bad = 0; maxsal = 0; }
+  ResidWord* rwt = reinterpret_cast<ResidWord*>(packed + rwtab_offset(nblk));
+  __shared__ int bad;
+  __shared__ uint32_t total;
+  if (threadIdx.x == 0) bad = 0;
   __syncthreads();
   for (int b = threadIdx.x; b < nblk; b += blockDim.x) {
     uint64_t lo = salient[2 * b], hi = salient[2 * b + 1];
@@ -29,7 +32,8 @@ __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ 
     bi[b].salient[0] = lo;
     bi[b].salient[1] = hi;
     bi[b].nsal = (uint32_t)ns;
-    bi[b].pad[0] = bi[b].pad[1] = bi[b].pad[2] = 0;
+    bi[b].nrw = (uint32_t)resid_words_for(ns);
+    bi[b].pad = 0;
     int q = 0;
     for (int h = 0; h < 2; ++h) {
       uint64_t mk = h ? hi : lo;
@@ -39,26 +43,36 @@ __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ 
       }
     }
     for (; q < kMaxSalient; ++q) bi[b].cols[q] = 0;
-    atomicMax(&maxsal, ns);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
+    uint32_t off = 0;
+    for (int b = 0; b < nblk; ++b) { bi[b].rw_off = off; off += bi[b].nrw; }
+    total = off;
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < nblk; b += blockDim.x)
+    for (uint32_t wq = 0; wq < bi[b].nrw; ++wq) {
+      ResidWord e;
+      e.block = (uint32_t)b;
+      for (int k = 0; k < 4; ++k) e.cols[k] = bi[b].cols[4 * wq + k];
+      rwt[bi[b].rw_off + wq] = e;
+    }
+  if (threadIdx.x == 0) {
     const int ntile = (n + kTileRows - 1) / kTileRows;
-    const int spb = spb_for(maxsal);
     const uint32_t tb = tile_bytes(N);
-    const uint64_t tiles = (uint64_t)nblk * (uint64_t)ntile;
     hdr->magic = kMagic;
-    hdr->version = 2;
+    hdr->version = 3;
     hdr->n = n; hdr->m = m; hdr->N = N;
     hdr->nblk = nblk;
     hdr->ntile = ntile;
     hdr->tiles_offset = tiles_offset(nblk);
     hdr->rt_stride = (uint64_t)tb * (uint64_t)nblk;
-    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + ((uint64_t)tb + resid_tile_bytes(spb)) * tiles;
+    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + (hdr->rt_stride + resid_rt_bytes(total)) * (uint64_t)ntile;
     hdr->status = bad ? (uint32_t)STB_ERR_CORRUPT : 0u;
     hdr->tile_bytes = tb;
-    hdr->spb = (uint32_t)spb;
-    hdr->pad = 0;
+    hdr->nrw = total;
+    hdr->rwtab_offset = rwtab_offset(nblk);
     if (bad && dev_status) *dev_status = STB_ERR_CORRUPT;
   }
 }
@@ -103,10 +117,10 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
   Header* hdr = reinterpret_cast<Header*>(packed);
   const BlockInfo* bi = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header)) + b;
   const uint64_t sal_lo = bi->salient[0], sal_hi = bi->salient[1];
-  const int nsal = (int)bi->nsal, spb = (int)hdr->spb;
+  const int nsal = (int)bi->nsal, nrw_b = (int)bi->nrw;
   uint8_t* tile = packed + hdr->tiles_offset + ((size_t)rt * nblk + b) * (size_t)hdr->tile_bytes;
   uint8_t* resid = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                   ((size_t)rt * nblk + b) * (size_t)resid_tile_bytes(spb);
+                   (size_t)rt * resid_rt_bytes(hdr->nrw) + resid_word_off(bi->rw_off, 0);
 
   // ---- phase 1: lane = row ----
   // rows past n: nothing kept, all signs "+", zero scales
@@ -170,7 +184,7 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
     int q = 0;
     uint64_t mk = sal_lo;
     int base = 0;
-    for (int wq = 0; wq < (spb >> 2); ++wq) {
+    for (int wq = 0; wq < nrw_b; ++wq) {
       uint32_t word = 0;
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
@@ -189,7 +203,7 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
       }
       word |= __shfl_xor_sync(0xFFFFFFFFu, word, 8);
       word |= __shfl_xor_sync(0xFFFFFFFFu, word, 16);
-      if (lane < 8) *reinterpret_cast<uint32_t*>(resid + resid_word_off(spb, lane, wq)) = word;
+      if (lane < 8) *reinterpret_cast<uint32_t*>(resid + resid_word_off((uint32_t)wq, lane)) = word;
     }
   }
   __syncwarp();
@@ -253,7 +267,7 @@ extern "C" int stb_pack_size(int n, int m, int N, size_t* bytes) {
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
   const size_t nblk = (size_t)m / stb::kBlock, ntile = ((size_t)n + 31) / 32;
-  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * (size_t)(stb::tile_bytes(N) + stb::resid_tile_bytes(stb::kMaxSalient));
+  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * ((size_t)stb::tile_bytes(N) + (size_t)stb::resid_rt_bytes(stb::kMaxResidWords));
   return STB_OK;
 }
 
@@ -297,7 +311,7 @@ extern "C" int stb_packed_info(const void* packed, stb_info* info, void* stream)
   info->n = h.n; info->m = h.m; info->N = h.N;
   info->status = (int)h.status;
   info->used_bytes = h.used_bytes;
-  info->stream_bytes = (h.rt_stride + (uint64_t)stb::resid_tile_bytes((int)h.spb) * (uint64_t)h.nblk) * (uint64_t)h.ntile;
+  info->stream_bytes = (h.rt_stride + stb::resid_rt_bytes(h.nrw)) * (uint64_t)h.ntile;
   return STB_OK;
 }
 

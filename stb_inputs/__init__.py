@@ -79,14 +79,15 @@ def _mask_table(N: int) -> np.ndarray:
 
 
 def logical_layer(n: int, m: int, N: int, seed: int, max_salient: int = 3,
-                  region_p=(0.68, 0.26, 0.06)) -> dict:
+                  region_p=(0.68, 0.26, 0.06), salient_counts=None) -> dict:
     """Draw a logical structured-binary layer directly (no quantizer).
 
     Returns a dict of C-contiguous numpy arrays in the logical format:
       keep u8[n][m/8], sign u8[n][m/8], region u16[n][m/8], sign2 u32[n][m/128],
       salient u64[m/128][2], scale u16[n][m/128][5] (fp16 bits).
     Structure: every group of 8 columns keeps exactly N (uniform over the C(8,N) masks);
-    1..max_salient salient columns per 128-column block; non-salient kept weights get
+    1..max_salient salient columns per 128-column block (or salient_counts[b % len] of them in block b,
+    when that list is given); non-salient kept weights get
     region 0/1/2 (dense/intermediate/sparse) with probabilities region_p; kept weights in
     salient columns get region 3 and a residual sign; scales are positive fp16.
     """
@@ -101,6 +102,8 @@ def logical_layer(n: int, m: int, N: int, seed: int, max_salient: int = 3,
     salflag = np.zeros((nblk, BLOCK), dtype=bool)
     for b in range(nblk):
         k = 0 if max_salient == 0 else int(g.integers(1, max_salient + 1))
+        if salient_counts is not None:
+            k = int(salient_counts[b % len(salient_counts)])
         salflag[b, g.permutation(BLOCK)[:k]] = True
     sal_bits = np.packbits(salflag, axis=1, bitorder="little")         # [nblk][16] bytes
     salient = np.ascontiguousarray(sal_bits).view(np.uint64).reshape(nblk, 2).copy()
@@ -144,3 +147,38 @@ SHAPES_13B = {"q": (5120, 5120), "k": (5120, 5120), "v": (5120, 5120), "o": (512
               "gate": (13824, 5120), "up": (13824, 5120), "down": (5120, 13824)}
 SHAPES_70B = {"q": (8192, 8192), "k": (1024, 8192), "v": (1024, 8192), "o": (8192, 8192),
               "gate": (28672, 8192), "up": (28672, 8192), "down": (8192, 28672)}
+
+
+# Which dense layer (shape, N, seed) stands behind every named linear of the five workloads.  The seed
+# feeds dense_weight / calib_norms; item numbers: workload 2: gate, up, down = 0, 1, 2; workloads 3 and 4:
+# q, k, v, o, gate, up, down = 0..6; workload 5: one layer per (shape, N) family, item = 3 * shape + (N - 4)
+# with shape 0 = 4096 x 4096, 1 = 11008 x 4096, 2 = 4096 x 11008 (the 32 decoder layers reuse the family's
+# layer at distinct addresses: the kernels' work does not depend on which layer of a family it is).
+_ORDER = ("q", "k", "v", "o", "gate", "up", "down")
+
+
+def workload_layer(config: int, name: str, N: int = 0):
+    """(n, m, N, seed) of linear `name` of workload `config` (1..5)."""
+    if config == 1:
+        return 4096, 4096, 4, seed_for(1, 0)
+    if config == 2:
+        n, m = SHAPES_7B[name]
+        return n, m, 6, seed_for(2, ("gate", "up", "down").index(name))
+    if config == 3:
+        n, m = SHAPES_13B[name]
+        return n, m, 5, seed_for(3, _ORDER.index(name))
+    if config == 4:
+        n, m = SHAPES_70B[name]
+        return n, m, 4, seed_for(4, _ORDER.index(name))
+    if config == 5:
+        n, m = SHAPES_7B[name]
+        shape = {(4096, 4096): 0, (11008, 4096): 1, (4096, 11008): 2}[(n, m)]
+        assert N in (4, 5, 6)
+        return n, m, N, seed_for(5, 3 * shape + (N - 4))
+    raise ValueError(config)
+
+
+def stack_N_per_layer(layers: int = 32):
+    """Workload 5: N of each decoder layer, drawn from {4, 5, 6} (seeded)."""
+    rng = np.random.default_rng(seed_for(5, 15))
+    return [int(v) for v in rng.choice([4, 5, 6], size=layers)]

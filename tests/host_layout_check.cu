@@ -54,7 +54,8 @@ static int check(int trials, int spb) {
       for (int q = 0; q < 32; ++q) rcode[r][q] = q < spb ? (uint8_t)(rnd() % 3) : 1;
     }
     const uint32_t tb = tile_bytes(N);
-    std::vector<uint8_t> tile(tb + 64, 0), resid(resid_tile_bytes(spb) + 64, 0);
+    const uint32_t w0 = 3;     // the block's first residual word inside the row tile's residual codes
+    std::vector<uint8_t> tile(tb + 64, 0), resid(resid_rt_bytes(w0 + spb / 4) + 64, 0);
     auto put32 = [&](uint32_t off, uint32_t v) { std::memcpy(&tile[off], &v, 4); };
     auto or32 = [&](uint32_t off, uint32_t v) { uint32_t o; std::memcpy(&o, &tile[off], 4); o |= v; std::memcpy(&tile[off], &o, 4); };
     for (int lane = 0; lane < 32; ++lane) {
@@ -90,13 +91,13 @@ static int check(int trials, int spb) {
       std::memcpy(&tile[sal2_off(N, g, j)], &scale[r][4], 2);
       for (int q = 0; q < spb; ++q) {
         uint32_t o;
-        std::memcpy(&o, &resid[resid_word_off(spb, g, q >> 2)], 4);
+        std::memcpy(&o, &resid[resid_word_off(w0 + (uint32_t)(q >> 2), g)], 4);
         o |= (uint32_t)rcode[r][q] << code_bit(4 * j + (q & 3));
-        std::memcpy(&resid[resid_word_off(spb, g, q >> 2)], &o, 4);
+        std::memcpy(&resid[resid_word_off(w0 + (uint32_t)(q >> 2), g)], &o, 4);
       }
     }
     // every offset must stay inside the tile
-    if (sal2_off(N, 7, 3) + 2u != tb || resid_word_off(spb ? spb : 4, 7, (spb ? spb : 4) / 4 - 1) + 4u != resid_tile_bytes(spb ? spb : 4)) {
+    if (sal2_off(N, 7, 3) + 2u != tb || resid_word_off(w0 + 8u - 1u, 7) + 4u != resid_rt_bytes(w0 + 8u) || resid_words_for(5) != 2 || resid_words_for(32) != kMaxResidWords) {
       ++errors; std::printf("N=%d tile size mismatch\n", N);
     }
 
@@ -128,7 +129,7 @@ static int check(int trials, int spb) {
         if (sal2_bits<N>(lt, j) != scale[r][4]) { if (++errors < 10) std::printf("sal2 N=%d\n", N); }
         for (int q = 0; q < spb; ++q) {
           uint32_t word;
-          std::memcpy(&word, &resid[resid_word_off(spb, g, q >> 2)], 4);
+          std::memcpy(&word, &resid[resid_word_off(w0 + (uint32_t)(q >> 2), g)], 4);
           if (resid_code(word, j, q & 3) != rcode[r][q]) { if (++errors < 10) std::printf("resid code N=%d\n", N); }
           if (((resid_selector(word, j) >> (4 * (q & 3))) & 0xFu) != rcode[r][q]) { if (++errors < 10) std::printf("resid selector N=%d\n", N); }
         }

@@ -33,7 +33,7 @@ def test_pack_size_formula_and_errors(stb):
     # (two bits for each of up to 32 salient columns)
     for N, per in ((4, 50), (5, 56), (6, 62)):
         n, m = 4096, 4096
-        hdr = (64 + 64 * (m // 128) + 255) // 256 * 256
+        hdr = (64 + 128 * (m // 128) + 255) // 256 * 256       # header, block table, residual word table
         assert stb.pack_size(n, m, N) == hdr + (n // 32) * (m // 128) * 32 * (per + 8)
     assert stb.pack_size(33, 128, 4) == 256 + 2 * 32 * 58      # ragged rows pad to a tile of 32
     for args, code in (((0, 128, 4), stb.STB_ERR_SHAPE), ((8, 100, 4), stb.STB_ERR_SHAPE),
