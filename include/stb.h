@@ -176,6 +176,36 @@ int stb_gemm_noalloc(const void *packed, int n, int m, int N, const void *X, int
  * N:M assignment, Section 3.3).  steps is a HOST array.  Launches only. */
 int stb_layer_stack(const stb_step *steps, int count, int *dev_status, void *stream);
 
+/* stb_layer_stack as ONE resident kernel (Section 3.3: per-layer N:M; Appendix C.2: decoding is
+ * memory-bound, so the weight stream must not stop between layers).  One CTA per SM stays on the
+ * machine for the whole list: consecutive steps that read the same activations (q / k / v,
+ * gate / up) are dealt to the SMs together in equal shares of 32 x 128 tiles, every warp keeps
+ * streaming packed weights across layer boundaries, and a layer that reads an earlier layer's
+ * output starts its arithmetic when a counter in the workspace says that every earlier step
+ * is complete (bounded poll; STB_ERR_TIMEOUT through *dev_status).  Results are reproducible:
+ * every sum has a fixed order.  Steps must have N = 4, 5 or 6 and batch <= 8, else
+ * STB_ERR_UNSUPPORTED (use stb_layer_stack).  Lists of more than 64 groups of same-input steps
+ * run as several launches.
+ * ws: caller-owned DEVICE workspace of stb_layer_stack_resident_workspace bytes, 256-byte
+ * aligned, ZEROED by the caller before its first use; every call leaves it zeroed again, also
+ * after a wait that ran out.  Calls that share a workspace must not overlap on the GPU.
+ * The launch is cooperative: it fails with STB_ERR_CUDA when the GPU cannot hold one 512-thread
+ * CTA per SM at once. */
+int stb_layer_stack_resident_workspace(const stb_step *steps, int count, size_t *bytes);
+int stb_layer_stack_resident(const stb_step *steps, int count, void *ws, size_t ws_bytes,
+                             int *dev_status, void *stream);
+
+/* stb_layer_stack_host through the resident kernel (same copies before and after). */
+int stb_layer_stack_resident_host(const stb_step *steps, int count, void *ws, size_t ws_bytes,
+                                  const void *in_host, size_t in_bytes, void *out_host,
+                                  size_t out_bytes, int *dev_status, void *stream);
+
+/* Self-test of the resident kernel's bounded waits, in the manner of stb_gemv_wait_selftest:
+ * weight copies off, wait limit about 50 microseconds.  *dev_status (required) becomes
+ * STB_ERR_TIMEOUT, every CTA leaves, the workspace is zero again; outputs are meaningless. */
+int stb_layer_stack_resident_wait_selftest(const stb_step *steps, int count, void *ws,
+                                           size_t ws_bytes, int *dev_status, void *stream);
+
 /* stb_layer_stack for a caller whose activations live in HOST memory: copies in_bytes from
  * in_host (HOST, pinned for the copy to be asynchronous) into steps[0].in, runs the steps,
  * then copies out_bytes from steps[count-1].out to out_host (HOST).  The device buffers named

@@ -9,6 +9,7 @@ from __future__ import annotations
 
 import hashlib
 import os
+import sys
 import tempfile
 import time
 
@@ -57,7 +58,7 @@ def quantized_layer(n: int, m: int, N: int, seed: int, use_cache: bool = True, v
         os.replace(tmp, path)
     d.update(n=n, m=m, N=N)
     if verbose:
-        print("quantized %dx%d at %d:8 (seed %x) in %.1f s" % (n, m, N, seed, time.time() - t0), flush=True)
+        print("quantized %dx%d at %d:8 (seed %x) in %.1f s" % (n, m, N, seed, time.time() - t0), file=sys.stderr, flush=True)
     return d
 
 

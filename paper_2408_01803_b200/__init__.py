@@ -21,7 +21,9 @@ STB_ERR_UNSUPPORTED, STB_ERR_CORRUPT, STB_ERR_TIMEOUT, STB_ERR_CUDA = 5, 6, 7, 8
 STB_F16, STB_BF16, STB_F32 = 0, 1, 2
 
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
-           "stb_gemm_workspace", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host", "stb_status_str"]
+           "stb_gemm_workspace", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
+           "stb_layer_stack_resident_workspace", "stb_layer_stack_resident", "stb_layer_stack_resident_host",
+           "stb_layer_stack_resident_wait_selftest", "stb_status_str"]
 
 
 class StbError(RuntimeError):
@@ -64,6 +66,10 @@ def _load():
     lib.stb_gemm_noalloc.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_layer_stack.argtypes = [p(_Step), i, v, v]
     lib.stb_layer_stack_host.argtypes = [p(_Step), i, v, z, v, z, v, v]
+    lib.stb_layer_stack_resident_workspace.argtypes = [p(_Step), i, p(z)]
+    lib.stb_layer_stack_resident.argtypes = [p(_Step), i, v, z, v, v]
+    lib.stb_layer_stack_resident_wait_selftest.argtypes = [p(_Step), i, v, z, v, v]
+    lib.stb_layer_stack_resident_host.argtypes = [p(_Step), i, v, z, v, z, v, z, v, v]
     lib.stb_status_str.argtypes = [i]
     lib.stb_status_str.restype = C.c_char_p
     for name in EXPORTS:
@@ -254,3 +260,28 @@ def layer_stack_host(marshalled, x_host, y_host, dev_status=None, stream=None):
                                      x_host.numel() * x_host.element_size(), C.c_void_p(y_host.data_ptr()),
                                      y_host.numel() * y_host.element_size(), _ptr(dev_status), _stream(stream)),
            "stb_layer_stack_host")
+
+
+def resident_workspace(marshalled, device="cuda"):
+    """A zeroed workspace (torch.uint8 CUDA tensor) of the size stb_layer_stack_resident wants for these steps."""
+    import torch
+    out = C.c_size_t()
+    _check(_lib.stb_layer_stack_resident_workspace(marshalled, len(marshalled), C.byref(out)),
+           "stb_layer_stack_resident_workspace")
+    return torch.zeros(max(out.value, 256), dtype=torch.uint8, device=device)
+
+
+def layer_stack_resident(steps, ws, dev_status=None, stream=None, marshalled=None, selftest=False):
+    """stb_layer_stack_resident over a list of (PackedLayer, x, out) triples (or a pre-marshalled array);
+    ws from resident_workspace().  selftest=True runs the wait self-test instead."""
+    arr = marshalled if marshalled is not None else make_steps(steps)
+    fn = _lib.stb_layer_stack_resident_wait_selftest if selftest else _lib.stb_layer_stack_resident
+    _check(fn(arr, len(arr), _ptr(ws), ws.numel(), _ptr(dev_status), _stream(stream)), "stb_layer_stack_resident")
+
+
+def layer_stack_resident_host(marshalled, ws, x_host, y_host, dev_status=None, stream=None):
+    """stb_layer_stack_resident_host: x_host / y_host are pinned CPU tensors."""
+    _check(_lib.stb_layer_stack_resident_host(marshalled, len(marshalled), _ptr(ws), ws.numel(),
+                                              C.c_void_p(x_host.data_ptr()), x_host.numel() * x_host.element_size(),
+                                              C.c_void_p(y_host.data_ptr()), y_host.numel() * y_host.element_size(),
+                                              _ptr(dev_status), _stream(stream)), "stb_layer_stack_resident_host")

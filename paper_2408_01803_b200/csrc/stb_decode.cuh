@@ -44,7 +44,6 @@ struct LaneTile {
   uint32_t S[kFull > 0 ? kFull : 1];    // full sign words (low part, then high part)
   uint32_t half;                        // shared half sign word, already in lower-lane form
   uint32_t A[4], B[4];                  // per row j: low / high bytes of the four main scales
-  uint32_t sal2[2];                     // a_sal2 of rows 0,1 / 2,3 (two fp16 per word)
 };
 
 template <int NW>
@@ -96,18 +95,20 @@ STB_HD void load_lane_tile(const uint8_t* tile, int lane, LaneTile<N>& t, bool r
   const uint4 s1 = *reinterpret_cast<const uint4*>(tile + scale_off(N, g, 2));
   t.A[0] = s0.x; t.B[0] = s0.y; t.A[1] = s0.z; t.B[1] = s0.w;
   t.A[2] = s1.x; t.B[2] = s1.y; t.A[3] = s1.z; t.B[3] = s1.w;
-  const uint2 a2 = *reinterpret_cast<const uint2*>(tile + sal2_off(N, g, 0));
-  t.sal2[0] = a2.x; t.sal2[1] = a2.y;
 }
 
-// fp16 bit pattern of main scale q (0..3) / of a_sal2 of row j
+// fp16 bit pattern of main scale q (0..3) of row j
 template <int N>
 STB_HD uint32_t scale_bits(const LaneTile<N>& t, int j, int q) {
   return ((t.A[j] >> (8 * q)) & 0xFFu) | (((t.B[j] >> (8 * q)) & 0xFFu) << 8);
 }
-template <int N>
-STB_HD uint32_t sal2_bits(const LaneTile<N>& t, int j) {
-  return (t.sal2[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+// fp16 bit pattern of a_sal2 of row g + 8 j; `record` = the block's record in the row tile's residual stream
+STB_HD uint32_t sal2_bits(const uint8_t* record, int g, int j) {
+  return *reinterpret_cast<const uint16_t*>(record + resid_a2_off(g, j));
+}
+// residual word wq (0..7) of the block, as stored for lane group g
+STB_HD uint32_t resid_word(const uint8_t* record, uint32_t wq, int g) {
+  return *reinterpret_cast<const uint32_t*>(record + resid_code_off(wq, g));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -300,7 +301,6 @@ struct RowWords {
   uint32_t Rlo, Rhi;        // region words: ranks 0..3 of the row's four slots / the word holding its ranks 4..
   uint32_t Slo, Shi;        // sign words: the one holding ranks 0..3 / ranks 4.. (N = 5: the half word, lower-lane form)
   uint32_t A, B;            // low / high bytes of the four main scales
-  uint32_t sal2;            // a_sal2 (16 bits)
 };
 template <int N>
 STB_HD void load_row_words(const uint8_t* tile, int lane, int j, RowWords& w) {
@@ -329,7 +329,6 @@ STB_HD void load_row_words(const uint8_t* tile, int lane, int j, RowWords& w) {
   }
   const uint2 sc = *reinterpret_cast<const uint2*>(tile + scale_off(N, g, j));
   w.A = sc.x; w.B = sc.y;
-  w.sal2 = *reinterpret_cast<const uint16_t*>(tile + sal2_off(N, g, j));
 }
 
 template <int N>

@@ -31,8 +31,8 @@ dequant_kernel(const uint8_t* __restrict__ packed, int n, int m, T* __restrict__
   const BlockInfo* bi = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header)) + b;
   const uint8_t* tile = packed + hdr->tiles_offset + ((size_t)rt * nblk + b) * (size_t)hdr->tile_bytes;
   const int nslot = 4 * (int)bi->nrw;
-  const uint8_t* resid = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                         (size_t)rt * resid_rt_bytes(hdr->nrw) + resid_word_off(bi->rw_off, 0);
+  const uint8_t* record = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
+                          (size_t)rt * resid_rt_bytes(nblk, hdr->nrw) + resid_block_off(b, bi->rw_off);
   LaneTile<N> lt;
   load_lane_tile<N>(tile, lane, lt);
   const uint64_t sal[2] = {bi->salient[0], bi->salient[1]};
@@ -49,7 +49,7 @@ dequant_kernel(const uint8_t* __restrict__ packed, int n, int m, T* __restrict__
     qbase += __popcll(sal[grp >> 3] & ((1ull << (8 * (grp & 7))) - 1ull));
     float alpha[5];
     for (int q = 0; q < 4; ++q) alpha[q] = __half2float(__ushort_as_half((unsigned short)scale_bits<N>(lt, j, q)));
-    alpha[4] = __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(lt, j)));
+    alpha[4] = __half2float(__ushort_as_half((unsigned short)sal2_bits(record, g, j)));
     T* dst = W + (size_t)row * ldw + (size_t)b * kBlock + grp * 8;
     for (int c = 0; c < 8; ++c) {
       float v = 0.0f;
@@ -57,7 +57,7 @@ dequant_kernel(const uint8_t* __restrict__ packed, int n, int m, T* __restrict__
         const float s1 = neg[c] ? -1.0f : 1.0f;
         if (code[c] == 3u) {
           const int q = qbase + __popc(salb & ((1u << c) - 1u));
-          const uint32_t word = q < nslot ? *reinterpret_cast<const uint32_t*>(resid + resid_word_off((uint32_t)(q >> 2), g)) : 0x55555555u;
+          const uint32_t word = q < nslot ? resid_word(record, (uint32_t)(q >> 2), g) : 0x55555555u;
           const uint32_t rc = resid_code(word, j, q & 3);
           const float s2 = rc == 0u ? 1.0f : -1.0f;
           v = __fadd_rn(s1 * alpha[3], s2 * alpha[4]);

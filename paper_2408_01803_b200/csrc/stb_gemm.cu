@@ -152,21 +152,22 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                            (size_t)rtile * resid_rt_bytes(hdr->nrw);
+                            (size_t)rtile * resid_rt_bytes(nblk, hdr->nrw);
   constexpr uint32_t tbytes = tile_bytes(N);
   RowWords cur = {}, nxt = {};
   // salient metadata of a block, fetched one block ahead like the row's words: the count, and for the
   // lane's slots t, t + 4 (slots beyond 8 are fetched on demand) the column bytes and residual words
-  struct Sal { int nsal; uint32_t rwo; uint32_t cw[2], rw[2]; };
+  struct Sal { int nsal; const uint8_t* rec; uint32_t a2; uint32_t cw[2], rw[2]; };
   auto load_sal = [&](int b, Sal& z) {
     z.nsal = (int)__ldg(&binfo[b].nsal);
-    z.rwo = __ldg(&binfo[b].rw_off);
+    z.rec = resid_rt + resid_block_off(b, __ldg(&binfo[b].rw_off));       // the block's record of the residual stream
+    z.a2 = __ldg(reinterpret_cast<const uint16_t*>(z.rec + resid_a2_off(g, j)));
     z.cw[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols));
     z.cw[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + 1);
-    z.rw[0] = z.nsal > 0 ? __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(z.rwo, g))) : 0x55555555u;
-    z.rw[1] = z.nsal > 4 ? __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(z.rwo + 1u, g))) : 0x55555555u;
+    z.rw[0] = z.nsal > 0 ? __ldg(reinterpret_cast<const uint32_t*>(z.rec + resid_code_off(0u, g))) : 0x55555555u;
+    z.rw[1] = z.nsal > 4 ? __ldg(reinterpret_cast<const uint32_t*>(z.rec + resid_code_off(1u, g))) : 0x55555555u;
   };
-  Sal csal = {0, 0u, {0, 0}, {0, 0}}, nsalv = {0, 0u, {0, 0}, {0, 0}};
+  Sal csal = {0, nullptr, 0u, {0, 0}, {0, 0}}, nsalv = {0, nullptr, 0u, {0, 0}, {0, 0}};
   if (live && b0 < b1) { load_row_words<N>(rtbase + (size_t)b0 * tbytes, lane, j, cur); load_sal(b0, csal); }
   bool ok = true;
   for (int b = b0; b < b1 && ok; ++b) {
@@ -183,7 +184,7 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
         B16 |= (v >> 8) << (8 * c);
         if (c == 3) a1f = __half2float(__ushort_as_half((unsigned short)h16));
       }
-      a2f = __half2float(__ushort_as_half((unsigned short)cur.sal2));
+      a2f = __half2float(__ushort_as_half((unsigned short)csal.a2));
     }
     OneRow<N> row;
     row.init(cur, j, A16, B16);
@@ -226,7 +227,7 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
             const int sq = p;
             c = binfo[b].cols[sq];
             const uint32_t word = sq < 8 ? csal.rw[1] :
-                __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(csal.rwo + (uint32_t)(sq >> 2), g)));
+                __ldg(reinterpret_cast<const uint32_t*>(csal.rec + resid_code_off((uint32_t)(sq >> 2), g)));
             rc = resid_code(word, j, sq & 3);
           }
           if ((c >> 6) != h || rc == 1u) continue;

@@ -119,7 +119,7 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
   constexpr uint32_t tbytes = tile_bytes(N);
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)hdr->ntile +
-                            (size_t)rt * resid_rt_bytes(hdr->nrw);
+                            (size_t)rt * resid_rt_bytes(nblk, hdr->nrw);
   const uint32_t image_bytes = gemv_image_bytes(N, NB, batch, bpp);
   const GemvSmem L = gemv_smem(N, warps, ksplit, NB, image_bytes);
 
@@ -218,9 +218,11 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
     const uint32_t wi = rw0 + 4u * step + (uint32_t)t;
     if (wi < rw1) {
       const uint2 e = __ldg(reinterpret_cast<const uint2*>(rwt + wi));
-      w.block = e.x; w.cols = e.y;
-      w.rw = __ldg(reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(wi, g)));
-      w.a2 = __ldg(reinterpret_cast<const uint2*>(rtbase + (size_t)e.x * tbytes + sal2_off(N, g, 0)));
+      w.block = e.x >> 3; w.cols = e.y;
+      // the word's block record in the residual stream: a_sal2 of the lane's four rows, then the block's words
+      const uint8_t* rec = resid_rt + resid_block_off((int)w.block, wi - (e.x & 7u));
+      w.a2 = __ldg(reinterpret_cast<const uint2*>(rec + resid_a2_off(g, 0)));
+      w.rw = __ldg(reinterpret_cast<const uint32_t*>(rec + resid_code_off(e.x & 7u, g)));
     }
   };
   ResidWords rfirst;
@@ -588,7 +590,7 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
   const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rt * hdr->rt_stride;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)hdr->ntile +
-                            (size_t)rt * resid_rt_bytes(hdr->nrw);
+                            (size_t)rt * resid_rt_bytes(nblk, hdr->nrw);
 
   float acc[4][BT];
 #pragma unroll
@@ -601,14 +603,14 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
     LaneTile<N> lt;
     load_lane_tile<N>(tile, lane, lt);
     const uint64_t sal[2] = {binfo[b].salient[0], binfo[b].salient[1]};
-    const uint32_t rwo = binfo[b].rw_off;
+    const uint8_t* record = resid_rt + resid_block_off(b, binfo[b].rw_off);
     const int nslot = 4 * (int)binfo[b].nrw;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       float alpha[5];
 #pragma unroll
       for (int q = 0; q < 4; ++q) alpha[q] = __half2float(__ushort_as_half((unsigned short)scale_bits<N>(lt, j, q)));
-      alpha[4] = __half2float(__ushort_as_half((unsigned short)sal2_bits<N>(lt, j)));
+      alpha[4] = __half2float(__ushort_as_half((unsigned short)sal2_bits(record, g, j)));
 #pragma unroll 1
       for (int s = 0; s < 4; ++s) {
         const int grp = 4 * s + t;
@@ -625,7 +627,7 @@ gemv_general_kernel(const uint8_t* __restrict__ packed, int n, int m, const __ha
             const float s1 = neg[c] ? -1.0f : 1.0f;
             if (code[c] == 3u) {
               const int q = qbase + __popc(salb & ((1u << c) - 1u));
-              const uint32_t word = q < nslot ? *reinterpret_cast<const uint32_t*>(resid_rt + resid_word_off(rwo + (uint32_t)(q >> 2), g)) : 0x55555555u;
+              const uint32_t word = q < nslot ? resid_word(record, (uint32_t)(q >> 2), g) : 0x55555555u;
               const float s2 = resid_code(word, j, q & 3) == 0u ? 1.0f : -1.0f;
               w = __fadd_rn(s1 * alpha[3], s2 * alpha[4]);
             } else {

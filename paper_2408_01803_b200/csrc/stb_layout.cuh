@@ -4,9 +4,9 @@
 //
 // The unit of the layout is a TILE: 32 output rows x one 128-column block; all tiles of a layer
 // have the same size, which depends on N alone, and follow each other in (row tile, block)
-// order after a header, a per-block table and a table of residual words.  The residual codes of
-// the salient columns, whose size follows each block's own salient count, come after the tiles,
-// one run per row tile.  Inside a tile the work is split the way a warp-level tensor-core
+// order after a header, a per-block table and a table of residual words.  The residual stream
+// (the second scale of the salient columns and their residual codes, whose size follows each
+// block's own salient count) comes after the tiles, one run per row tile.  Inside a tile the work is split the way a warp-level tensor-core
 // instruction (m16n8k16) splits a 16 x 16 operand: lane = 4 g + t  (g = 0..7, t = 0..3) owns
 //     rows    r_j = g + 8 j      (j = 0..3) of the tile and, of each of them,
 //     groups  G_s = 4 s + t      (s = 0..3) of the block (a group = 8 columns),
@@ -45,22 +45,24 @@
 //                               a_inter, a_sparse, a_sal1; word B = their high bytes.  Rows
 //                               are stored in the order p = 4 (r % 8) + r / 8, so that the
 //                               four rows of a lane are contiguous.
-//   sal2    32 x u16            a_sal2 per row, same row order
-// and, outside the tile, in the residual region (32 bytes per row tile and residual word):
-//   resid   a block with S salient columns owns ceil(S / 4) residual words; the words of all
-//                               blocks are numbered block after block (BlockInfo::rw_off is the
-//                               number of a block's first word, Header::nrw their total).  Word w
-//                               of a row tile is stored once per lane group g (8 x 4 bytes): slot
-//                               q (the q-th salient column of the block, ascending; q / 4 picks
-//                               the word) of row r_j has the two-bit code 0 = +a_sal2,
+// and, outside the tile, in the residual stream of the row tile, one record per block, block after block:
+//   sal2    32 x u16            a_sal2 per row, rows in the order p = 4 (r % 8) + r / 8 like the scales
+//   resid   ceil(S / 4) words   for the block's S salient columns, each word stored once per lane group g
+//                               (8 x 4 bytes): slot q (the q-th salient column of the block, ascending;
+//                               q / 4 picks the word) of row r_j has the two-bit code 0 = +a_sal2,
 //                               2 = -a_sal2, 1 = no term (weight dropped, or q >= S), at
-//                               code_bit(4 j + q % 4).  The residual word table (ResidWord, one
-//                               entry per word, after the block table) names the word's block and
-//                               its four salient columns, so that a reader can walk the words of a
-//                               run of blocks without looking at the blocks.
+//                               code_bit(4 j + q % 4).
+//                               The words of all blocks are numbered block after block
+//                               (BlockInfo::rw_off = number of a block's first word, Header::nrw
+//                               their total), so block b's record starts 64 b + 32 rw_off bytes into
+//                               the row tile's stream and the records of a run of blocks are one
+//                               contiguous piece.  The residual word table (ResidWord, one entry per
+//                               word, after the block table) names the word's block, its place in
+//                               the block and its four salient columns, so that a reader can walk
+//                               the words of a run of blocks without looking at the blocks.
 //
-// Tile bytes = 512 + 192 N + 320   (50 / 56 / 62 bytes per row and block at N = 4 / 5 / 6),
-// plus ceil(S / 4) bytes per row and block in the residual region.
+// Tile bytes = 512 + 192 N + 256; with the record, 26 + 6 N bytes per row and block (50 / 56 / 62 at
+// N = 4 / 5 / 6) plus ceil(S / 4) bytes per row for the block's S salient columns.
 #pragma once
 #include <stdint.h>
 
@@ -89,8 +91,8 @@ struct Header {          // 64 bytes at the start of the packed buffer
   uint64_t used_bytes;
   uint32_t status;       // 0 or STB_ERR_CORRUPT
   uint32_t tile_bytes;
-  uint32_t nrw;          // residual words per row tile (all blocks); the residual region starts at
-                         // tiles_offset + rt_stride * ntile and holds 32 nrw bytes per row tile
+  uint32_t nrw;          // residual words per row tile (all blocks); the residual streams start at
+                         // tiles_offset + rt_stride * ntile, 64 nblk + 32 nrw bytes per row tile
   uint32_t rwtab_offset; // byte offset of the residual word table
 };
 static_assert(sizeof(Header) == 64, "header is 64 bytes");
@@ -106,7 +108,7 @@ struct BlockInfo {       // 64 bytes, one per block, right after the header
 static_assert(sizeof(BlockInfo) == 64, "block info is 64 bytes");
 
 struct ResidWord {       // 8 bytes, one per residual word, in word order
-  uint32_t block;        // the block the word belongs to
+  uint32_t block_wq;     // 8 * (the block the word belongs to) + (its number 0..7 among the block's words)
   uint8_t cols[4];       // its four salient columns (0..127); 0 for unused slots (their code is "no term")
 };
 static_assert(sizeof(ResidWord) == 8, "residual word entry is 8 bytes");
@@ -117,9 +119,14 @@ STB_HD constexpr int n_hi(int N) { return N > 4 ? N - 4 : 0; }
 STB_HD constexpr int sign_full_words(int N) { return (n_lo(N) >> 1) + (n_hi(N) >> 1); }
 STB_HD constexpr bool sign_has_half(int N) { return (N & 1) != 0; }
 
-STB_HD constexpr uint32_t tile_bytes(int N) { return 512u + 192u * (uint32_t)N + 320u; }
-// bytes of the residual codes of one row tile / of one residual word of a row tile
-STB_HD constexpr uint64_t resid_rt_bytes(uint32_t nrw) { return 32ull * nrw; }
+STB_HD constexpr uint32_t tile_bytes(int N) { return 512u + 192u * (uint32_t)N + 256u; }
+// Residual stream of a row tile: bytes in all, offset of block b's record, and inside a record the a_sal2 of
+// the four rows of lane group g (8 bytes: rows g, g + 8, g + 16, g + 24) and the codes of its word wq.
+constexpr uint32_t kResidA2Bytes = 64u, kResidWordBytes = 32u;
+STB_HD constexpr uint64_t resid_rt_bytes(int nblk, uint32_t nrw) { return (uint64_t)kResidA2Bytes * (uint32_t)nblk + (uint64_t)kResidWordBytes * nrw; }
+STB_HD constexpr uint64_t resid_block_off(int b, uint32_t rw_off) { return (uint64_t)kResidA2Bytes * (uint32_t)b + (uint64_t)kResidWordBytes * rw_off; }
+STB_HD constexpr uint32_t resid_a2_off(int g, int j) { return (uint32_t)(4 * g + j) * 2u; }
+STB_HD constexpr uint32_t resid_code_off(uint32_t wq, int g) { return kResidA2Bytes + (wq * 8u + (uint32_t)g) * 4u; }
 STB_HD constexpr uint32_t rwtab_offset(int nblk) { return (uint32_t)(sizeof(Header) + sizeof(BlockInfo) * (size_t)nblk); }
 // the table is sized for the most residual words a layer can have, so that the tiles start at an offset that
 // depends on the shape alone
@@ -140,7 +147,6 @@ STB_HD constexpr uint32_t pair_field_index(uint32_t field, int upper_row) {
 STB_HD constexpr uint32_t off_region(int) { return 512u; }
 STB_HD constexpr uint32_t off_sign(int N) { return 512u + 128u * (uint32_t)N; }
 STB_HD constexpr uint32_t off_scale(int N) { return 512u + 192u * (uint32_t)N; }
-STB_HD constexpr uint32_t off_sal2(int N) { return off_scale(N) + 256u; }
 
 // Byte offset (inside the tile) of word `iw` of a per-lane field of `nw` words that starts at
 // `base`: the words are laid out as uint4 planes, then (nw & 2) a uint2 plane, then (nw & 1)
@@ -164,12 +170,8 @@ STB_HD constexpr uint32_t sign_word_off(int N, int sw, int lane) {
 STB_HD constexpr uint32_t sign_half_off(int N, int lane) {
   return off_sign(N) + 128u * (uint32_t)sign_full_words(N) + (uint32_t)(lane & 15) * 4u;
 }
-// scale / sal2 / resid are indexed by the permuted row position p = 4 g + j of row g + 8 j
+// scales are indexed by the permuted row position p = 4 g + j of row g + 8 j
 STB_HD constexpr uint32_t scale_off(int N, int g, int j) { return off_scale(N) + (uint32_t)(4 * g + j) * 8u; }
-STB_HD constexpr uint32_t sal2_off(int N, int g, int j) { return off_sal2(N) + (uint32_t)(4 * g + j) * 2u; }
-// byte offset of residual word w (numbered over the whole row tile) of lane group g inside the row tile's
-// residual codes
-STB_HD constexpr uint64_t resid_word_off(uint32_t w, int g) { return ((uint64_t)w * 8u + (uint32_t)g) * 4u; }
 
 // bit position of the two-bit code number i (0..15) of a region word
 STB_HD constexpr int code_bit(int i) {

@@ -54,7 +54,7 @@ __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ 
   for (int b = threadIdx.x; b < nblk; b += blockDim.x)
     for (uint32_t wq = 0; wq < bi[b].nrw; ++wq) {
       ResidWord e;
-      e.block = (uint32_t)b;
+      e.block_wq = 8u * (uint32_t)b + wq;
       for (int k = 0; k < 4; ++k) e.cols[k] = bi[b].cols[4 * wq + k];
       rwt[bi[b].rw_off + wq] = e;
     }
@@ -62,13 +62,13 @@ __global__ void header_kernel(int n, int m, int N, const uint64_t* __restrict__ 
     const int ntile = (n + kTileRows - 1) / kTileRows;
     const uint32_t tb = tile_bytes(N);
     hdr->magic = kMagic;
-    hdr->version = 3;
+    hdr->version = 4;
     hdr->n = n; hdr->m = m; hdr->N = N;
     hdr->nblk = nblk;
     hdr->ntile = ntile;
     hdr->tiles_offset = tiles_offset(nblk);
     hdr->rt_stride = (uint64_t)tb * (uint64_t)nblk;
-    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + (hdr->rt_stride + resid_rt_bytes(total)) * (uint64_t)ntile;
+    hdr->used_bytes = (uint64_t)tiles_offset(nblk) + (hdr->rt_stride + resid_rt_bytes(nblk, total)) * (uint64_t)ntile;
     hdr->status = bad ? (uint32_t)STB_ERR_CORRUPT : 0u;
     hdr->tile_bytes = tb;
     hdr->nrw = total;
@@ -119,8 +119,9 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
   const uint64_t sal_lo = bi->salient[0], sal_hi = bi->salient[1];
   const int nsal = (int)bi->nsal, nrw_b = (int)bi->nrw;
   uint8_t* tile = packed + hdr->tiles_offset + ((size_t)rt * nblk + b) * (size_t)hdr->tile_bytes;
-  uint8_t* resid = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
-                   (size_t)rt * resid_rt_bytes(hdr->nrw) + resid_word_off(bi->rw_off, 0);
+  // the block's record in the row tile's residual stream: a_sal2 of the 32 rows, then the residual words
+  uint8_t* record = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
+                    (size_t)rt * resid_rt_bytes(nblk, hdr->nrw) + resid_block_off(b, bi->rw_off);
 
   // ---- phase 1: lane = row ----
   // rows past n: nothing kept, all signs "+", zero scales
@@ -176,7 +177,7 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
   const uint32_t A = (sc[0] & 0xFFu) | ((sc[1] & 0xFFu) << 8) | ((sc[2] & 0xFFu) << 16) | ((uint32_t)(sc[3] & 0xFFu) << 24);
   const uint32_t B = (sc[0] >> 8) | ((uint32_t)(sc[1] >> 8) << 8) | ((uint32_t)(sc[2] >> 8) << 16) | ((uint32_t)(sc[3] >> 8) << 24);
   *reinterpret_cast<uint2*>(tile + scale_off(N, pg, pj)) = make_uint2(A, B);
-  *reinterpret_cast<uint16_t*>(tile + sal2_off(N, pg, pj)) = sc[4];
+  *reinterpret_cast<uint16_t*>(record + resid_a2_off(pg, pj)) = sc[4];
 
   // residual codes of the block's salient columns: 0 = +a_sal2, 2 = -a_sal2, 1 = no term
   if (valid && nsal < 32 && (s2 >> nsal) != 0) bad = true;
@@ -203,7 +204,7 @@ pack_kernel(stb_logical L, uint8_t* __restrict__ packed, int* dev_status) {
       }
       word |= __shfl_xor_sync(0xFFFFFFFFu, word, 8);
       word |= __shfl_xor_sync(0xFFFFFFFFu, word, 16);
-      if (lane < 8) *reinterpret_cast<uint32_t*>(resid + resid_word_off((uint32_t)wq, lane)) = word;
+      if (lane < 8) *reinterpret_cast<uint32_t*>(record + resid_code_off((uint32_t)wq, lane)) = word;
     }
   }
   __syncwarp();
@@ -267,7 +268,7 @@ extern "C" int stb_pack_size(int n, int m, int N, size_t* bytes) {
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
   const size_t nblk = (size_t)m / stb::kBlock, ntile = ((size_t)n + 31) / 32;
-  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * ((size_t)stb::tile_bytes(N) + (size_t)stb::resid_rt_bytes(stb::kMaxResidWords));
+  *bytes = (size_t)stb::tiles_offset((int)nblk) + ntile * nblk * ((size_t)stb::tile_bytes(N) + (size_t)stb::resid_rt_bytes(1, stb::kMaxResidWords));
   return STB_OK;
 }
 
@@ -311,7 +312,7 @@ extern "C" int stb_packed_info(const void* packed, stb_info* info, void* stream)
   info->n = h.n; info->m = h.m; info->N = h.N;
   info->status = (int)h.status;
   info->used_bytes = h.used_bytes;
-  info->stream_bytes = (h.rt_stride + stb::resid_rt_bytes(h.nrw)) * (uint64_t)h.ntile;
+  info->stream_bytes = (h.rt_stride + stb::resid_rt_bytes(h.nblk, h.nrw)) * (uint64_t)h.ntile;
   return STB_OK;
 }
 

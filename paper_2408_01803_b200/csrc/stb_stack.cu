@@ -1,0 +1,832 @@
+// stb_layer_stack_resident: a whole list of decode GEMV steps as ONE resident kernel (batch 1..8, N = 4, 5, 6).
+//
+// The per-layer launches of stb_layer_stack pay, for every layer, a launch ramp, a copy of the activations per
+// CTA, a cluster reduction and a last wave that leaves SMs idle.  Here one CTA of 16 warps per SM stays
+// resident for the whole list (cooperative launch: all CTAs are on the machine together):
+//   * Consecutive steps that read the same activations (q / k / v, gate / up) form a PHASE.  The 32 x 128 tiles of
+//     a phase, in (row tile, block) order, are dealt to the CTAs as equal contiguous ranges, and a CTA's range
+//     to its 16 warps the same way: every SM gets the same number of tiles whatever the shapes are.
+//   * Each warp streams its tiles through a private ring in shared memory with 1-D bulk copies (mbarrier
+//     completion, bounded waits) and runs ahead into its range of the NEXT phase: packed weights never depend on
+//     activations, so the stream does not stop at a phase boundary.
+//   * Decode and multiply per tile are those of stb_gemv: 6:8 keeps the weights in rank order and lets
+//     mma.sp.m16n8k32 place them (activations from an image of x in operand order in shared memory, built once
+//     per phase and CTA); 4:8 and 5:8 (and 6:8 when the image does not fit or for more than two batch rows)
+//     decode to position order for mma.m16n8k16 with the activations read through L1.
+//   * The residual term of the salient columns (Eq. 4) is applied per span of up to five blocks from the span's
+//     records of the residual stream, brought into shared memory by one bulk copy while the span's tiles run.
+//   * Partial sums: a warp that covers a whole row tile writes y itself; the others leave their head / tail
+//     pieces in shared memory and the CTA adds them in tile order at the end of the phase; a row tile that
+//     straddles CTAs goes through partial tiles in the caller's workspace, summed in CTA order by whichever
+//     CTA arrives last (a counter per row tile).  Every sum has a fixed order: results are reproducible.
+//   * A phase may read what an earlier phase wrote: a CTA starts a phase's arithmetic only when the count of
+//     finished row tiles (one counter in the workspace, bumped once per CTA and phase) has reached the total
+//     of all earlier phases.  The poll is bounded; when it or an mbarrier wait runs out, an abort flag makes
+//     every CTA leave, STB_ERR_TIMEOUT is reported and the last CTA out restores the workspace to zero.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/stb.h"
+#include "stb_decode.cuh"
+#include "stb_layout.cuh"
+#include "stb_ptx.cuh"
+
+namespace stb {
+
+__device__ const Meta6Table g_meta6_stack = make_meta6_table();
+
+constexpr int kSWarps = 16;
+constexpr int kSThreads = kSWarps * 32;
+constexpr int kMaxPhases = 64;                // per launch; longer lists run as several launches
+constexpr int kMaxFusedSteps = 4;
+constexpr int kSDepth = 2, kSChunk = 2;       // ring: slots per warp, tiles per bulk copy
+constexpr uint32_t kSlotBytes = 4096;         // two tiles of at most 1920 bytes
+constexpr int kSpan = 5;                      // blocks per residual span
+constexpr uint32_t kStageBytes = 2048;        // per warp: the span's residual records (<= 5 x 320) + its word table
+constexpr uint32_t kStageTab = 1664;
+constexpr long long kSWaitLimit = 2000000000ll;        // about a second of SM clocks
+constexpr long long kSSelftestLimit = 100000ll;
+constexpr uint32_t kImgWordsPerBlock = 96;    // 6:8 operand-order image: words per block and batch row
+
+struct StackPhase {
+  const uint8_t* packed[kMaxFusedSteps];
+  void* y[kMaxFusedSteps];
+  uint32_t ldy[kMaxFusedSteps];
+  int32_t n[kMaxFusedSteps];
+  int32_t tile_start[kMaxFusedSteps + 1];     // row tiles of the phase: step i owns [tile_start[i], tile_start[i + 1])
+  const __half* x;
+  uint32_t ldx;
+  int32_t m;
+  uint8_t N, batch, count, f16_mask;          // f16_mask bit i: step i writes fp16
+  uint8_t use_image, pad[3];
+  uint32_t done_before;                       // row tiles finished by all earlier phases of this launch
+};
+
+struct StackParams {
+  StackPhase ph[kMaxPhases];
+  int32_t nphase;
+  uint32_t image_bytes;                       // shared memory set aside for the 6:8 activation image
+  uint32_t part_floats;                       // floats per partial slot: 32 rows x largest batch
+  uint32_t max_share;                         // most CTAs that share one row tile
+  uint32_t* sync;                             // [0] finished row tiles, [1] abort flag, [2] CTAs that left, [4..] per row tile arrivals
+  float* gpart;                               // partial tiles of row tiles that straddle CTAs
+  int* dev_status;
+  long long wait_limit;
+  int32_t copies_off;
+};
+
+// shared memory plan
+struct SSmem {
+  static constexpr uint32_t meta6 = 0;                               // 256 B
+  static constexpr uint32_t pos = 256;                               // 3 x 576 B position tables (N = 4, 5, 6)
+  static constexpr uint32_t bars = 256 + 3 * 576;                    // ring barriers: 16 warps x 2 + 16 stage barriers
+  static constexpr uint32_t ctl = bars + 8 * (kSWarps * kSDepth + kSWarps);   // control words
+  static constexpr uint32_t slots = ctl + 64;                        // partial slot descriptors: 32 x 16 B
+  static constexpr uint32_t ring = 3072;
+  static constexpr uint32_t stage = ring + kSWarps * kSDepth * kSlotBytes;
+  static constexpr uint32_t pdata = stage + kSWarps * kStageBytes;
+};
+static_assert(SSmem::slots + 32 * 16 <= SSmem::ring, "control area overflows");
+
+struct PartSlot { int32_t R, lo, hi, pad; };   // row tile (phase-wide number) or -1, block range [lo, hi)
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 ld_v4(const void* p) {      // coherent load (the activations are written by this kernel)
+  uint4 v;
+  asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_u16(const void* p) {
+  unsigned short v;
+  asm volatile("ld.global.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// T tiles are dealt to the first Ge = min(G, T) CTAs as ranges [c T / Ge, (c + 1) T / Ge): none of them is empty.
+__host__ __device__ __forceinline__ int dealt_ctas(long long T, int G) { return T < (long long)G ? (int)T : G; }
+// the CTA that owns tile L
+__host__ __device__ __forceinline__ int owner_of(long long L, long long T, int Ge) { return (int)(((L + 1) * Ge - 1) / T); }
+
+// One warp's walk through the tiles of all phases, in chunks of up to kSChunk tiles that never cross a packed
+// buffer.  The producer side (bulk copies) and the consumer side each hold one of these.
+struct TileWalk {
+  int phase;            // current phase (== nphase: finished)
+  long long L, hi;      // next tile of the warp's range of that phase, end of the range
+  int nb, N;
+  __device__ void enter(const StackParams& P, int ph, int cta, int G, int warp) {
+    phase = ph;
+    while (phase < P.nphase) {
+      const StackPhase& q = P.ph[phase];
+      nb = q.m / kBlock; N = q.N;
+      const long long T = (long long)q.tile_start[q.count] * nb;
+      const int Ge = dealt_ctas(T, G);
+      if (cta < Ge) {
+        const long long cl = T * cta / Ge, ch = T * (cta + 1) / Ge;
+        L = cl + (ch - cl) * warp / kSWarps;
+        hi = cl + (ch - cl) * (warp + 1) / kSWarps;
+        if (L < hi) return;
+      }
+      ++phase;
+    }
+  }
+  // next chunk: source address and number of tiles (0 when the walk is over)
+  __device__ int next(const StackParams& P, int cta, int G, int warp, const uint8_t*& src, int& ph_of_chunk) {
+    if (phase >= P.nphase) return 0;
+    const StackPhase& q = P.ph[phase];
+    const int R = (int)(L / nb);
+    int i = 0;
+#pragma unroll
+    for (int k = 1; k < kMaxFusedSteps; ++k)
+      if (k < q.count && R >= q.tile_start[k]) i = k;
+    const long long step_end = (long long)q.tile_start[i + 1] * nb;
+    long long e = L + kSChunk;
+    if (e > hi) e = hi;
+    if (e > step_end) e = step_end;
+    const int cnt = (int)(e - L);
+    src = q.packed[i] + tiles_offset(nb) + (size_t)(L - (long long)q.tile_start[i] * nb) * tile_bytes(N);
+    ph_of_chunk = phase;
+    L = e;
+    if (L >= hi) enter(P, phase + 1, cta, G, warp);
+    return cnt;
+  }
+};
+
+// ------------------------------------------------------------------------------------------
+// One 32 x 128 tile at 6:8 through the sparse instruction, activations from the image (see stb_gemv.cu).
+__device__ __forceinline__ void tile_sp6(const LaneTile<6>& lt, const uint8_t* smem, const uint32_t* xi0, bool xlive,
+                                         float (&acc)[2][4]) {
+  FastRows<6> fr;
+  fr.init(lt, lt.A, lt.B);
+  uint32_t E[2][3];
+#pragma unroll
+  for (int bb = 0; bb < 2; ++bb) {
+    uint32_t en[2][4];
+#pragma unroll
+    for (int tq = 0; tq < 4; ++tq)
+#pragma unroll
+      for (int rp = 0; rp < 2; ++rp) {
+        const uint32_t off = prmt(lt.mask[2 * bb + (tq >> 1)], 0u, 0x4440u + (uint32_t)(2 * (tq & 1) + rp));
+        en[rp][tq] = *reinterpret_cast<const uint32_t*>(smem + SSmem::meta6 + off);
+      }
+    meta6_words(en, E[bb]);
+  }
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt) {
+    uint32_t XLh[2][2], XHh[2][2];
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+      for (int sp = 0; sp < 2; ++sp) fr.high(2 * mt + jj, sp, XLh[jj][sp], XHh[jj][sp]);
+#pragma unroll
+    for (int sl = 0; sl < 2; ++sl) {
+      uint32_t R[2][2][3];
+#pragma unroll
+      for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) fr.pairs(2 * mt + jj, 2 * h + sl, XLh[jj][h], XHh[jj][h], R[jj][h]);
+#pragma unroll
+      for (int i = 0; i < 3; ++i) {
+        uint4 bx = make_uint4(0, 0, 0, 0);
+        if (xlive) bx = *reinterpret_cast<const uint4*>(xi0 + sl * 12 + 4 * i);
+        if (mt == 0) mma_sp16832<0>(acc[0], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
+        else mma_sp16832<1>(acc[1], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
+      }
+    }
+  }
+}
+
+// One tile in position order (N = 4, 5, 6): byte-permute decode into m16n8k16 operands; activations of batch row g
+// through L1 (xrow = x + g ldx + 8 t + 128 b, or null for lanes beyond the batch).
+template <int N>
+__device__ __forceinline__ void tile_dense(const LaneTile<N>& lt, const uint2* ptab, const __half* xrow, float (&acc)[2][4]) {
+  FastRows<N> fr;
+  fr.init(lt, lt.A, lt.B);
+  uint32_t XL[4] = {0, 0, 0, 0}, XH[4] = {0, 0, 0, 0};
+  if (N == 5) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) fr.high(j, 0, XL[j], XH[j]);
+  }
+  uint2 P[16];
+#pragma unroll
+  for (int u = 0; u < 16; ++u) P[u] = ptab[keep_index_of(lt.mask, u >> 2, u & 3)];
+  uint4 xf[4];
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    xf[s] = make_uint4(0, 0, 0, 0);
+    if (xrow) xf[s] = ld_v4(xrow + s * 32);
+  }
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    uint32_t f[4][4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (N == 6 && (s & 1) == 0) fr.high(j, s >> 1, XL[j], XH[j]);
+      fr.slot2(j, s, P[4 * j + s].x, P[4 * j + s].y, XL[j], XH[j], f[j]);
+    }
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      mma16816(acc[mt], f[2 * mt][0], f[2 * mt + 1][0], f[2 * mt][1], f[2 * mt + 1][1], xf[s].x, xf[s].y);
+      mma16816(acc[mt], f[2 * mt][2], f[2 * mt + 1][2], f[2 * mt][3], f[2 * mt + 1][3], xf[s].z, xf[s].w);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSThreads, 1)
+stack_kernel(const __grid_constant__ StackParams P) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
+  const int cta = (int)blockIdx.x, G = (int)gridDim.x;
+  volatile int* ctl = reinterpret_cast<volatile int*>(smem + SSmem::ctl);      // [0] failed, [1] row tiles finished by this CTA, [2] last CTA out, [3] a packed header does not match
+  PartSlot* pslot = reinterpret_cast<PartSlot*>(smem + SSmem::slots);
+  float* pdata = reinterpret_cast<float*>(smem + SSmem::pdata);
+  uint32_t* ximg = reinterpret_cast<uint32_t*>(smem + SSmem::pdata + 32u * P.part_floats * 4u);
+
+  // Packed headers must match the steps; every CTA reads the same headers and takes the same way out, before it
+  // has touched the workspace.
+  {
+    if (threadIdx.x == 0) ctl[3] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < P.nphase * kMaxFusedSteps; i += blockDim.x) {
+      const StackPhase& q = P.ph[i / kMaxFusedSteps];
+      const int k = i % kMaxFusedSteps;
+      if (k < q.count && !header_matches(reinterpret_cast<const Header*>(q.packed[k]), q.n[k], q.m, q.N)) ctl[3] = 1;
+    }
+    __syncthreads();
+    if (ctl[3]) {
+      if (threadIdx.x == 0 && cta == 0 && P.dev_status) *P.dev_status = STB_ERR_CORRUPT;
+      return;
+    }
+  }
+
+  // tables, barriers, control words
+  for (int i = threadIdx.x; i < kMeta6Entries; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + SSmem::meta6)[i] = g_meta6_stack.v[i];
+  for (int i = threadIdx.x; i < 3 * kPosTableEntries; i += blockDim.x)
+    reinterpret_cast<uint2*>(smem + SSmem::pos)[i] = g_pos_table.v[4 + i / kPosTableEntries][i % kPosTableEntries];
+  const uint32_t bar0 = smem_u32(smem + SSmem::bars) + (uint32_t)warp * kSDepth * 8u;
+  const uint32_t bar_stage = smem_u32(smem + SSmem::bars) + (uint32_t)(kSWarps * kSDepth + warp) * 8u;
+  uint8_t* ring = smem + SSmem::ring + (size_t)warp * kSDepth * kSlotBytes;
+  uint8_t* stage = smem + SSmem::stage + (size_t)warp * kStageBytes;
+  if (lane == 0) {
+    for (int i = 0; i < kSDepth; ++i) mbar_init(bar0 + 8u * i, 1);
+    mbar_init(bar_stage, 1);
+    fence_async_smem();
+  }
+  if (threadIdx.x == 0) { ctl[0] = 0; ctl[1] = 0; ctl[2] = 0; }
+  __syncwarp();
+
+  // ring: the producer walk runs kSDepth chunks ahead of the tiles the warp consumes
+  TileWalk prod;
+  prod.enter(P, 0, cta, G, warp);
+  int chunk_cnt[kSDepth], chunk_ph[kSDepth];       // what was issued into each slot
+  uint32_t issued = 0, consumed = 0;                // chunk counters
+#pragma unroll
+  for (int i = 0; i < kSDepth; ++i) { chunk_cnt[i] = 0; chunk_ph[i] = 0; }
+  auto issue = [&](int slot) {
+    const uint8_t* src = nullptr;
+    int ph = 0;
+    const int Ncur = prod.phase < P.nphase ? prod.N : 0;
+    const int cnt = prod.next(P, cta, G, warp, src, ph);
+    chunk_cnt[slot] = cnt; chunk_ph[slot] = ph;
+    if (cnt > 0) {
+      if (lane == 0) {
+        const uint32_t bytes = (uint32_t)cnt * tile_bytes(Ncur);
+        fence_async_smem();
+        mbar_expect_tx(bar0 + 8u * slot, bytes);
+        if (!P.copies_off) bulk_g2s(smem_u32(ring + (size_t)slot * kSlotBytes), src, bytes, bar0 + 8u * slot);
+      }
+      ++issued;
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < kSDepth; ++i) issue(i);
+  __syncthreads();
+
+  bool failed = false;           // this warp gave up (its own wait ran out, or the CTA was told to)
+  uint32_t stage_use = 0;        // residual stage copies issued by this warp (barrier parity)
+  int cur_slot = 0, cur_in = 0;  // consumer position inside the ring: slot and tile inside its chunk
+
+  for (int ph = 0; ph < P.nphase; ++ph) {
+    const StackPhase& q = P.ph[ph];
+    const int nb = q.m / kBlock, N = q.N, batch = q.batch;
+    const long long T = (long long)q.tile_start[q.count] * nb;
+    const int Ge = dealt_ctas(T, G);
+    long long wl = 0, wh = 0;
+    if (cta < Ge) {
+      const long long cl = T * cta / Ge, ch = T * (cta + 1) / Ge;
+      wl = cl + (ch - cl) * warp / kSWarps; wh = cl + (ch - cl) * (warp + 1) / kSWarps;
+    }
+
+    // ---- wait until every earlier phase has finished, then (6:8) lay the activations out in operand order ----
+    if (threadIdx.x == 0 && !ctl[0] && q.done_before > 0) {
+      const long long t0 = clock64();
+      while (ld_acquire_u32(P.sync) < q.done_before) {
+        if (ld_acquire_u32(P.sync + 1) != 0u) { ctl[0] = 1; break; }
+        if (clock64() - t0 > P.wait_limit) {
+          ctl[0] = 1;
+          atomicExch(P.sync + 1, 1u);
+          if (P.dev_status) *P.dev_status = STB_ERR_TIMEOUT;
+          break;
+        }
+      }
+    }
+    __syncthreads();
+    if (ctl[0]) failed = true;
+    const uint32_t img_row_words = (uint32_t)nb * kImgWordsPerBlock;
+    if (q.use_image && !ctl[0]) {
+      // one item = the 8 activations of one group of one batch row: a 16-byte load, six 4-byte stores (see stb_gemv.cu)
+      const int items = batch * nb * 16;
+      for (int base = 0; base < items; base += 4 * kSThreads) {
+        uint4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int it = base + k * kSThreads + (int)threadIdx.x;
+          v[k] = make_uint4(0, 0, 0, 0);
+          if (it < items) {
+            const int r = it / (nb * 16), qq = it - r * nb * 16;
+            v[k] = ld_v4(q.x + (size_t)r * q.ldx + (size_t)qq * 8);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int it = base + k * kSThreads + (int)threadIdx.x;
+          if (it < items) {
+            const int r = it / (nb * 16), qq = it - r * nb * 16, blk = qq >> 4, Gp = qq & 15;
+            uint32_t* d = ximg + (uint32_t)r * img_row_words + (uint32_t)blk * kImgWordsPerBlock +
+                          (uint32_t)((4 * (Gp & 1) + ((Gp >> 2) & 1)) * 12 + 2 * (Gp >> 3) + ((Gp >> 1) & 1));
+            d[0] = v[k].x; d[4] = v[k].y; d[8] = v[k].z;
+            d[24] = v[k].y; d[28] = v[k].z; d[32] = v[k].w;
+          }
+        }
+      }
+    }
+    if (lane == 0) { pslot[2 * warp].R = -1; pslot[2 * warp + 1].R = -1; }
+    __syncthreads();
+
+    // ---- this warp's tiles ----
+    const uint2* ptab = reinterpret_cast<const uint2*>(smem + SSmem::pos) + (N - 4) * kPosTableEntries;
+    const __half* xg = g < batch ? q.x + (size_t)g * q.ldx : nullptr;       // batch row of this lane group
+    long long L = wl;
+    int nslot_used = 0;
+    while (L < wh && !failed) {
+      const int R = (int)(L / nb);
+      int si = 0;
+#pragma unroll
+      for (int k = 1; k < kMaxFusedSteps; ++k)
+        if (k < q.count && R >= q.tile_start[k]) si = k;
+      const int rt = R - q.tile_start[si];
+      const uint8_t* packed = q.packed[si];
+      const Header* hdr = reinterpret_cast<const Header*>(packed);
+      const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+      const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + rwtab_offset(nb));
+      const int ntile = (q.n[si] + kTileRows - 1) / kTileRows;
+      const uint32_t nrw_all = __ldg(&hdr->nrw);
+      const uint8_t* resid_rt = packed + tiles_offset(nb) + (size_t)tile_bytes(N) * nb * ntile + (size_t)rt * resid_rt_bytes(nb, nrw_all);
+      const int b_first = (int)(L - (long long)R * nb);
+      const long long seg_end_l = (long long)(R + 1) * nb < wh ? (long long)(R + 1) * nb : wh;
+      const int b_end = (int)(seg_end_l - (long long)R * nb);
+      float acc[2][4];
+#pragma unroll
+      for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int d = 0; d < 4; ++d) acc[a][d] = 0.0f;
+
+      for (int bs = b_first; bs < b_end && !failed; bs += kSpan) {
+        const int be = bs + kSpan < b_end ? bs + kSpan : b_end;
+        // the span's records of the residual stream and its residual word table, one bulk copy each
+        const uint32_t rw0 = __ldg(&binfo[bs].rw_off), rw1 = __ldg(&binfo[be - 1].rw_off) + __ldg(&binfo[be - 1].nrw);
+        const uint32_t rec_bytes = (uint32_t)(resid_block_off(be, rw1) - resid_block_off(bs, rw0));
+        const uint32_t tab0 = rw0 & ~1u, tab_bytes = ((rw1 - tab0) * 8u + 15u) & ~15u;       // 16-byte aligned piece of the table
+        __syncwarp();
+        if (lane == 0) {
+          fence_async_smem();
+          mbar_expect_tx(bar_stage, rec_bytes + (rw1 > rw0 ? tab_bytes : 0u));
+          if (!P.copies_off) {
+            bulk_g2s(smem_u32(stage), resid_rt + resid_block_off(bs, rw0), rec_bytes, bar_stage);
+            if (rw1 > rw0) bulk_g2s(smem_u32(stage + kStageTab), rwt + tab0, tab_bytes, bar_stage);
+          }
+        }
+        const uint32_t stage_parity = stage_use & 1u;
+        ++stage_use;
+
+        for (int b = bs; b < be; ++b) {
+          if (cur_in == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(bar0 + 8u * cur_slot, (consumed / kSDepth) & 1u, P.wait_limit))) { failed = true; break; }
+          const uint8_t* tile = ring + (size_t)cur_slot * kSlotBytes + (size_t)cur_in * tile_bytes(N);
+          const bool last_of_chunk = cur_in + 1 == chunk_cnt[cur_slot];
+          if (N == 6 && q.use_image) {
+            LaneTile<6> lt;
+            load_lane_tile<6>(tile, lane, lt, true);
+            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
+            tile_sp6(lt, smem, ximg + (uint32_t)g * img_row_words + (uint32_t)b * kImgWordsPerBlock + (uint32_t)(t * 24), g < batch, acc);
+          } else if (N == 6) {
+            LaneTile<6> lt;
+            load_lane_tile<6>(tile, lane, lt);
+            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
+            tile_dense<6>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
+          } else if (N == 5) {
+            LaneTile<5> lt;
+            load_lane_tile<5>(tile, lane, lt);
+            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
+            tile_dense<5>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
+          } else {
+            LaneTile<4> lt;
+            load_lane_tile<4>(tile, lane, lt);
+            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
+            tile_dense<4>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
+          }
+          if (last_of_chunk) { cur_in = 0; cur_slot = (cur_slot + 1) % kSDepth; ++consumed; }
+          else ++cur_in;
+        }
+        if (failed) break;
+
+        // residual term of the span's salient columns: four residual words (16 salient slots) per tensor-core step
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_stage, stage_parity, P.wait_limit))) { failed = true; break; }
+        if (rw1 > rw0) {
+          const uint32_t nstep = (rw1 - rw0 + 3u) >> 2;
+#pragma unroll 1
+          for (uint32_t i = 0; i < nstep; ++i) {
+            const uint32_t wi = rw0 + 4u * i + (uint32_t)t;
+            uint32_t rw = 0x55555555u, cols = 0u, block = (uint32_t)bs;
+            uint2 a2 = make_uint2(0u, 0u);
+            if (wi < rw1) {
+              const uint2 e = *reinterpret_cast<const uint2*>(stage + kStageTab + (wi - tab0) * 8u);
+              block = e.x >> 3; cols = e.y;
+              const uint8_t* rec = stage + kResidA2Bytes * (block - (uint32_t)bs) + kResidWordBytes * (wi - (e.x & 7u) - rw0);
+              a2 = *reinterpret_cast<const uint2*>(rec + resid_a2_off(g, 0));
+              rw = *reinterpret_cast<const uint32_t*>(rec + resid_code_off(e.x & 7u, g));
+            }
+            uint32_t fa[4][2];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t h = (((j & 2) ? a2.y : a2.x) >> (16 * (j & 1))) & 0xFFFFu;
+              const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
+              const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
+              const uint32_t sel = resid_selector(rw, j);
+              const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
+              fa[j][0] = prmt(lo4, hi4, 0x5140u);
+              fa[j][1] = prmt(lo4, hi4, 0x7362u);
+            }
+            uint2 xr = make_uint2(0, 0);
+            if (xg) {
+              const __half* xq = xg + (size_t)block * kBlock;
+              xr.x = ld_u16(xq + (cols & 0xFFu)) | (ld_u16(xq + ((cols >> 8) & 0xFFu)) << 16);
+              xr.y = ld_u16(xq + ((cols >> 16) & 0xFFu)) | (ld_u16(xq + (cols >> 24)) << 16);
+            }
+            mma16816(acc[0], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
+            mma16816(acc[1], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
+          }
+        }
+      }
+      if (failed) break;
+
+      // ---- the segment [b_first, b_end) of row tile R is summed: a whole row tile goes to y, a piece to shared memory ----
+      if (b_first == 0 && b_end == nb) {
+        const bool f16 = (q.f16_mask >> si) & 1;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int d = 0; d < 4; ++d) {
+            const int row = rt * kTileRows + g + 16 * mt + 8 * (d >> 1), bc = 2 * t + (d & 1);
+            if (row < q.n[si] && bc < batch) {
+              if (f16) static_cast<__half*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = __float2half_rn(acc[mt][d]);
+              else static_cast<float*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = acc[mt][d];
+            }
+          }
+        if (lane == 0) atomicAdd(const_cast<int*>(&ctl[1]), 1);
+      } else {
+        const int slot = 2 * warp + nslot_used;
+        ++nslot_used;
+        float* pd = pdata + (size_t)slot * P.part_floats;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int d = 0; d < 4; ++d) {
+            const int r = g + 16 * mt + 8 * (d >> 1), bc = 2 * t + (d & 1);
+            if (bc < batch) pd[r * batch + bc] = acc[mt][d];
+          }
+        if (lane == 0) { pslot[slot].R = R; pslot[slot].lo = b_first; pslot[slot].hi = b_end; }
+      }
+      L = seg_end_l;
+    }
+    if (failed && lane == 0 && !ctl[0]) {
+      // this warp's own wait ran out: tell the CTA and the grid
+      ctl[0] = 1;
+      atomicExch(P.sync + 1, 1u);
+      if (P.dev_status) *P.dev_status = STB_ERR_TIMEOUT;
+    }
+    __syncthreads();
+
+    // ---- pieces of row tiles, added in tile order.  Slot 2 w (head piece of warp w), 2 w + 1 (tail piece) are in tile
+    // order; a run of slots with the same row tile is one group, handled by the warp that owns its first slot. ----
+    if (!ctl[0]) {
+      for (int s0 = 2 * warp; s0 < 2 * warp + 2; ++s0) {
+        const int R = pslot[s0].R;
+        if (R < 0) continue;
+        // the nearest used slot before s0 decides whether s0 starts a group
+        int prev = s0 - 1;
+        while (prev >= 0 && pslot[prev].R < 0) --prev;
+        if (prev >= 0 && pslot[prev].R == R) continue;
+        int s1 = s0, hi_b = pslot[s0].hi;
+        for (int s = s0 + 1; s < 2 * kSWarps; ++s) {
+          if (pslot[s].R < 0) continue;
+          if (pslot[s].R != R) break;
+          s1 = s; hi_b = pslot[s].hi;
+        }
+        const int lo_b = pslot[s0].lo;
+        int si = 0;
+#pragma unroll
+        for (int k = 1; k < kMaxFusedSteps; ++k)
+          if (k < q.count && R >= q.tile_start[k]) si = k;
+        const int rt = R - q.tile_start[si];
+        const bool f16 = (q.f16_mask >> si) & 1;
+        const int nval = 32 * batch;                 // values of the row tile: [row][batch column]
+        const bool whole = lo_b == 0 && hi_b == nb;
+        float* gp = nullptr;
+        int share = 1;
+        if (!whole) {
+          const int c_first = owner_of((long long)R * nb, T, Ge), c_last = owner_of((long long)(R + 1) * nb - 1, T, Ge);
+          share = c_last - c_first + 1;
+          gp = P.gpart + ((size_t)R * P.max_share + (size_t)(cta - c_first)) * P.part_floats;
+        }
+        for (int v = lane; v < nval; v += 32) {
+          float sum = 0.0f;
+          for (int s = s0; s <= s1; ++s)
+            if (pslot[s].R == R) sum += pdata[(size_t)s * P.part_floats + v];
+          if (whole) {
+            const int row = rt * kTileRows + v / batch, bc = v % batch;
+            if (row < q.n[si]) {
+              if (f16) static_cast<__half*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = __float2half_rn(sum);
+              else static_cast<float*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = sum;
+            }
+          } else {
+            gp[v] = sum;
+          }
+        }
+        if (whole) {
+          if (lane == 0) atomicAdd(const_cast<int*>(&ctl[1]), 1);
+        } else {
+          // the row tile straddles CTAs: whoever arrives last adds the partial tiles in CTA order
+          __syncwarp();
+          uint32_t old = 0;
+          if (lane == 0) { __threadfence(); old = atomicAdd(P.sync + 4 + R, 1u); }
+          old = __shfl_sync(0xFFFFFFFFu, old, 0);
+          if ((int)old == share - 1) {
+            __threadfence();
+            const float* g0 = P.gpart + (size_t)R * P.max_share * P.part_floats;
+            for (int v = lane; v < nval; v += 32) {
+              float sum = 0.0f;
+              for (int k = 0; k < share; ++k) sum += __ldcg(g0 + (size_t)k * P.part_floats + v);
+              const int row = rt * kTileRows + v / batch, bc = v % batch;
+              if (row < q.n[si]) {
+                if (f16) static_cast<__half*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = __float2half_rn(sum);
+                else static_cast<float*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = sum;
+              }
+            }
+            if (lane == 0) { P.sync[4 + R] = 0u; atomicAdd(const_cast<int*>(&ctl[1]), 1); }
+          }
+        }
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int fin = ctl[1];
+      ctl[1] = 0;
+      if (fin > 0 && !ctl[0]) { __threadfence(); atomicAdd(P.sync, (uint32_t)fin); }
+    }
+  }
+
+  // ---- leaving: let copies in flight land, then the last CTA out restores the workspace ----
+  if (ctl[0] || failed) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000) {}
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const uint32_t old = atomicAdd(P.sync + 2, 1u);
+    ctl[2] = (old == (uint32_t)G - 1u) ? 1 : 0;
+  }
+  __syncthreads();
+  if (ctl[2]) {
+    __threadfence();
+    const bool aborted = ld_acquire_u32(P.sync + 1) != 0u;
+    if (aborted) {
+      int maxR = 0;
+      for (int ph = 0; ph < P.nphase; ++ph) maxR = max(maxR, P.ph[ph].tile_start[P.ph[ph].count]);
+      for (int i = threadIdx.x; i < maxR; i += blockDim.x) P.sync[4 + i] = 0u;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) { P.sync[0] = 0u; P.sync[1] = 0u; P.sync[2] = 0u; __threadfence(); }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side: steps -> phases -> launches.
+struct StackPlan {
+  size_t sync_bytes, gpart_bytes;
+};
+
+static bool same_input(const stb_step& a, const stb_step& b) {
+  return a.in == b.in && a.ldin == b.ldin && a.batch == b.batch && a.m == b.m && a.N == b.N && b.out != a.in;
+}
+
+static int check_step(const stb_step& s) {
+  if (!s.packed || !s.in || !s.out) return STB_ERR_ARG;
+  if (s.n < 1 || s.m < kBlock || s.m % kBlock != 0) return STB_ERR_SHAPE;
+  if (s.N < 1 || s.N > 8) return STB_ERR_NM;
+  if (s.N < 4 || s.N > 6) return STB_ERR_UNSUPPORTED;
+  if (s.batch < 1 || s.batch > 64) return STB_ERR_SIZE;
+  if (s.batch > 8) return STB_ERR_UNSUPPORTED;
+  if (s.odt != STB_F32 && s.odt != STB_F16) return STB_ERR_UNSUPPORTED;
+  if (s.ldin < (size_t)s.m || s.ldout < (size_t)s.n || (s.ldin % 8) != 0 || (reinterpret_cast<uintptr_t>(s.in) & 15u)) return STB_ERR_ARG;
+  if (s.ldin > 0xFFFFFFFFull || s.ldout > 0xFFFFFFFFull) return STB_ERR_ARG;
+  return STB_OK;
+}
+
+// most CTAs that share one row tile of a phase of R row tiles x nb blocks dealt to G CTAs
+static uint32_t max_share_of(long long R, int nb, int G) {
+  const long long T = R * nb;
+  const int Ge = dealt_ctas(T, G);
+  uint32_t best = 1;
+  for (long long r = 0; r < R; ++r) {
+    const int c0 = owner_of(r * nb, T, Ge), c1 = owner_of((r + 1) * nb - 1, T, Ge);
+    const uint32_t s = (uint32_t)(c1 - c0 + 1);
+    if (s > best) best = s;
+  }
+  return best;
+}
+
+static int stack_sm_count(int* out) {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return STB_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return STB_ERR_CUDA;
+  if (!cached[dev]) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1) return STB_ERR_CUDA;
+    cached[dev] = v;
+  }
+  *out = cached[dev];
+  return STB_OK;
+}
+
+constexpr uint32_t kSmemLimit = 227 * 1024;
+
+// Builds the phases of steps [i0, ...) into `sp` (at most kMaxPhases), returns the index of the first step not taken.
+static int build_phases(const stb_step* steps, int count, int i0, int G, StackParams& sp, size_t& sync_need, size_t& gpart_need) {
+  sp.nphase = 0;
+  sp.image_bytes = 0; sp.part_floats = 32; sp.max_share = 1;
+  uint32_t done = 0;
+  long long maxR = 0;
+  int i = i0;
+  // first pass: phases and the largest batch (the partial slots are sized by it)
+  while (i < count && sp.nphase < kMaxPhases) {
+    StackPhase& q = sp.ph[sp.nphase];
+    const stb_step& st = steps[i];
+    int j = i + 1;
+    while (j < count && j - i < kMaxFusedSteps && same_input(st, steps[j])) ++j;
+    q.count = (uint8_t)(j - i);
+    q.tile_start[0] = 0;
+    q.f16_mask = 0;
+    for (int k = 0; k < kMaxFusedSteps; ++k) { q.packed[k] = nullptr; q.y[k] = nullptr; q.ldy[k] = 0; q.n[k] = 0; q.tile_start[k + 1] = 0; }
+    for (int k = i; k < j; ++k) {
+      const stb_step& sk = steps[k];
+      q.packed[k - i] = static_cast<const uint8_t*>(sk.packed);
+      q.y[k - i] = sk.out; q.ldy[k - i] = (uint32_t)sk.ldout; q.n[k - i] = sk.n;
+      if (sk.odt == STB_F16) q.f16_mask |= (uint8_t)(1u << (k - i));
+      q.tile_start[k - i + 1] = q.tile_start[k - i] + (sk.n + kTileRows - 1) / kTileRows;
+    }
+    for (int k = q.count; k < kMaxFusedSteps; ++k) q.tile_start[k + 1] = q.tile_start[q.count];
+    q.x = static_cast<const __half*>(st.in);
+    q.ldx = (uint32_t)st.ldin; q.m = st.m; q.N = (uint8_t)st.N; q.batch = (uint8_t)st.batch;
+    q.use_image = 0; q.pad[0] = q.pad[1] = q.pad[2] = 0;
+    q.done_before = done;
+    const long long R = q.tile_start[q.count];
+    done += (uint32_t)R;
+    if (R > maxR) maxR = R;
+    if ((uint32_t)(32 * st.batch) > sp.part_floats) sp.part_floats = (uint32_t)(32 * st.batch);
+    const uint32_t share = max_share_of(R, st.m / kBlock, G);
+    if (share > sp.max_share) sp.max_share = share;
+    ++sp.nphase;
+    i = j;
+  }
+  // second pass: which 6:8 phases get the operand-order image of their activations in shared memory
+  const uint32_t fixed = SSmem::pdata + 32u * sp.part_floats * 4u;
+  for (int p = 0; p < sp.nphase; ++p) {
+    StackPhase& q = sp.ph[p];
+    if (q.N != 6 || q.batch > 2) continue;
+    const uint32_t need = (uint32_t)q.batch * (uint32_t)(q.m / kBlock) * kImgWordsPerBlock * 4u;
+    if (fixed + need <= kSmemLimit) {
+      q.use_image = 1;
+      if (need > sp.image_bytes) sp.image_bytes = need;
+    }
+  }
+  const size_t s_need = (size_t)(4 + maxR) * sizeof(uint32_t);
+  const size_t g_need = (size_t)maxR * sp.max_share * sp.part_floats * sizeof(float);
+  if (s_need > sync_need) sync_need = s_need;
+  if (g_need > gpart_need) gpart_need = g_need;
+  return i;
+}
+
+static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+}  // namespace stb
+
+extern "C" int stb_layer_stack_resident_workspace(const stb_step* steps, int count, size_t* bytes) {
+  if (!steps || count < 1 || !bytes) return STB_ERR_ARG;
+  for (int i = 0; i < count; ++i) {
+    const int rc = stb::check_step(steps[i]);
+    if (rc != STB_OK) return rc;
+  }
+  int G = 0;
+  int rc = stb::stack_sm_count(&G);
+  if (rc != STB_OK) return rc;
+  size_t sync_need = 0, gpart_need = 0;
+  static thread_local stb::StackParams sp;
+  int i = 0;
+  while (i < count) i = stb::build_phases(steps, count, i, G, sp, sync_need, gpart_need);
+  *bytes = stb::align256(sync_need) + stb::align256(gpart_need);
+  return STB_OK;
+}
+
+static int stack_resident_impl(const stb_step* steps, int count, void* ws, size_t ws_bytes, int* dev_status, void* stream,
+                               bool selftest) {
+  if (!steps || count < 1 || !ws) return STB_ERR_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return STB_ERR_ARG;
+  for (int i = 0; i < count; ++i) {
+    const int rc = stb::check_step(steps[i]);
+    if (rc != STB_OK) return rc;
+  }
+  int G = 0;
+  int rc = stb::stack_sm_count(&G);
+  if (rc != STB_OK) return rc;
+  // the whole list must fit the workspace before anything is launched
+  size_t sync_need = 0, gpart_need = 0;
+  static thread_local stb::StackParams sp;
+  {
+    int i = 0;
+    while (i < count) i = stb::build_phases(steps, count, i, G, sp, sync_need, gpart_need);
+  }
+  const size_t sync_bytes = stb::align256(sync_need);
+  if (ws_bytes < sync_bytes + stb::align256(gpart_need)) return STB_ERR_SIZE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  static bool attr_done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return STB_ERR_CUDA;
+  if (!attr_done[dev]) {
+    if (cudaFuncSetAttribute(stb::stack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stb::kSmemLimit) != cudaSuccess) return STB_ERR_CUDA;
+    attr_done[dev] = true;
+  }
+  int i = 0;
+  while (i < count) {
+    size_t a = 0, b = 0;
+    i = stb::build_phases(steps, count, i, G, sp, a, b);
+    sp.sync = static_cast<uint32_t*>(ws);
+    sp.gpart = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + sync_bytes);
+    sp.dev_status = dev_status;
+    sp.wait_limit = selftest ? stb::kSSelftestLimit : stb::kSWaitLimit;
+    sp.copies_off = selftest ? 1 : 0;
+    const uint32_t smem = stb::SSmem::pdata + 32u * sp.part_floats * 4u + sp.image_bytes;
+    if (smem > stb::kSmemLimit) return STB_ERR_UNSUPPORTED;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)G, 1, 1);
+    cfg.blockDim = dim3((unsigned)stb::kSThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, stb::stack_kernel, sp) != cudaSuccess) return STB_ERR_CUDA;
+  }
+  return STB_OK;
+}
+
+extern "C" int stb_layer_stack_resident(const stb_step* steps, int count, void* ws, size_t ws_bytes, int* dev_status,
+                                        void* stream) {
+  return stack_resident_impl(steps, count, ws, ws_bytes, dev_status, stream, false);
+}
+
+extern "C" int stb_layer_stack_resident_wait_selftest(const stb_step* steps, int count, void* ws, size_t ws_bytes,
+                                                      int* dev_status, void* stream) {
+  if (!dev_status) return STB_ERR_ARG;
+  return stack_resident_impl(steps, count, ws, ws_bytes, dev_status, stream, true);
+}
+
+extern "C" int stb_layer_stack_resident_host(const stb_step* steps, int count, void* ws, size_t ws_bytes, const void* in_host,
+                                             size_t in_bytes, void* out_host, size_t out_bytes, int* dev_status, void* stream) {
+  if (!steps || count < 1 || !in_host || !out_host || !steps[0].in || !steps[count - 1].out) return STB_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(const_cast<void*>(steps[0].in), in_host, in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return STB_ERR_CUDA;
+  const int rc = stb_layer_stack_resident(steps, count, ws, ws_bytes, dev_status, stream);
+  if (rc != STB_OK) return rc;
+  if (cudaMemcpyAsync(out_host, steps[count - 1].out, out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return STB_ERR_CUDA;
+  return STB_OK;
+}

@@ -54,8 +54,10 @@ static int check(int trials, int spb) {
       for (int q = 0; q < 32; ++q) rcode[r][q] = q < spb ? (uint8_t)(rnd() % 3) : 1;
     }
     const uint32_t tb = tile_bytes(N);
-    const uint32_t w0 = 3;     // the block's first residual word inside the row tile's residual codes
-    std::vector<uint8_t> tile(tb + 64, 0), resid(resid_rt_bytes(w0 + spb / 4) + 64, 0);
+    const int blk = 2;         // the tile's block number and its first residual word inside the row tile's stream
+    const uint32_t w0 = 3;
+    std::vector<uint8_t> tile(tb + 64, 0), stream(resid_rt_bytes(blk + 1, w0 + spb / 4) + 64, 0);
+    uint8_t* record = stream.data() + resid_block_off(blk, w0);
     auto put32 = [&](uint32_t off, uint32_t v) { std::memcpy(&tile[off], &v, 4); };
     auto or32 = [&](uint32_t off, uint32_t v) { uint32_t o; std::memcpy(&o, &tile[off], 4); o |= v; std::memcpy(&tile[off], &o, 4); };
     for (int lane = 0; lane < 32; ++lane) {
@@ -88,16 +90,17 @@ static int check(int trials, int spb) {
       uint32_t A = 0, B = 0;
       for (int q = 0; q < 4; ++q) { A |= (uint32_t)(scale[r][q] & 0xFF) << (8 * q); B |= (uint32_t)(scale[r][q] >> 8) << (8 * q); }
       put32(scale_off(N, g, j), A); put32(scale_off(N, g, j) + 4, B);
-      std::memcpy(&tile[sal2_off(N, g, j)], &scale[r][4], 2);
+      std::memcpy(record + resid_a2_off(g, j), &scale[r][4], 2);
       for (int q = 0; q < spb; ++q) {
         uint32_t o;
-        std::memcpy(&o, &resid[resid_word_off(w0 + (uint32_t)(q >> 2), g)], 4);
+        std::memcpy(&o, record + resid_code_off((uint32_t)(q >> 2), g), 4);
         o |= (uint32_t)rcode[r][q] << code_bit(4 * j + (q & 3));
-        std::memcpy(&resid[resid_word_off(w0 + (uint32_t)(q >> 2), g)], &o, 4);
+        std::memcpy(record + resid_code_off((uint32_t)(q >> 2), g), &o, 4);
       }
     }
     // every offset must stay inside the tile
-    if (sal2_off(N, 7, 3) + 2u != tb || resid_word_off(w0 + 8u - 1u, 7) + 4u != resid_rt_bytes(w0 + 8u) || resid_words_for(5) != 2 || resid_words_for(32) != kMaxResidWords) {
+    if (scale_off(N, 7, 3) + 8u != tb || resid_block_off(blk, w0) + resid_code_off(7u, 7) + 4u != resid_rt_bytes(blk + 1, w0 + 8u) ||
+        resid_a2_off(7, 3) + 2u != kResidA2Bytes || resid_words_for(5) != 2 || resid_words_for(32) != kMaxResidWords) {
       ++errors; std::printf("N=%d tile size mismatch\n", N);
     }
 
@@ -126,10 +129,10 @@ static int check(int trials, int spb) {
         const int r = g + 8 * j;
         for (int q = 0; q < 4; ++q)
           if (scale_bits<N>(lt, j, q) != scale[r][q]) { if (++errors < 10) std::printf("scale N=%d\n", N); }
-        if (sal2_bits<N>(lt, j) != scale[r][4]) { if (++errors < 10) std::printf("sal2 N=%d\n", N); }
+        if (sal2_bits(record, g, j) != scale[r][4]) { if (++errors < 10) std::printf("sal2 N=%d\n", N); }
         for (int q = 0; q < spb; ++q) {
           uint32_t word;
-          std::memcpy(&word, &resid[resid_word_off(w0 + (uint32_t)(q >> 2), g)], 4);
+          word = resid_word(record, (uint32_t)(q >> 2), g);
           if (resid_code(word, j, q & 3) != rcode[r][q]) { if (++errors < 10) std::printf("resid code N=%d\n", N); }
           if (((resid_selector(word, j) >> (4 * (q & 3))) & 0xFu) != rcode[r][q]) { if (++errors < 10) std::printf("resid selector N=%d\n", N); }
         }
@@ -217,7 +220,7 @@ static int check(int trials, int spb) {
               uint32_t f1[4];
               const uint32_t pp = position_selector(mask_from_index(N, (rw.mask >> (8 * s)) & 0xFFu));
               orow.slot(s, pp & 0xFFFFu, pp >> 16, f1);
-              if (f1[0] != f[0] || f1[1] != f[1] || f1[2] != f[2] || f1[3] != f[3] || rw.sal2 != sal2_bits<N>(lt, j)) {
+              if (f1[0] != f[0] || f1[1] != f[1] || f1[2] != f[2] || f1[3] != f[3]) {
                 if (++errors < 10) std::printf("one row N=%d lane %d j %d s %d\n", N, lane, j, s);
               }
             }
