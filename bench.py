@@ -42,8 +42,8 @@ MLP = ("gate", "up", "down")
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 MIN_TIMED_S = 0.25
-KERNEL_SOURCES = ("stb_gemv.cu", "stb_decode.cuh", "stb_layout.cuh", "stb_ptx.cuh")
-TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic_gemv_llama7b_mlp_6of8_batch1.txt")
+KERNEL_SOURCES = ("stb_stack.cu", "stb_decode.cuh", "stb_layout.cuh", "stb_ptx.cuh")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic_stack_kernel_llama7b_mlp_6of8_batch1.txt")
 
 
 def peaks():
@@ -215,8 +215,8 @@ def clone_layer(stb, lay, used):
 class Workload:
     """The MLP layers packed on the device, `copies` times each at distinct addresses."""
 
-    def __init__(self, stb, torch, copies):
-        self.stb, self.torch = stb, torch
+    def __init__(self, stb, torch, copies, resident=True):
+        self.stb, self.torch, self.resident = stb, torch, resident
         self.logical = [quantized(2, name) for name in MLP]
         self.layers = []          # [copy][k]
         first = [stb.pack_numpy(d) for d in self.logical]
@@ -235,22 +235,34 @@ class Workload:
         self.steps = [stb.make_steps([(ls[0], self.x, self.h_gate), (ls[1], self.x, self.h_up),
                                       (ls[2], self.h_gate, self.y)]) for ls in self.layers]
         self.bytes_step = sum(i["stream_bytes"] for i in self.infos)
-        self.launches_per_pass = 2          # gate and up read the same input and run as one grid; down is the second launch
+        self.ws = stb.resident_workspace(self.steps[0])      # one pass and many passes need the same workspace: it is sized by the largest group
 
     def step(self, c):
-        self.stb.layer_stack(None, dev_status=self.status, marshalled=self.steps[c % len(self.steps)])
+        if self.resident:
+            self.stb.layer_stack_resident(None, self.ws, dev_status=self.status, marshalled=self.steps[c % len(self.steps)])
+        else:
+            self.stb.layer_stack(None, dev_status=self.status, marshalled=self.steps[c % len(self.steps)])
+
+    def step_host(self, c, xh, yh):
+        if self.resident:
+            self.stb.layer_stack_resident_host(self.steps[c % len(self.steps)], self.ws, xh, yh, dev_status=self.status)
+        else:
+            self.stb.layer_stack_host(self.steps[c % len(self.steps)], xh, yh, dev_status=self.status)
 
     def run_steps(self, first, count):
-        """`count` consecutive passes (copies first, first + 1, ...) as ONE stb_layer_stack call, the way a
-        model's whole stack of linears is queued: every layer after the first is chained to its
-        predecessor by a programmatic dependent launch."""
+        """`count` consecutive passes (copies first, first + 1, ...) as ONE call, the way a model's whole stack of
+        linears is queued: stb_layer_stack_resident (one resident kernel for the whole list) or stb_layer_stack
+        (one launch per group of same-input layers, chained by programmatic dependent launches)."""
         trip = []
         for c in range(first, first + count):
             ls = self.layers[c % len(self.layers)]
             trip += [(ls[0], self.x, self.h_gate), (ls[1], self.x, self.h_up), (ls[2], self.h_gate, self.y)]
         arr = self.stb.make_steps(trip)
         self._keep = getattr(self, "_keep", []) + [arr]
-        self.stb.layer_stack(None, dev_status=self.status, marshalled=arr)
+        if self.resident:
+            self.stb.layer_stack_resident(None, self.ws, dev_status=self.status, marshalled=arr)
+        else:
+            self.stb.layer_stack(None, dev_status=self.status, marshalled=arr)
 
 
 def capture(torch, fns):
@@ -415,6 +427,9 @@ def gemm_table(stb, torch, pk, real_ffn):
     return out
 
 
+CALL = {True: "stb_layer_stack_resident (one resident kernel)", False: "stb_layer_stack (per-layer launches)"}
+
+
 def decoder(h, f):
     return [("q", h, h), ("k", h, h), ("v", h, h), ("o", h, h), ("gate", f, h), ("up", f, h), ("down", h, f)]
 
@@ -434,8 +449,9 @@ def build_stack(stb, config, names_N):
     return layers
 
 
-def run_stack(stb, torch, layers, h, f, batch, nl, min_calls):
-    """All linears of `nl` decoder layers as ONE stb_layer_stack call in a CUDA graph; microseconds per call."""
+def run_stack(stb, torch, layers, h, f, batch, nl, min_calls, resident):
+    """All linears of `nl` decoder layers as ONE stb_layer_stack_resident (or stb_layer_stack) call in a CUDA graph;
+    microseconds per call."""
     x = torch.from_numpy(si.activations(batch, h, si.seed_for(5, 40))).cuda()
     hb = [torch.empty(batch, h, dtype=torch.float16, device="cuda") for _ in range(5)]     # q k v o + layer output
     fb = [torch.empty(batch, f, dtype=torch.float16, device="cuda") for _ in range(2)]
@@ -447,7 +463,11 @@ def run_stack(stb, torch, layers, h, f, batch, nl, min_calls):
         cur = hb[4]      # (the data flow of attention / activation functions is not part of this path)
     arr = stb.make_steps(steps)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    fn = lambda: stb.layer_stack(None, dev_status=status, marshalled=arr)
+    if resident:
+        ws = stb.resident_workspace(arr)
+        fn = lambda: stb.layer_stack_resident(None, ws, dev_status=status, marshalled=arr)
+    else:
+        fn = lambda: stb.layer_stack(None, dev_status=status, marshalled=arr)
     g = capture(torch, [fn])
     us = time_graph(torch, g, 1, min_calls=min_calls)
     assert int(status.item()) == 0
@@ -465,27 +485,31 @@ def stack_tables(stb, torch, pk):
     out = []
     l13 = build_stack(stb, 3, [(nm, 5) for nm, _, _ in decoder(5120, 13824)])
     b13 = sum(b for _, _, b in l13)
-    us = run_stack(stb, torch, l13, 5120, 13824, 1, 1, 200)
-    out.append({"stack": "LLaMA-2-13B decoder block, 7 linears, 5:8, batch 1", "us": round(us, 1), "packed_MB": round(b13 / 1e6, 1),
-                "GBps": round(b13 / us / 1e3, 1), "frac_of_measured_hbm": round(b13 / us / 1e3 / pk["hbm_gbs"], 4)})
+    for resident in (True, False):
+        us = run_stack(stb, torch, l13, 5120, 13824, 1, 1, 200, resident)
+        out.append({"stack": "LLaMA-2-13B decoder block, 7 linears, 5:8, batch 1", "call": CALL[resident], "us": round(us, 1),
+                    "packed_MB": round(b13 / 1e6, 1), "GBps": round(b13 / us / 1e3, 1),
+                    "frac_of_measured_hbm": round(b13 / us / 1e3 / pk["hbm_gbs"], 4)})
     del l13
     torch.cuda.empty_cache()
     Nl = si.stack_N_per_layer(32)
     names_N = [(nm, Nl[l]) for l in range(32) for nm, _, _ in decoder(4096, 11008)]
     l7 = build_stack(stb, 5, names_N)
     b7 = sum(b for _, _, b in l7)
-    launches = 32 * 4                 # q/k/v as one grid, o, gate/up as one grid, down
-    for batch in (1, 8, 64):
-        us = run_stack(stb, torch, l7, 4096, 11008, batch, 32, 20)
+    for batch, resident in ((1, True), (1, False), (8, True), (8, False), (64, False)):
+        # resident: 128 groups of same-input linears = two launches of 64 groups; per-layer launches: q/k/v as one grid,
+        # o, gate/up as one grid, down = 128 launches
+        launches = 2 if resident else 32 * 4
+        us = run_stack(stb, torch, l7, 4096, 11008, batch, 32, 20, resident)
         row = {"stack": "LLaMA-2-7B, 32 decoder layers x 7 linears, N per layer from {4,5,6} (%d/%d/%d layers)" % (
-                   Nl.count(4), Nl.count(5), Nl.count(6)), "batch": batch, "us": round(us, 1),
+                   Nl.count(4), Nl.count(5), Nl.count(6)), "call": CALL[resident], "batch": batch, "us": round(us, 1),
                "packed_GB": round(b7 / 1e9, 3), "GBps": round(b7 / us / 1e3, 1),
                "frac_of_measured_hbm": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "us_per_linear": round(us / 224, 2)}
-        if batch == 1:
+        if batch == 1 and resident:
             row["roofline"] = {"bound": "hbm", "achieved": round(b7 / us / 1e3, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                                "frac": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "traffic": None,
-                               "bytes_per_launch": round(b7 / launches), "launch_us": round(us / launches, 3),
-                               "launches": launches, "peak_source": pk["_source"]}
+                               "kernel": "stb::stack_kernel", "bytes_per_launch": round(b7 / launches),
+                               "launch_us": round(us / launches, 3), "launches": launches, "peak_source": pk["_source"]}
         out.append(row)
     del l7
     torch.cuda.empty_cache()
@@ -532,10 +556,10 @@ def cuda_arm(args):
     import paper_2408_01803_b200 as stb
     pk = peaks()
 
-    copies = 12          # 12 distinct copies of the three layers per rotation: more than 6 x L2
+    copies = args.copies          # 12 distinct copies of the three layers per rotation: more than 6 x L2
     if world > 1 and rank != 0:
         dist.barrier()   # rank 0 quantizes (and caches) the layers first
-    wl = Workload(stb, torch, copies)
+    wl = Workload(stb, torch, copies, resident=not args.per_layer_launches)
     if world > 1 and rank == 0:
         dist.barrier()
     K, W = args.steps, args.warmup
@@ -546,7 +570,7 @@ def cuda_arm(args):
         wl.step(i)
     us_pass = time_graph(torch, g_full, copies, min_calls=20 * copies)
     # a step = `reps` graph replays, sized so that the K steps of the timed region last MIN_TIMED_S
-    reps = max(1, int(np.ceil(MIN_TIMED_S / (K * copies * us_pass * 1e-6))))
+    reps = max(1, int(np.ceil(args.min_timed_s / (K * copies * us_pass * 1e-6))))
     if world > 1:
         t = torch.tensor([reps], device="cuda", dtype=torch.int64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -576,10 +600,12 @@ def cuda_arm(args):
         t = torch.tensor([ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
-    launches = wl.launches_per_pass * passes
+    # resident: one launch per graph replay (`copies` passes, 2 groups each); per-layer launches: gate and up as one
+    # grid + down = 2 launches per pass
+    launches = K * reps if wl.resident else 2 * passes
     value = world * wl.bytes_step * passes / (ms * 1e-3) / 1e9
     launch_us = 1e3 * ms / launches
-    per_launch_bytes = wl.bytes_step / float(wl.launches_per_pass)
+    per_launch_bytes = wl.bytes_step * passes / float(launches)
     achieved = per_launch_bytes / launch_us / 1e3
 
     # end to end: x from pinned host memory, y back to the host, every pass
@@ -587,14 +613,14 @@ def cuda_arm(args):
     yh = torch.empty(1, 4096, dtype=torch.float32).pin_memory()
     Ke = max(200, min(passes, 4000))
     for i in range(5):
-        stb.layer_stack_host(wl.steps[i % copies], xh, yh, dev_status=wl.status)
+        wl.step_host(i, xh, yh)
         torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     w0 = time.perf_counter()
     for i in range(Ke):
-        stb.layer_stack_host(wl.steps[i % copies], xh, yh, dev_status=wl.status)
+        wl.step_host(i, xh, yh)
         torch.cuda.current_stream().synchronize()
     w1 = time.perf_counter()
     e2e_s = w1 - w0
@@ -618,27 +644,39 @@ def cuda_arm(args):
         "config": {"workload": WORKLOAD, "inputs": "oracle-quantized", "batch": 1, "layers_per_step": 3,
                    "packed_bytes_per_step": wl.bytes_step, "us_per_layer": round(1e3 * ms / (3 * passes), 3),
                    "step": "ms_per_step is per pass over the three layers; each of the %d steps of the timed region is %d passes "
-                           "(%d graph replays) so that the region lasts >= %.2f s" % (K, reps * copies, reps, MIN_TIMED_S),
+                           "(%d graph replays) so that the region lasts >= %.2f s" % (K, reps * copies, reps, args.min_timed_s),
                    "passes_timed": passes, "timed_region_ms": round(ms, 3),
                    "salient_columns_per_block": {name: salient_histogram(d) for name, d in zip(MLP, wl.logical)},
                    "l2": "cold: %d distinct packed copies of each layer (%.0f MB per rotation, L2 is 126 MB)" % (
                        copies, copies * wl.bytes_step / 1e6),
-                   "launch": "one stb_layer_stack call of %d passes (3 linears each) captured in a CUDA graph and replayed; %d launches "
-                             "per pass (gate+up as one grid, down), chained by programmatic dependent launch" % (copies, wl.launches_per_pass),
+                   "launch": ("one stb_layer_stack_resident call of %d passes (3 linears each) captured in a CUDA graph and replayed: one "
+                              "cooperative launch of one 512-thread CTA per SM for the whole list" % copies) if wl.resident else
+                             ("one stb_layer_stack call of %d passes (3 linears each) captured in a CUDA graph and replayed; 2 launches "
+                              "per pass (gate+up as one grid, down), chained by programmatic dependent launch" % copies),
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks,
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": xh.numel() * 2, "d2h_bytes_per_step": yh.numel() * 4,
                 "steps": Ke, "us_per_step": round(1e6 * e2e_s / Ke, 2),
-                "call": "stb_layer_stack_host: pinned host x -> device, 3 GEMVs, y -> pinned host, stream sync per pass"},
+                "call": ("stb_layer_stack_resident_host" if wl.resident else "stb_layer_stack_host") +
+                        ": pinned host x -> device, 3 GEMVs, y -> pinned host, stream sync per pass"},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": traffic, "traffic_source": traffic_note,
-                     "kernel": "stb::gemv_mma_kernel<6,1>", "peak_source": pk["_source"],
+                     "kernel": "stb::stack_kernel" if wl.resident else "stb::gemv_mma_kernel<6,1>", "peak_source": pk["_source"],
                      "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
-                     "note": "launch_us = timed region / launches (includes the gaps between launches; a launch is gate+up or down, "
-                             "bytes_per_launch is their mean); chained launches of one stb_layer_stack call"},
+                     "note": "launch_us = timed region / launches (includes the gaps between launches)"},
     }
     if world == 1 and not args.no_extras:
+        # the same passes through the other entry point
+        other = not wl.resident
+        wl.resident = other
+        g_other = capture(torch, [lambda: wl.run_steps(0, copies)])
+        us_other = time_graph(torch, g_other, copies, min_calls=100 * copies)
+        wl.resident = not other
+        del g_other
+        line["same_passes_other_call"] = {"call": CALL[other], "us_per_pass": round(us_other, 3),
+                                          "GBps": round(wl.bytes_step / us_other / 1e3, 1),
+                                          "frac_of_measured_hbm": round(wl.bytes_step / us_other / 1e3 / pk["hbm_gbs"], 4)}
         tab, ctx = gemv_table(stb, torch, wl, pk)
         line["gemv_layers"] = tab
         iso = [r for r in tab if r["batch"] == 1 and r["N"] == 6]
@@ -690,6 +728,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-layer tables, the prefill GEMM and the decoder stacks")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--copies", type=int, default=12, help="distinct packed copies of the layers per rotation (cold L2 needs >= 3)")
+    ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S, help="shortest timed region; 0 for a profiler capture")
+    ap.add_argument("--per-layer-launches", action="store_true", help="headline through stb_layer_stack instead of stb_layer_stack_resident")
     ap.add_argument("--real-ffn", action="store_true", help="prefill GEMM: quantize the real 28672-wide FFN layers (CPU minutes)")
     args = ap.parse_args()
     args.steps = args.steps or 20

@@ -187,8 +187,10 @@ int stb_layer_stack(const stb_step *steps, int count, int *dev_status, void *str
  * STB_ERR_UNSUPPORTED (use stb_layer_stack).  Lists of more than 64 groups of same-input steps
  * run as several launches.
  * ws: caller-owned DEVICE workspace of stb_layer_stack_resident_workspace bytes, 256-byte
- * aligned, ZEROED by the caller before its first use; every call leaves it zeroed again, also
- * after a wait that ran out.  Calls that share a workspace must not overlap on the GPU.
+ * aligned, ZEROED by the caller before its first use; every call leaves its counters zero
+ * again (also after a wait that ran out), so the same workspace serves call after call without
+ * being cleared; the rest of it holds partial sums that are written before they are read.
+ * Calls that share a workspace must not overlap on the GPU.
  * The launch is cooperative: it fails with STB_ERR_CUDA when the GPU cannot hold one 512-thread
  * CTA per SM at once. */
 int stb_layer_stack_resident_workspace(const stb_step *steps, int count, size_t *bytes);

@@ -281,6 +281,20 @@ constexpr Meta6Table make_meta6_table() {
   }
   return t;
 }
+// Joint table keyed by the pair field of two rows (stb_layout.cuh): entry J = i0 + 28 i1 holds, in word i, the
+// nibble of chunk i of the mask with index i0 at bit 0 and that of the mask with index i1 at bit 16; the
+// metadata word of chunk i is then  sum over the quad's lanes tq of  word_i(J_tq) << 4 tq.
+struct Meta6Joint { uint32_t v[kMasks6 * kMasks6][4]; };
+constexpr Meta6Joint make_meta6_joint() {
+  Meta6Joint t{};
+  for (uint32_t i1 = 0; i1 < kMasks6; ++i1)
+    for (uint32_t i0 = 0; i0 < kMasks6; ++i0) {
+      for (int i = 0; i < 3; ++i)
+        t.v[i0 + kMasks6 * i1][i] = meta6_nibble(kMaskTables.mask[6][i0], i) | (meta6_nibble(kMaskTables.mask[6][i1], i) << 16);
+      t.v[i0 + kMasks6 * i1][3] = 0;
+    }
+  return t;
+}
 // The six metadata words of a lane from the table entries en[rp][tq] (row g + 16 mt + 8 rp, lane tq of the quad)
 // of one of its two slots: word i has the nibble of lane tq at bit 4 tq (row rp = 0) and 16 + 4 tq (rp = 1).
 STB_HD void meta6_words(const uint32_t (&en)[2][4], uint32_t (&E)[3]) {

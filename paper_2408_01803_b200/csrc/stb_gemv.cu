@@ -262,12 +262,12 @@ gemv_mma_kernel(const __grid_constant__ GemvLayers layers, int m, const __half* 
       for (int bb = 0; bb < 2; ++bb) {
         uint32_t en[2][4];
 #pragma unroll
-        for (int tq = 0; tq < 4; ++tq)
-#pragma unroll
-          for (int rp = 0; rp < 2; ++rp) {
-            const uint32_t off = prmt(lt.mask[2 * bb + (tq >> 1)], 0u, 0x4440u + (uint32_t)(2 * (tq & 1) + rp));
-            en[rp][tq] = *reinterpret_cast<const uint32_t*>(smem + off);
-          }
+        for (int tq = 0; tq < 4; ++tq) {
+          // the pair field of the two rows whose metadata this lane supplies
+          const uint32_t f = (lt.mask[2 * bb + (tq >> 1)] >> (16 * (tq & 1))) & 0xFFFFu;
+          en[0][tq] = reinterpret_cast<const uint32_t*>(smem)[pair_field_index(f, 0)];
+          en[1][tq] = reinterpret_cast<const uint32_t*>(smem)[pair_field_index(f, 1)];
+        }
         meta6_words(en, E[bb]);
       }
       if (image_bytes != 0u) {

@@ -25,10 +25,11 @@
 //                               GEMV multiplies rank-ordered weights with the sparse tensor-core
 //                               instruction, whose selection metadata for rows g + 16 mt and
 //                               g + 16 mt + 8 comes from lanes 2 mt and 2 mt + 1 of the quad.  So
-//                               lane (g, t) holds, at byte 8 b + 2 tq + rp, four times the
-//                               keep-mask index of group 4 (2 (t & 1) + b) + tq of row
-//                               g + 16 (t >> 1) + 8 rp (four times: the byte offset into a table
-//                               of 4-byte entries).
+//                               lane (g, t) holds, at bytes 8 b + 2 tq (16 bits), the pair field
+//                               16 (i0 + 28 i1) of the keep-mask indices i0, i1 of group
+//                               4 (2 (t & 1) + b) + tq of rows g + 16 (t >> 1) and g + 16 (t >> 1) + 8:
+//                               the byte offset into a table of 784 16-byte entries that holds the
+//                               metadata of both rows.
 //   region  N words per lane    two-bit region codes, 16 per word, of the lane's 16 N kept
 //                               weights: first the "low" part (ranks k < min(N, 4) of every
 //                               slot, weight number wl = u NL + k), then the "high" part
@@ -140,9 +141,11 @@ STB_HD constexpr bool mask_pairs(int N) { return N == 6; }
 STB_HD constexpr uint32_t pair_field_off(int g, int mt, int s, int tq) {
   return 16u * (uint32_t)(4 * g + 2 * mt + (s >> 1)) + 8u * (uint32_t)(s & 1) + 2u * (uint32_t)tq;
 }
-STB_HD constexpr uint32_t pair_field(uint32_t i0, uint32_t i1) { return (4u * i0) | ((4u * i1) << 8); }
+constexpr uint32_t kMasks6 = 28;               // C(8, 6)
+STB_HD constexpr uint32_t pair_field(uint32_t i0, uint32_t i1) { return 16u * (i0 + kMasks6 * i1); }
 STB_HD constexpr uint32_t pair_field_index(uint32_t field, int upper_row) {
-  return upper_row ? ((field >> 10) & 63u) : ((field >> 2) & 63u);
+  const uint32_t J = (field >> 4) & 0xFFFu, i1 = (J * 2341u) >> 16;     // J / 28 for J < 784
+  return upper_row ? i1 : J - kMasks6 * i1;
 }
 STB_HD constexpr uint32_t off_region(int) { return 512u; }
 STB_HD constexpr uint32_t off_sign(int N) { return 512u + 128u * (uint32_t)N; }

@@ -4,8 +4,10 @@
 // CTA, a cluster reduction and a last wave that leaves SMs idle.  Here one CTA of 16 warps per SM stays
 // resident for the whole list (cooperative launch: all CTAs are on the machine together):
 //   * Consecutive steps that read the same activations (q / k / v, gate / up) form a PHASE.  The 32 x 128 tiles of
-//     a phase, in (row tile, block) order, are dealt to the CTAs as equal contiguous ranges, and a CTA's range
-//     to its 16 warps the same way: every SM gets the same number of tiles whatever the shapes are.
+//     a phase, in (row tile, block) order, are dealt to the CTAs as contiguous ranges and a CTA's range to its 16
+//     warps as equal contiguous runs.  When whole row tiles can be dealt with little imbalance (at least 85 % of
+//     the SM time used) every CTA gets whole row tiles and no sum crosses CTAs; otherwise the ranges are equal
+//     in tiles and a row tile may straddle CTAs.
 //   * Each warp streams its tiles through a private ring in shared memory with 1-D bulk copies (mbarrier
 //     completion, bounded waits) and runs ahead into its range of the NEXT phase: packed weights never depend on
 //     activations, so the stream does not stop at a phase boundary.
@@ -34,13 +36,14 @@
 
 namespace stb {
 
-__device__ const Meta6Table g_meta6_stack = make_meta6_table();
+__device__ const Meta6Joint g_meta6_joint = make_meta6_joint();
 
 constexpr int kSWarps = 16;
 constexpr int kSThreads = kSWarps * 32;
 constexpr int kMaxPhases = 64;                // per launch; longer lists run as several launches
 constexpr int kMaxFusedSteps = 4;
 constexpr int kSDepth = 2, kSChunk = 2;       // ring: slots per warp, tiles per bulk copy
+static_assert(kSDepth == 2, "the warp state keeps the two slots' chunk sizes in two registers");
 constexpr uint32_t kSlotBytes = 4096;         // two tiles of at most 1920 bytes
 constexpr int kSpan = 5;                      // blocks per residual span
 constexpr uint32_t kStageBytes = 2048;        // per warp: the span's residual records (<= 5 x 320) + its word table
@@ -59,7 +62,7 @@ struct StackPhase {
   uint32_t ldx;
   int32_t m;
   uint8_t N, batch, count, f16_mask;          // f16_mask bit i: step i writes fp16
-  uint8_t use_image, pad[3];
+  uint8_t use_image, aligned, pad[2];         // aligned: CTA ranges are whole row tiles
   uint32_t done_before;                       // row tiles finished by all earlier phases of this launch
 };
 
@@ -78,16 +81,17 @@ struct StackParams {
 
 // shared memory plan
 struct SSmem {
-  static constexpr uint32_t meta6 = 0;                               // 256 B
-  static constexpr uint32_t pos = 256;                               // 3 x 576 B position tables (N = 4, 5, 6)
-  static constexpr uint32_t bars = 256 + 3 * 576;                    // ring barriers: 16 warps x 2 + 16 stage barriers
+  static constexpr uint32_t meta6 = 0;                               // joint 6:8 metadata table, 784 x 16 B, at offset 0: a pair
+                                                                     // field of a tile is the shared-memory address of its entry
+  static constexpr uint32_t pos = kMasks6 * kMasks6 * 16;            // 3 x 576 B position tables (N = 4, 5, 6)
+  static constexpr uint32_t bars = pos + 3 * 576;                    // ring barriers: 16 warps x 2 + 16 stage barriers
   static constexpr uint32_t ctl = bars + 8 * (kSWarps * kSDepth + kSWarps);   // control words
   static constexpr uint32_t slots = ctl + 64;                        // partial slot descriptors: 32 x 16 B
-  static constexpr uint32_t ring = 3072;
+  static constexpr uint32_t ring = 15360;
   static constexpr uint32_t stage = ring + kSWarps * kSDepth * kSlotBytes;
   static constexpr uint32_t pdata = stage + kSWarps * kStageBytes;
 };
-static_assert(SSmem::slots + 32 * 16 <= SSmem::ring, "control area overflows");
+static_assert(SSmem::slots + 32 * 16 <= SSmem::ring && SSmem::ring % 128 == 0, "control area overflows");
 
 struct PartSlot { int32_t R, lo, hi, pad; };   // row tile (phase-wide number) or -1, block range [lo, hi)
 
@@ -107,73 +111,113 @@ __device__ __forceinline__ uint32_t ld_u16(const void* p) {
   return v;
 }
 
-// T tiles are dealt to the first Ge = min(G, T) CTAs as ranges [c T / Ge, (c + 1) T / Ge): none of them is empty.
-__host__ __device__ __forceinline__ int dealt_ctas(long long T, int G) { return T < (long long)G ? (int)T : G; }
-// the CTA that owns tile L
+// Dealing the T = R nb tiles of a phase (R row tiles of nb blocks) to G CTAs.
+//   aligned:  the first Ge = min(G, R) CTAs get whole row tiles, CTA c the row tiles [c R / Ge, (c + 1) R / Ge)
+//   else:     the first Ge = min(G, T) CTAs get the tiles [c T / Ge, (c + 1) T / Ge)
+// (no CTA below Ge is empty); a CTA's range is cut into 16 equal runs for its warps.
+__host__ __device__ __forceinline__ int dealt_ctas(int R, int nb, bool aligned, int G) {
+  const long long units = aligned ? (long long)R : (long long)R * nb;
+  return units < (long long)G ? (int)units : G;
+}
+__host__ __device__ __forceinline__ void cta_range(int R, int nb, bool aligned, int Ge, int c, int& lo, int& hi) {
+  if (aligned) {
+    lo = (int)((long long)R * c / Ge) * nb;
+    hi = (int)((long long)R * (c + 1) / Ge) * nb;
+  } else {
+    const long long T = (long long)R * nb;
+    lo = (int)(T * c / Ge);
+    hi = (int)(T * (c + 1) / Ge);
+  }
+}
+// the CTA that owns tile L (not aligned)
 __host__ __device__ __forceinline__ int owner_of(long long L, long long T, int Ge) { return (int)(((L + 1) * Ge - 1) / T); }
 
-// One warp's walk through the tiles of all phases, in chunks of up to kSChunk tiles that never cross a packed
-// buffer.  The producer side (bulk copies) and the consumer side each hold one of these.
+__device__ __forceinline__ void warp_range(const StackPhase& q, int nb, int cta, int G, int warp, int& lo, int& hi) {
+  const int R = q.tile_start[q.count];
+  const int Ge = dealt_ctas(R, nb, q.aligned != 0, G);
+  lo = hi = 0;
+  if (cta >= Ge) return;
+  int cl, ch;
+  cta_range(R, nb, q.aligned != 0, Ge, cta, cl, ch);
+  lo = cl + (int)(((long long)(ch - cl) * warp) >> 4);
+  hi = cl + (int)(((long long)(ch - cl) * (warp + 1)) >> 4);
+}
+static_assert(kSWarps == 16, "warp_range divides by 16 with a shift");
+
+__device__ __forceinline__ int step_of(const StackPhase& q, int R) {
+  int i = 0;
+#pragma unroll
+  for (int k = 1; k < kMaxFusedSteps; ++k)
+    if (k < q.count && R >= q.tile_start[k]) i = k;
+  return i;
+}
+
+// The producer side of a warp's ring: a walk through the warp's tiles of all phases in chunks of up to kSChunk
+// tiles that never cross a packed buffer.  Between chunks it only bumps a pointer and two counters.
 struct TileWalk {
-  int phase;            // current phase (== nphase: finished)
-  long long L, hi;      // next tile of the warp's range of that phase, end of the range
-  int nb, N;
+  int phase;              // current phase (== nphase: finished)
+  const uint8_t* src;     // next tile
+  int left_range;         // tiles left in the warp's range of this phase
+  int left_step;          // tiles left in the packed buffer `src` points into
+  int step;
+  uint32_t tb;            // tile bytes of this phase
   __device__ void enter(const StackParams& P, int ph, int cta, int G, int warp) {
     phase = ph;
     while (phase < P.nphase) {
       const StackPhase& q = P.ph[phase];
-      nb = q.m / kBlock; N = q.N;
-      const long long T = (long long)q.tile_start[q.count] * nb;
-      const int Ge = dealt_ctas(T, G);
-      if (cta < Ge) {
-        const long long cl = T * cta / Ge, ch = T * (cta + 1) / Ge;
-        L = cl + (ch - cl) * warp / kSWarps;
-        hi = cl + (ch - cl) * (warp + 1) / kSWarps;
-        if (L < hi) return;
+      const int nb = q.m / kBlock;
+      int lo, hi;
+      warp_range(q, nb, cta, G, warp, lo, hi);
+      if (lo < hi) {
+        tb = tile_bytes(q.N);
+        left_range = hi - lo;
+        step = step_of(q, lo / nb);
+        left_step = q.tile_start[step + 1] * nb - lo;
+        src = q.packed[step] + tiles_offset(nb) + (size_t)(lo - q.tile_start[step] * nb) * tb;
+        return;
       }
       ++phase;
     }
   }
-  // next chunk: source address and number of tiles (0 when the walk is over)
-  __device__ int next(const StackParams& P, int cta, int G, int warp, const uint8_t*& src, int& ph_of_chunk) {
+  // next chunk: source address, bytes per tile and number of tiles (0 when the walk is over)
+  __device__ int next(const StackParams& P, int cta, int G, int warp, const uint8_t*& chunk_src, uint32_t& chunk_tb) {
     if (phase >= P.nphase) return 0;
-    const StackPhase& q = P.ph[phase];
-    const int R = (int)(L / nb);
-    int i = 0;
-#pragma unroll
-    for (int k = 1; k < kMaxFusedSteps; ++k)
-      if (k < q.count && R >= q.tile_start[k]) i = k;
-    const long long step_end = (long long)q.tile_start[i + 1] * nb;
-    long long e = L + kSChunk;
-    if (e > hi) e = hi;
-    if (e > step_end) e = step_end;
-    const int cnt = (int)(e - L);
-    src = q.packed[i] + tiles_offset(nb) + (size_t)(L - (long long)q.tile_start[i] * nb) * tile_bytes(N);
-    ph_of_chunk = phase;
-    L = e;
-    if (L >= hi) enter(P, phase + 1, cta, G, warp);
+    int cnt = kSChunk;
+    if (cnt > left_range) cnt = left_range;
+    if (cnt > left_step) cnt = left_step;
+    chunk_src = src; chunk_tb = tb;
+    src += (size_t)cnt * tb;
+    left_range -= cnt; left_step -= cnt;
+    if (left_range == 0) enter(P, phase + 1, cta, G, warp);
+    else if (left_step == 0) {
+      const StackPhase& q = P.ph[phase];
+      const int nb = q.m / kBlock;
+      ++step;
+      src = q.packed[step] + tiles_offset(nb);
+      left_step = (q.tile_start[step + 1] - q.tile_start[step]) * nb;
+    }
     return cnt;
   }
 };
 
 // ------------------------------------------------------------------------------------------
 // One 32 x 128 tile at 6:8 through the sparse instruction, activations from the image (see stb_gemv.cu).
-__device__ __forceinline__ void tile_sp6(const LaneTile<6>& lt, const uint8_t* smem, const uint32_t* xi0, bool xlive,
-                                         float (&acc)[2][4]) {
+__device__ __forceinline__ void tile_sp6(const LaneTile<6>& lt, const uint32_t (&fld)[8], const uint8_t* smem, const uint32_t* xi0,
+                                         bool xlive, float (&acc)[2][4]) {
   FastRows<6> fr;
   fr.init(lt, lt.A, lt.B);
+  // Metadata: fld[4 bb + tq] is the pair field (= the address of the joint-table entry) of slot 2 h + bb of lane tq of
+  // the quad, for the two rows whose metadata this lane supplies; word i of the entries, shifted to the lane's
+  // nibble and added (multiply-adds: the integer pipe is the busy one), is the metadata of chunk i.
   uint32_t E[2][3];
 #pragma unroll
   for (int bb = 0; bb < 2; ++bb) {
-    uint32_t en[2][4];
+    uint4 en[4];
 #pragma unroll
-    for (int tq = 0; tq < 4; ++tq)
-#pragma unroll
-      for (int rp = 0; rp < 2; ++rp) {
-        const uint32_t off = prmt(lt.mask[2 * bb + (tq >> 1)], 0u, 0x4440u + (uint32_t)(2 * (tq & 1) + rp));
-        en[rp][tq] = *reinterpret_cast<const uint32_t*>(smem + SSmem::meta6 + off);
-      }
-    meta6_words(en, E[bb]);
+    for (int tq = 0; tq < 4; ++tq) en[tq] = *reinterpret_cast<const uint4*>(smem + SSmem::meta6 + fld[4 * bb + tq]);
+    E[bb][0] = ((en[3].x * 16u + en[2].x) * 16u + en[1].x) * 16u + en[0].x;
+    E[bb][1] = ((en[3].y * 16u + en[2].y) * 16u + en[1].y) * 16u + en[0].y;
+    E[bb][2] = ((en[3].z * 16u + en[2].z) * 16u + en[1].z) * 16u + en[0].z;
   }
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt) {
@@ -237,10 +281,179 @@ __device__ __forceinline__ void tile_dense(const LaneTile<N>& lt, const uint2* p
 }
 
 // ------------------------------------------------------------------------------------------
+// What a warp carries through the whole kernel.
+struct WarpState {
+  TileWalk prod;                      // producer side of the ring
+  int chunk_cnt0, chunk_cnt1;         // tiles of the chunk in ring slot 0 / 1
+  uint32_t consumed;                  // chunks consumed (slot = consumed % kSDepth, barrier parity = consumed / kSDepth)
+  int cur_in;                         // tile inside the current chunk
+  uint32_t stage_use;                 // residual stage copies issued (barrier parity)
+  bool failed;                        // a wait ran out, or the CTA was told to stop
+};
+
+struct WarpEnv {
+  const StackParams* P;
+  uint8_t* smem;
+  uint8_t* ring;
+  uint8_t* stage;
+  uint32_t bar0, bar_stage;
+  int cta, G, warp, lane, g, t;
+};
+
+__device__ __forceinline__ void ring_issue(const WarpEnv& E, WarpState& W, int slot) {
+  const uint8_t* src = nullptr;
+  uint32_t tb = 0;
+  const int cnt = W.prod.next(*E.P, E.cta, E.G, E.warp, src, tb);
+  if (slot == 0) W.chunk_cnt0 = cnt; else W.chunk_cnt1 = cnt;
+  if (cnt > 0 && E.lane == 0) {
+    const uint32_t bytes = (uint32_t)cnt * tb;
+    fence_async_smem();
+    mbar_expect_tx(E.bar0 + 8u * slot, bytes);
+    if (!E.P->copies_off) bulk_g2s(smem_u32(E.ring + (size_t)slot * kSlotBytes), src, bytes, E.bar0 + 8u * slot);
+  }
+}
+
+// The warp's tiles [lo, hi) of phase q: main stream, residual term per span, partial sums out.
+template <int N, bool kImage>
+__device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const StackPhase& q, int lo, int hi,
+                                          const uint32_t* ximg, PartSlot* pslot, float* pdata, volatile int* ctl) {
+  const StackParams& P = *E.P;
+  const int lane = E.lane, g = E.g, t = E.t, warp = E.warp;
+  const int nb = q.m / kBlock, batch = q.batch;
+  constexpr uint32_t tb = tile_bytes(N);
+  const uint2* ptab = reinterpret_cast<const uint2*>(E.smem + SSmem::pos) + (N - 4) * kPosTableEntries;
+  const __half* xg = g < batch ? q.x + (size_t)g * q.ldx : nullptr;       // batch row of this lane group
+  const uint32_t img_row_words = (uint32_t)nb * kImgWordsPerBlock;
+  int R = lo / nb, b_first = lo - R * nb, left = hi - lo, nslot_used = 0;
+  while (left > 0 && !W.failed) {
+    const int seg = left < nb - b_first ? left : nb - b_first, b_end = b_first + seg;
+    const int si = step_of(q, R);
+    const int rt = R - q.tile_start[si];
+    const uint8_t* packed = q.packed[si];
+    const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+    const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + rwtab_offset(nb));
+    const int ntile = (q.n[si] + kTileRows - 1) / kTileRows;
+    const uint32_t nrw_all = __ldg(&reinterpret_cast<const Header*>(packed)->nrw);
+    const uint8_t* resid_rt = packed + tiles_offset(nb) + (size_t)tb * nb * ntile + (size_t)rt * resid_rt_bytes(nb, nrw_all);
+    float acc[2][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int d = 0; d < 4; ++d) acc[a][d] = 0.0f;
+
+    for (int bs = b_first; bs < b_end && !W.failed; bs += kSpan) {
+      const int be = bs + kSpan < b_end ? bs + kSpan : b_end;
+      // the span's records of the residual stream and its piece of the residual word table: one bulk copy each
+      const uint32_t rw0 = __ldg(&binfo[bs].rw_off), rw1 = __ldg(&binfo[be - 1].rw_off) + __ldg(&binfo[be - 1].nrw);
+      const uint32_t rec_bytes = (uint32_t)(be - bs) * kResidA2Bytes + (rw1 - rw0) * kResidWordBytes;
+      const uint32_t tab0 = rw0 & ~1u, tab_bytes = ((rw1 - tab0) * 8u + 15u) & ~15u;       // 16-byte aligned piece of the table
+      __syncwarp();
+      if (lane == 0) {
+        fence_async_smem();
+        mbar_expect_tx(E.bar_stage, rec_bytes + (rw1 > rw0 ? tab_bytes : 0u));
+        if (!P.copies_off) {
+          bulk_g2s(smem_u32(E.stage), resid_rt + resid_block_off(bs, rw0), rec_bytes, E.bar_stage);
+          if (rw1 > rw0) bulk_g2s(smem_u32(E.stage + kStageTab), rwt + tab0, tab_bytes, E.bar_stage);
+        }
+      }
+      const uint32_t stage_parity = W.stage_use & 1u;
+      ++W.stage_use;
+
+      for (int b = bs; b < be; ++b) {
+        const int slot = (int)(W.consumed % kSDepth);
+        if (W.cur_in == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(E.bar0 + 8u * slot, (W.consumed / kSDepth) & 1u, P.wait_limit))) { W.failed = true; break; }
+        const uint8_t* tile = E.ring + (size_t)slot * kSlotBytes + (size_t)W.cur_in * tb;
+        const bool last_of_chunk = W.cur_in + 1 == (slot == 0 ? W.chunk_cnt0 : W.chunk_cnt1);
+        LaneTile<N> lt;
+        load_lane_tile<N>(tile, lane, lt, kImage);
+        uint32_t fld[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        if constexpr (kImage) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) fld[k] = *reinterpret_cast<const uint16_t*>(tile + lane * 16 + 2 * k);
+        }
+        if (last_of_chunk) { __syncwarp(); ring_issue(E, W, slot); W.cur_in = 0; ++W.consumed; }
+        else ++W.cur_in;
+        if constexpr (kImage) tile_sp6(lt, fld, E.smem, ximg + (uint32_t)g * img_row_words + (uint32_t)b * kImgWordsPerBlock + (uint32_t)(t * 24), g < batch, acc);
+        else tile_dense<N>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
+      }
+      if (W.failed) break;
+
+      // residual term of the span's salient columns: four residual words (16 salient slots) per tensor-core step
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(E.bar_stage, stage_parity, P.wait_limit))) { W.failed = true; break; }
+      if (rw1 > rw0) {
+        const uint32_t nstep = (rw1 - rw0 + 3u) >> 2;
+#pragma unroll 1
+        for (uint32_t i = 0; i < nstep; ++i) {
+          const uint32_t wi = rw0 + 4u * i + (uint32_t)t;
+          uint32_t rw = 0x55555555u, cols = 0u, block = (uint32_t)bs;
+          uint2 a2 = make_uint2(0u, 0u);
+          if (wi < rw1) {
+            const uint2 e = *reinterpret_cast<const uint2*>(E.stage + kStageTab + (wi - tab0) * 8u);
+            block = e.x >> 3; cols = e.y;
+            const uint8_t* rec = E.stage + kResidA2Bytes * (block - (uint32_t)bs) + kResidWordBytes * (wi - (e.x & 7u) - rw0);
+            a2 = *reinterpret_cast<const uint2*>(rec + resid_a2_off(g, 0));
+            rw = *reinterpret_cast<const uint32_t*>(rec + resid_code_off(e.x & 7u, g));
+          }
+          uint32_t fa[4][2];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t h = (((j & 2) ? a2.y : a2.x) >> (16 * (j & 1))) & 0xFFFFu;
+            const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
+            const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
+            const uint32_t sel = resid_selector(rw, j);
+            const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
+            fa[j][0] = prmt(lo4, hi4, 0x5140u);
+            fa[j][1] = prmt(lo4, hi4, 0x7362u);
+          }
+          uint2 xr = make_uint2(0, 0);
+          if (xg) {
+            const __half* xq = xg + (size_t)block * kBlock;
+            xr.x = ld_u16(xq + (cols & 0xFFu)) | (ld_u16(xq + ((cols >> 8) & 0xFFu)) << 16);
+            xr.y = ld_u16(xq + ((cols >> 16) & 0xFFu)) | (ld_u16(xq + (cols >> 24)) << 16);
+          }
+          mma16816(acc[0], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
+          mma16816(acc[1], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
+        }
+      }
+    }
+    if (W.failed) break;
+
+    // ---- the segment [b_first, b_end) of row tile R is summed: a whole row tile goes to y, a piece to shared memory ----
+    if (b_first == 0 && b_end == nb) {
+      const bool f16 = (q.f16_mask >> si) & 1;
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int d = 0; d < 4; ++d) {
+          const int row = rt * kTileRows + g + 16 * mt + 8 * (d >> 1), bc = 2 * t + (d & 1);
+          if (row < q.n[si] && bc < batch) {
+            if (f16) static_cast<__half*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = __float2half_rn(acc[mt][d]);
+            else static_cast<float*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = acc[mt][d];
+          }
+        }
+      if (lane == 0) atomicAdd(const_cast<int*>(&ctl[1]), 1);
+    } else {
+      const int slot = 2 * warp + nslot_used;
+      ++nslot_used;
+      float* pd = pdata + (size_t)slot * P.part_floats;
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int d = 0; d < 4; ++d) {
+          const int r = g + 16 * mt + 8 * (d >> 1), bc = 2 * t + (d & 1);
+          if (bc < batch) pd[r * batch + bc] = acc[mt][d];
+        }
+      if (lane == 0) { pslot[slot].R = R; pslot[slot].lo = b_first; pslot[slot].hi = b_end; }
+    }
+    left -= seg; ++R; b_first = 0;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSThreads, 1)
 stack_kernel(const __grid_constant__ StackParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int cta = (int)blockIdx.x, G = (int)gridDim.x;
   volatile int* ctl = reinterpret_cast<volatile int*>(smem + SSmem::ctl);      // [0] failed, [1] row tiles finished by this CTA, [2] last CTA out, [3] a packed header does not match
   PartSlot* pslot = reinterpret_cast<PartSlot*>(smem + SSmem::slots);
@@ -265,62 +478,37 @@ stack_kernel(const __grid_constant__ StackParams P) {
   }
 
   // tables, barriers, control words
-  for (int i = threadIdx.x; i < kMeta6Entries; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + SSmem::meta6)[i] = g_meta6_stack.v[i];
+  for (int i = threadIdx.x; i < (int)(kMasks6 * kMasks6); i += blockDim.x)
+    reinterpret_cast<uint4*>(smem + SSmem::meta6)[i] = *reinterpret_cast<const uint4*>(g_meta6_joint.v[i]);
   for (int i = threadIdx.x; i < 3 * kPosTableEntries; i += blockDim.x)
     reinterpret_cast<uint2*>(smem + SSmem::pos)[i] = g_pos_table.v[4 + i / kPosTableEntries][i % kPosTableEntries];
-  const uint32_t bar0 = smem_u32(smem + SSmem::bars) + (uint32_t)warp * kSDepth * 8u;
-  const uint32_t bar_stage = smem_u32(smem + SSmem::bars) + (uint32_t)(kSWarps * kSDepth + warp) * 8u;
-  uint8_t* ring = smem + SSmem::ring + (size_t)warp * kSDepth * kSlotBytes;
-  uint8_t* stage = smem + SSmem::stage + (size_t)warp * kStageBytes;
+  WarpEnv E;
+  E.P = &P; E.smem = smem; E.cta = cta; E.G = G; E.warp = warp; E.lane = lane; E.g = lane >> 2; E.t = lane & 3;
+  E.bar0 = smem_u32(smem + SSmem::bars) + (uint32_t)warp * kSDepth * 8u;
+  E.bar_stage = smem_u32(smem + SSmem::bars) + (uint32_t)(kSWarps * kSDepth + warp) * 8u;
+  E.ring = smem + SSmem::ring + (size_t)warp * kSDepth * kSlotBytes;
+  E.stage = smem + SSmem::stage + (size_t)warp * kStageBytes;
   if (lane == 0) {
-    for (int i = 0; i < kSDepth; ++i) mbar_init(bar0 + 8u * i, 1);
-    mbar_init(bar_stage, 1);
+    for (int i = 0; i < kSDepth; ++i) mbar_init(E.bar0 + 8u * i, 1);
+    mbar_init(E.bar_stage, 1);
     fence_async_smem();
   }
   if (threadIdx.x == 0) { ctl[0] = 0; ctl[1] = 0; ctl[2] = 0; }
   __syncwarp();
 
   // ring: the producer walk runs kSDepth chunks ahead of the tiles the warp consumes
-  TileWalk prod;
-  prod.enter(P, 0, cta, G, warp);
-  int chunk_cnt[kSDepth], chunk_ph[kSDepth];       // what was issued into each slot
-  uint32_t issued = 0, consumed = 0;                // chunk counters
+  WarpState W;
+  W.prod.enter(P, 0, cta, G, warp);
+  W.consumed = 0; W.cur_in = 0; W.stage_use = 0; W.failed = false;
 #pragma unroll
-  for (int i = 0; i < kSDepth; ++i) { chunk_cnt[i] = 0; chunk_ph[i] = 0; }
-  auto issue = [&](int slot) {
-    const uint8_t* src = nullptr;
-    int ph = 0;
-    const int Ncur = prod.phase < P.nphase ? prod.N : 0;
-    const int cnt = prod.next(P, cta, G, warp, src, ph);
-    chunk_cnt[slot] = cnt; chunk_ph[slot] = ph;
-    if (cnt > 0) {
-      if (lane == 0) {
-        const uint32_t bytes = (uint32_t)cnt * tile_bytes(Ncur);
-        fence_async_smem();
-        mbar_expect_tx(bar0 + 8u * slot, bytes);
-        if (!P.copies_off) bulk_g2s(smem_u32(ring + (size_t)slot * kSlotBytes), src, bytes, bar0 + 8u * slot);
-      }
-      ++issued;
-    }
-  };
-#pragma unroll
-  for (int i = 0; i < kSDepth; ++i) issue(i);
+  for (int i = 0; i < kSDepth; ++i) ring_issue(E, W, i);
   __syncthreads();
-
-  bool failed = false;           // this warp gave up (its own wait ran out, or the CTA was told to)
-  uint32_t stage_use = 0;        // residual stage copies issued by this warp (barrier parity)
-  int cur_slot = 0, cur_in = 0;  // consumer position inside the ring: slot and tile inside its chunk
 
   for (int ph = 0; ph < P.nphase; ++ph) {
     const StackPhase& q = P.ph[ph];
-    const int nb = q.m / kBlock, N = q.N, batch = q.batch;
-    const long long T = (long long)q.tile_start[q.count] * nb;
-    const int Ge = dealt_ctas(T, G);
-    long long wl = 0, wh = 0;
-    if (cta < Ge) {
-      const long long cl = T * cta / Ge, ch = T * (cta + 1) / Ge;
-      wl = cl + (ch - cl) * warp / kSWarps; wh = cl + (ch - cl) * (warp + 1) / kSWarps;
-    }
+    const int nb = q.m / kBlock, batch = q.batch;
+    int wl, wh;
+    warp_range(q, nb, cta, G, warp, wl, wh);
 
     // ---- wait until every earlier phase has finished, then (6:8) lay the activations out in operand order ----
     if (threadIdx.x == 0 && !ctl[0] && q.done_before > 0) {
@@ -336,11 +524,11 @@ stack_kernel(const __grid_constant__ StackParams P) {
       }
     }
     __syncthreads();
-    if (ctl[0]) failed = true;
-    const uint32_t img_row_words = (uint32_t)nb * kImgWordsPerBlock;
+    if (ctl[0]) W.failed = true;
     if (q.use_image && !ctl[0]) {
       // one item = the 8 activations of one group of one batch row: a 16-byte load, six 4-byte stores (see stb_gemv.cu)
-      const int items = batch * nb * 16;
+      const uint32_t img_row_words = (uint32_t)nb * kImgWordsPerBlock;
+      const int per_row = nb * 16, items = batch * per_row;
       for (int base = 0; base < items; base += 4 * kSThreads) {
         uint4 v[4];
 #pragma unroll
@@ -348,7 +536,7 @@ stack_kernel(const __grid_constant__ StackParams P) {
           const int it = base + k * kSThreads + (int)threadIdx.x;
           v[k] = make_uint4(0, 0, 0, 0);
           if (it < items) {
-            const int r = it / (nb * 16), qq = it - r * nb * 16;
+            const int r = it >= per_row ? 1 : 0, qq = it - r * per_row;       // the image serves one or two batch rows
             v[k] = ld_v4(q.x + (size_t)r * q.ldx + (size_t)qq * 8);
           }
         }
@@ -356,7 +544,7 @@ stack_kernel(const __grid_constant__ StackParams P) {
         for (int k = 0; k < 4; ++k) {
           const int it = base + k * kSThreads + (int)threadIdx.x;
           if (it < items) {
-            const int r = it / (nb * 16), qq = it - r * nb * 16, blk = qq >> 4, Gp = qq & 15;
+            const int r = it >= per_row ? 1 : 0, qq = it - r * per_row, blk = qq >> 4, Gp = qq & 15;
             uint32_t* d = ximg + (uint32_t)r * img_row_words + (uint32_t)blk * kImgWordsPerBlock +
                           (uint32_t)((4 * (Gp & 1) + ((Gp >> 2) & 1)) * 12 + 2 * (Gp >> 3) + ((Gp >> 1) & 1));
             d[0] = v[k].x; d[4] = v[k].y; d[8] = v[k].z;
@@ -369,151 +557,13 @@ stack_kernel(const __grid_constant__ StackParams P) {
     __syncthreads();
 
     // ---- this warp's tiles ----
-    const uint2* ptab = reinterpret_cast<const uint2*>(smem + SSmem::pos) + (N - 4) * kPosTableEntries;
-    const __half* xg = g < batch ? q.x + (size_t)g * q.ldx : nullptr;       // batch row of this lane group
-    long long L = wl;
-    int nslot_used = 0;
-    while (L < wh && !failed) {
-      const int R = (int)(L / nb);
-      int si = 0;
-#pragma unroll
-      for (int k = 1; k < kMaxFusedSteps; ++k)
-        if (k < q.count && R >= q.tile_start[k]) si = k;
-      const int rt = R - q.tile_start[si];
-      const uint8_t* packed = q.packed[si];
-      const Header* hdr = reinterpret_cast<const Header*>(packed);
-      const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
-      const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + rwtab_offset(nb));
-      const int ntile = (q.n[si] + kTileRows - 1) / kTileRows;
-      const uint32_t nrw_all = __ldg(&hdr->nrw);
-      const uint8_t* resid_rt = packed + tiles_offset(nb) + (size_t)tile_bytes(N) * nb * ntile + (size_t)rt * resid_rt_bytes(nb, nrw_all);
-      const int b_first = (int)(L - (long long)R * nb);
-      const long long seg_end_l = (long long)(R + 1) * nb < wh ? (long long)(R + 1) * nb : wh;
-      const int b_end = (int)(seg_end_l - (long long)R * nb);
-      float acc[2][4];
-#pragma unroll
-      for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int d = 0; d < 4; ++d) acc[a][d] = 0.0f;
-
-      for (int bs = b_first; bs < b_end && !failed; bs += kSpan) {
-        const int be = bs + kSpan < b_end ? bs + kSpan : b_end;
-        // the span's records of the residual stream and its residual word table, one bulk copy each
-        const uint32_t rw0 = __ldg(&binfo[bs].rw_off), rw1 = __ldg(&binfo[be - 1].rw_off) + __ldg(&binfo[be - 1].nrw);
-        const uint32_t rec_bytes = (uint32_t)(resid_block_off(be, rw1) - resid_block_off(bs, rw0));
-        const uint32_t tab0 = rw0 & ~1u, tab_bytes = ((rw1 - tab0) * 8u + 15u) & ~15u;       // 16-byte aligned piece of the table
-        __syncwarp();
-        if (lane == 0) {
-          fence_async_smem();
-          mbar_expect_tx(bar_stage, rec_bytes + (rw1 > rw0 ? tab_bytes : 0u));
-          if (!P.copies_off) {
-            bulk_g2s(smem_u32(stage), resid_rt + resid_block_off(bs, rw0), rec_bytes, bar_stage);
-            if (rw1 > rw0) bulk_g2s(smem_u32(stage + kStageTab), rwt + tab0, tab_bytes, bar_stage);
-          }
-        }
-        const uint32_t stage_parity = stage_use & 1u;
-        ++stage_use;
-
-        for (int b = bs; b < be; ++b) {
-          if (cur_in == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(bar0 + 8u * cur_slot, (consumed / kSDepth) & 1u, P.wait_limit))) { failed = true; break; }
-          const uint8_t* tile = ring + (size_t)cur_slot * kSlotBytes + (size_t)cur_in * tile_bytes(N);
-          const bool last_of_chunk = cur_in + 1 == chunk_cnt[cur_slot];
-          if (N == 6 && q.use_image) {
-            LaneTile<6> lt;
-            load_lane_tile<6>(tile, lane, lt, true);
-            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
-            tile_sp6(lt, smem, ximg + (uint32_t)g * img_row_words + (uint32_t)b * kImgWordsPerBlock + (uint32_t)(t * 24), g < batch, acc);
-          } else if (N == 6) {
-            LaneTile<6> lt;
-            load_lane_tile<6>(tile, lane, lt);
-            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
-            tile_dense<6>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
-          } else if (N == 5) {
-            LaneTile<5> lt;
-            load_lane_tile<5>(tile, lane, lt);
-            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
-            tile_dense<5>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
-          } else {
-            LaneTile<4> lt;
-            load_lane_tile<4>(tile, lane, lt);
-            if (last_of_chunk) { __syncwarp(); issue(cur_slot); }
-            tile_dense<4>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
-          }
-          if (last_of_chunk) { cur_in = 0; cur_slot = (cur_slot + 1) % kSDepth; ++consumed; }
-          else ++cur_in;
-        }
-        if (failed) break;
-
-        // residual term of the span's salient columns: four residual words (16 salient slots) per tensor-core step
-        if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_stage, stage_parity, P.wait_limit))) { failed = true; break; }
-        if (rw1 > rw0) {
-          const uint32_t nstep = (rw1 - rw0 + 3u) >> 2;
-#pragma unroll 1
-          for (uint32_t i = 0; i < nstep; ++i) {
-            const uint32_t wi = rw0 + 4u * i + (uint32_t)t;
-            uint32_t rw = 0x55555555u, cols = 0u, block = (uint32_t)bs;
-            uint2 a2 = make_uint2(0u, 0u);
-            if (wi < rw1) {
-              const uint2 e = *reinterpret_cast<const uint2*>(stage + kStageTab + (wi - tab0) * 8u);
-              block = e.x >> 3; cols = e.y;
-              const uint8_t* rec = stage + kResidA2Bytes * (block - (uint32_t)bs) + kResidWordBytes * (wi - (e.x & 7u) - rw0);
-              a2 = *reinterpret_cast<const uint2*>(rec + resid_a2_off(g, 0));
-              rw = *reinterpret_cast<const uint32_t*>(rec + resid_code_off(e.x & 7u, g));
-            }
-            uint32_t fa[4][2];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint32_t h = (((j & 2) ? a2.y : a2.x) >> (16 * (j & 1))) & 0xFFFFu;
-              const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
-              const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
-              const uint32_t sel = resid_selector(rw, j);
-              const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
-              fa[j][0] = prmt(lo4, hi4, 0x5140u);
-              fa[j][1] = prmt(lo4, hi4, 0x7362u);
-            }
-            uint2 xr = make_uint2(0, 0);
-            if (xg) {
-              const __half* xq = xg + (size_t)block * kBlock;
-              xr.x = ld_u16(xq + (cols & 0xFFu)) | (ld_u16(xq + ((cols >> 8) & 0xFFu)) << 16);
-              xr.y = ld_u16(xq + ((cols >> 16) & 0xFFu)) | (ld_u16(xq + (cols >> 24)) << 16);
-            }
-            mma16816(acc[0], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
-            mma16816(acc[1], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
-          }
-        }
-      }
-      if (failed) break;
-
-      // ---- the segment [b_first, b_end) of row tile R is summed: a whole row tile goes to y, a piece to shared memory ----
-      if (b_first == 0 && b_end == nb) {
-        const bool f16 = (q.f16_mask >> si) & 1;
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-          for (int d = 0; d < 4; ++d) {
-            const int row = rt * kTileRows + g + 16 * mt + 8 * (d >> 1), bc = 2 * t + (d & 1);
-            if (row < q.n[si] && bc < batch) {
-              if (f16) static_cast<__half*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = __float2half_rn(acc[mt][d]);
-              else static_cast<float*>(q.y[si])[(size_t)bc * q.ldy[si] + row] = acc[mt][d];
-            }
-          }
-        if (lane == 0) atomicAdd(const_cast<int*>(&ctl[1]), 1);
-      } else {
-        const int slot = 2 * warp + nslot_used;
-        ++nslot_used;
-        float* pd = pdata + (size_t)slot * P.part_floats;
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-          for (int d = 0; d < 4; ++d) {
-            const int r = g + 16 * mt + 8 * (d >> 1), bc = 2 * t + (d & 1);
-            if (bc < batch) pd[r * batch + bc] = acc[mt][d];
-          }
-        if (lane == 0) { pslot[slot].R = R; pslot[slot].lo = b_first; pslot[slot].hi = b_end; }
-      }
-      L = seg_end_l;
+    if (!W.failed && wl < wh) {
+      if (q.N == 6 && q.use_image) run_tiles<6, true>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      else if (q.N == 6) run_tiles<6, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      else if (q.N == 5) run_tiles<5, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      else run_tiles<4, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
     }
-    if (failed && lane == 0 && !ctl[0]) {
+    if (W.failed && lane == 0 && !ctl[0]) {
       // this warp's own wait ran out: tell the CTA and the grid
       ctl[0] = 1;
       atomicExch(P.sync + 1, 1u);
@@ -524,24 +574,19 @@ stack_kernel(const __grid_constant__ StackParams P) {
     // ---- pieces of row tiles, added in tile order.  Slot 2 w (head piece of warp w), 2 w + 1 (tail piece) are in tile
     // order; a run of slots with the same row tile is one group, handled by the warp that owns its first slot. ----
     if (!ctl[0]) {
+      const int Rall = q.tile_start[q.count];
+      // every warp looks at all 32 slot descriptors at once, one per lane
+      const PartSlot mine = pslot[lane];
+      const uint32_t used = __ballot_sync(0xFFFFFFFFu, mine.R >= 0);
       for (int s0 = 2 * warp; s0 < 2 * warp + 2; ++s0) {
-        const int R = pslot[s0].R;
-        if (R < 0) continue;
+        if (!((used >> s0) & 1u)) continue;
+        const int R = __shfl_sync(0xFFFFFFFFu, mine.R, s0);
         // the nearest used slot before s0 decides whether s0 starts a group
-        int prev = s0 - 1;
-        while (prev >= 0 && pslot[prev].R < 0) --prev;
-        if (prev >= 0 && pslot[prev].R == R) continue;
-        int s1 = s0, hi_b = pslot[s0].hi;
-        for (int s = s0 + 1; s < 2 * kSWarps; ++s) {
-          if (pslot[s].R < 0) continue;
-          if (pslot[s].R != R) break;
-          s1 = s; hi_b = pslot[s].hi;
-        }
-        const int lo_b = pslot[s0].lo;
-        int si = 0;
-#pragma unroll
-        for (int k = 1; k < kMaxFusedSteps; ++k)
-          if (k < q.count && R >= q.tile_start[k]) si = k;
+        const uint32_t below = used & ((1u << s0) - 1u);
+        if (below != 0u && __shfl_sync(0xFFFFFFFFu, mine.R, 31 - __clz(below)) == R) continue;
+        const uint32_t members = __ballot_sync(0xFFFFFFFFu, mine.R == R);
+        const int lo_b = __shfl_sync(0xFFFFFFFFu, mine.lo, s0), hi_b = __shfl_sync(0xFFFFFFFFu, mine.hi, 31 - __clz(members));
+        const int si = step_of(q, R);
         const int rt = R - q.tile_start[si];
         const bool f16 = (q.f16_mask >> si) & 1;
         const int nval = 32 * batch;                 // values of the row tile: [row][batch column]
@@ -549,14 +594,15 @@ stack_kernel(const __grid_constant__ StackParams P) {
         float* gp = nullptr;
         int share = 1;
         if (!whole) {
+          const long long T = (long long)Rall * nb;
+          const int Ge = dealt_ctas(Rall, nb, false, G);
           const int c_first = owner_of((long long)R * nb, T, Ge), c_last = owner_of((long long)(R + 1) * nb - 1, T, Ge);
           share = c_last - c_first + 1;
           gp = P.gpart + ((size_t)R * P.max_share + (size_t)(cta - c_first)) * P.part_floats;
         }
         for (int v = lane; v < nval; v += 32) {
           float sum = 0.0f;
-          for (int s = s0; s <= s1; ++s)
-            if (pslot[s].R == R) sum += pdata[(size_t)s * P.part_floats + v];
+          for (uint32_t mm = members; mm != 0u; mm &= mm - 1u) sum += pdata[(size_t)(__ffs(mm) - 1) * P.part_floats + v];
           if (whole) {
             const int row = rt * kTileRows + v / batch, bc = v % batch;
             if (row < q.n[si]) {
@@ -601,7 +647,7 @@ stack_kernel(const __grid_constant__ StackParams P) {
   }
 
   // ---- leaving: let copies in flight land, then the last CTA out restores the workspace ----
-  if (ctl[0] || failed) {
+  if (ctl[0] || W.failed) {
     const long long t0 = clock64();
     while (clock64() - t0 < 200000) {}
   }
@@ -648,10 +694,17 @@ static int check_step(const stb_step& s) {
   return STB_OK;
 }
 
-// most CTAs that share one row tile of a phase of R row tiles x nb blocks dealt to G CTAs
+// Whole row tiles per CTA when that keeps at least 85 % of the SM time busy: R row tiles on G CTAs take
+// ceil(R / G) rounds of which R / G are needed.
+static bool deal_aligned(long long R, int G) {
+  const long long rounds = (R + G - 1) / G;
+  return (double)R / (double)G >= 0.85 * (double)rounds;
+}
+
+// most CTAs that share one row tile of a phase of R row tiles x nb blocks dealt to G CTAs by equal tile counts
 static uint32_t max_share_of(long long R, int nb, int G) {
   const long long T = R * nb;
-  const int Ge = dealt_ctas(T, G);
+  const int Ge = dealt_ctas((int)R, nb, false, G);
   uint32_t best = 1;
   for (long long r = 0; r < R; ++r) {
     const int c0 = owner_of(r * nb, T, Ge), c1 = owner_of((r + 1) * nb - 1, T, Ge);
@@ -704,13 +757,14 @@ static int build_phases(const stb_step* steps, int count, int i0, int G, StackPa
     for (int k = q.count; k < kMaxFusedSteps; ++k) q.tile_start[k + 1] = q.tile_start[q.count];
     q.x = static_cast<const __half*>(st.in);
     q.ldx = (uint32_t)st.ldin; q.m = st.m; q.N = (uint8_t)st.N; q.batch = (uint8_t)st.batch;
-    q.use_image = 0; q.pad[0] = q.pad[1] = q.pad[2] = 0;
+    q.use_image = 0; q.pad[0] = q.pad[1] = 0;
     q.done_before = done;
     const long long R = q.tile_start[q.count];
     done += (uint32_t)R;
     if (R > maxR) maxR = R;
     if ((uint32_t)(32 * st.batch) > sp.part_floats) sp.part_floats = (uint32_t)(32 * st.batch);
-    const uint32_t share = max_share_of(R, st.m / kBlock, G);
+    q.aligned = deal_aligned(R, G) ? 1 : 0;
+    const uint32_t share = q.aligned ? 1u : max_share_of(R, st.m / kBlock, G);
     if (share > sp.max_share) sp.max_share = share;
     ++sp.nphase;
     i = j;

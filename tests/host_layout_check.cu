@@ -181,21 +181,26 @@ static int check(int trials, int spb) {
         static const Meta6Table meta = make_meta6_table();
         LaneTile<N> raw;
         load_lane_tile<N>(tile.data(), lane, raw, true);
+        static const Meta6Joint joint = make_meta6_joint();
         for (int bb = 0; bb < 2; ++bb) {
-          uint32_t en[2][4], E[3];
-          for (int tq = 0; tq < 4; ++tq)
-            for (int rp = 0; rp < 2; ++rp) {
-              const uint32_t off = prmt(raw.mask[2 * bb + (tq >> 1)], 0u, 0x4440u + (uint32_t)(2 * (tq & 1) + rp));
-              if (off % 4 != 0 || off / 4 >= 28) { ++errors; continue; }
-              en[rp][tq] = meta.v[off / 4];
-            }
+          uint32_t en[2][4], E[3], EJ[3] = {0, 0, 0};
+          for (int tq = 0; tq < 4; ++tq) {
+            // the pair field of lane tq's slot: two keep-mask indices (one way), or the joint-table entry (the other)
+            const uint32_t f = (raw.mask[2 * bb + (tq >> 1)] >> (16 * (tq & 1))) & 0xFFFFu;
+            if (f % 16 != 0 || f / 16 >= kMasks6 * kMasks6) { ++errors; continue; }
+            en[0][tq] = meta.v[pair_field_index(f, 0)];
+            en[1][tq] = meta.v[pair_field_index(f, 1)];
+            for (int i = 0; i < 3; ++i) EJ[i] += joint.v[f / 16][i] << (4 * tq);
+          }
           meta6_words(en, E);
-          for (int i = 0; i < 3; ++i)
+          for (int i = 0; i < 3; ++i) {
+            if (E[i] != EJ[i]) { if (++errors < 10) std::printf("joint metadata word N=%d\n", N); }
             for (int tq = 0; tq < 4; ++tq)
               for (int rp = 0; rp < 2; ++rp) {
                 const int r = g + 16 * (t >> 1) + 8 * rp, grp = 4 * (2 * (t & 1) + bb) + tq;
                 if (((E[i] >> (4 * tq + 16 * rp)) & 0xFu) != meta6_nibble(keep[r][grp], i)) { if (++errors < 10) std::printf("metadata word N=%d\n", N); }
               }
+          }
         }
       }
       if constexpr (N >= 4 && N <= 6) {
