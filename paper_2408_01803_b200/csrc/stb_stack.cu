@@ -100,6 +100,17 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const void* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+// product of two fp16 pairs given and returned as bit patterns
+__device__ __forceinline__ uint32_t hmul2_bits(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
 __device__ __forceinline__ uint4 ld_v4(const void* p) {      // coherent load (the activations are written by this kernel)
   uint4 v;
   asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
@@ -394,16 +405,18 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
             a2 = *reinterpret_cast<const uint2*>(rec + resid_a2_off(g, 0));
             rw = *reinterpret_cast<const uint32_t*>(rec + resid_code_off(e.x & 7u, g));
           }
+          // operand registers of the lane's four rows: the two-bit codes pick the high byte of +1, 0 or -1 (one byte
+          // permute per row), two more spread them to fp16 pairs, and one fp16 multiply per register (not on the
+          // busy integer pipe) scales them by the row's a_sal2: exact, the factors are +-1 and 0
           uint32_t fa[4][2];
+          const uint32_t code_lo = rw & 0x33333333u, code_hi = (rw >> 2) & 0x33333333u;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const uint32_t h = (((j & 2) ? a2.y : a2.x) >> (16 * (j & 1))) & 0xFFFFu;
-            const uint32_t L2 = prmt(h, 0u, 0x4040u);                 // (lo, 0, lo, 0)
-            const uint32_t H2 = prmt(h, h ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
-            const uint32_t sel = resid_selector(rw, j);
-            const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
-            fa[j][0] = prmt(lo4, hi4, 0x5140u);
-            fa[j][1] = prmt(lo4, hi4, 0x7362u);
+            const uint32_t codes = (j & 2) ? code_hi : code_lo;
+            const uint32_t unit = prmt(0x00BC003Cu, 0u, (j & 1) ? (codes >> 16) : codes);          // high bytes of +1, 0, -1, 0 by code
+            const uint32_t s2 = prmt((j & 2) ? a2.y : a2.x, 0u, (j & 1) ? 0x3232u : 0x1010u);     // (a_sal2, a_sal2) of row j
+            fa[j][0] = hmul2_bits(prmt(unit, 0u, 0x1404u), s2);
+            fa[j][1] = hmul2_bits(prmt(unit, 0u, 0x3424u), s2);
           }
           uint2 xr = make_uint2(0, 0);
           if (xg) {
@@ -513,8 +526,11 @@ stack_kernel(const __grid_constant__ StackParams P) {
     // ---- wait until every earlier phase has finished, then (6:8) lay the activations out in operand order ----
     if (threadIdx.x == 0 && !ctl[0] && q.done_before > 0) {
       const long long t0 = clock64();
-      while (ld_acquire_u32(P.sync) < q.done_before) {
-        if (ld_acquire_u32(P.sync + 1) != 0u) { ctl[0] = 1; break; }
+      for (;;) {
+        // one load brings the count of finished row tiles (low word) and the abort flag (high word)
+        const unsigned long long v = ld_acquire_u64(P.sync);
+        if ((uint32_t)v >= q.done_before) break;
+        if ((uint32_t)(v >> 32) != 0u) { ctl[0] = 1; break; }
         if (clock64() - t0 > P.wait_limit) {
           ctl[0] = 1;
           atomicExch(P.sync + 1, 1u);
