@@ -136,18 +136,24 @@ int stb_gemv_wait_selftest(const void *packed, int n, int m, int N, const void *
                            size_t ldx, void *y, stb_dtype ydt, size_t ldy, int *dev_status,
                            void *stream);
 
-/* Bytes of workspace stb_gemm wants for T tokens (0 if none).  HOST result.  Two cases ask for one:
- * few output tiles (every tile is then split along K and the partial tiles are summed afterwards:
- * the workspace is required), and many output tiles whose last wave of 148 would be small (only
- * that wave's tiles are split: the workspace is optional, without it those tiles run unsplit). */
+/* Bytes of workspace stb_gemm wants for T tokens.  HOST result.  The workspace always holds the
+ * activations of the residual slots, gathered per call (T x m / 4 bf16: room for 32 salient columns in
+ * every block).  Beyond that, two cases add fp32 partial tiles: few output tiles (every tile is then
+ * split along K and the partial tiles are summed afterwards: required), and many output tiles whose
+ * last wave of 148 would be small (only that wave's tiles are split: optional, without it those tiles
+ * run unsplit).  stb_gemm_workspace gives the size with the optional part, stb_gemm_workspace_min the
+ * size stb_gemm cannot do without. */
 int stb_gemm_workspace(int n, int m, int N, int T, size_t *bytes);
+int stb_gemm_workspace_min(int n, int m, int N, int T, size_t *bytes);
 
 /* Prefill GEMM:  Y[t][i] = sum_j W^[i][j] * X[t][j]  on the tensor cores (tcgen05, fp32
- * accumulation in tensor memory); W^ is decoded tile by tile to bf16 (RN-even).
+ * accumulation in tensor memory); W^ is decoded tile by tile to bf16 (RN-even): a kept weight is
+ * s bf16(a_region), a kept salient weight s1 bf16(a_sal1) + s2 bf16(a_sal2) with the second term
+ * multiplied in as extra K (Eq. 4: the two binarizations of a salient weight are two terms).
  * X: bf16 [T][ldx]; Y: fp32 or bf16 [T][ldy] (ydt).  The compute-bound case of Appendix C.2
- * (prefilling stage, N = sequence length x batch).  ws / ws_bytes: caller-owned workspace of
- * stb_gemm_workspace bytes (may be NULL when that is 0).  A smaller or missing workspace gives
- * STB_ERR_SIZE when the split is required and the unsplit launch when it is optional. */
+ * (prefilling stage, N = sequence length x batch).  ws / ws_bytes: caller-owned workspace, 256-byte
+ * aligned, of at least stb_gemm_workspace_min bytes (else STB_ERR_SIZE); with stb_gemm_workspace
+ * bytes the optional split is used too.  Three launches at most: gather, GEMM, sum of partial tiles. */
 int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size_t ldx, void *Y,
              stb_dtype ydt, size_t ldy, void *ws, size_t ws_bytes, int *dev_status,
              void *stream);
@@ -156,16 +162,16 @@ int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size
  * for the integration, not for the method).  Some hosts of this library may not allocate device
  * memory while they run: a serving process that gave its whole memory budget to one arena at
  * start-up, or a latency-critical loop in which a cudaMalloc (which synchronises the device)
- * is forbidden.  For them the split-K partial sums go into a fixed 8 MiB array that is part of
- * the library image: every GPU that loads the library holds these 8 MiB until the process
+ * is forbidden.  For them stb_gemm's workspace (gathered residual activations, split-K partial
+ * sums) is a fixed 8 MiB array that is part of the library image: every GPU that loads the library holds these 8 MiB until the process
  * exits.  Same arguments, results and errors as stb_gemm, except:
- *   - a call whose required workspace (see stb_gemm_workspace) exceeds 8 MiB returns
+ *   - a call whose required workspace (see stb_gemm_workspace_min) exceeds 8 MiB returns
  *     STB_ERR_SIZE and launches nothing (use stb_gemm with your own workspace for it); an
- *     optional split is used only if its partial tiles fit the array;
+ *     optional split is used only if its partial tiles fit the array too;
  *   - the first call on each device looks the array's device address up (with that device
  *     current); make that first call outside any stream capture;
  *   - all calls share the one array.  It keeps whatever the last call left there; nothing in
- *     it has to start at zero, because every call writes each partial sum before reading it.
+ *     it has to start at zero, because every call writes what it reads there before reading it.
  *     Two calls that may run on the GPU at the same time (different streams) would overwrite
  *     each other's partial sums: keep calls of this entry point on one stream, or order them.
  * It calls no allocation routine of CUDA or of any library. */

@@ -21,7 +21,7 @@ STB_ERR_UNSUPPORTED, STB_ERR_CORRUPT, STB_ERR_TIMEOUT, STB_ERR_CUDA = 5, 6, 7, 8
 STB_F16, STB_BF16, STB_F32 = 0, 1, 2
 
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
-           "stb_gemm_workspace", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
+           "stb_gemm_workspace", "stb_gemm_workspace_min", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
            "stb_layer_stack_resident_workspace", "stb_layer_stack_resident", "stb_layer_stack_resident_host",
            "stb_layer_stack_resident_wait_selftest", "stb_status_str"]
 
@@ -62,6 +62,7 @@ def _load():
     lib.stb_gemv.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_gemv_wait_selftest.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_gemm_workspace.argtypes = [i, i, i, i, p(z)]
+    lib.stb_gemm_workspace_min.argtypes = [i, i, i, i, p(z)]
     lib.stb_gemm.argtypes = [v, i, i, i, v, i, z, v, i, z, v, z, v, v]
     lib.stb_gemm_noalloc.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_layer_stack.argtypes = [p(_Step), i, v, v]
@@ -196,9 +197,10 @@ def gemv_wait_selftest(layer: PackedLayer, x, out, dev_status, stream=None):
                                        _stream(stream)), "stb_gemv_wait_selftest")
 
 
-def gemm_workspace(n, m, N, T) -> int:
+def gemm_workspace(n, m, N, T, minimum=False) -> int:
     out = C.c_size_t()
-    _check(_lib.stb_gemm_workspace(n, m, N, T, C.byref(out)), "stb_gemm_workspace")
+    fn = _lib.stb_gemm_workspace_min if minimum else _lib.stb_gemm_workspace
+    _check(fn(n, m, N, T, C.byref(out)), "stb_gemm_workspace")
     return out.value
 
 

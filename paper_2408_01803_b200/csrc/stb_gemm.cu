@@ -20,6 +20,10 @@
 //               (RN-even) and writes the two 64-column halves of the block into two stages;
 //               afterwards the same warps read the accumulator (TMEM lanes 32 (w % 4) ..) and
 //               store Y.
+// The residual term of the salient columns (Eq. 4) is more K: a small kernel first gathers the activations of
+// every residual slot (four per residual word, in word order) into Xs[token][slot]; after the blocks of its K
+// range a CTA runs the residual slots of those blocks as further stages, A = +-bf16(a_sal2) or 0 by the two-bit
+// residual codes, B = Xs through a second tensor map.  The main stages give a salient weight s1 bf16(a_sal1).
 // One CTA fits an SM, so the grid runs in waves of 148 output tiles; tiles of a small last wave
 // (and all tiles when there are few) are split along K into fp32 partial tiles in the caller's
 // workspace and summed by a second kernel.
@@ -127,6 +131,8 @@ struct DecodeArgs {
   const uint8_t* packed; const Header* hdr; uint8_t* smem; volatile int* abort_flag;
   uint32_t bar_full, bar_empty;
   int mt, b0, b1, nblk, ntile, q, lane;
+  uint32_t rw0, rw1;        // residual words of the blocks [b0, b1)
+  int nres;                 // residual stages (64 slots = 16 words each, the first one starts at word rw0 & ~1)
 };
 
 // Decode role of one warp: row j (of the four rows g + 8 j each lane owns) of packed row tile 4 mt + q, for
@@ -155,26 +161,12 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
                             (size_t)rtile * resid_rt_bytes(nblk, hdr->nrw);
   constexpr uint32_t tbytes = tile_bytes(N);
   RowWords cur = {}, nxt = {};
-  // salient metadata of a block, fetched one block ahead like the row's words: the count, and for the
-  // lane's slots t, t + 4 (slots beyond 8 are fetched on demand) the column bytes and residual words
-  struct Sal { int nsal; const uint8_t* rec; uint32_t a2; uint32_t cw[2], rw[2]; };
-  auto load_sal = [&](int b, Sal& z) {
-    z.nsal = (int)__ldg(&binfo[b].nsal);
-    z.rec = resid_rt + resid_block_off(b, __ldg(&binfo[b].rw_off));       // the block's record of the residual stream
-    z.a2 = __ldg(reinterpret_cast<const uint16_t*>(z.rec + resid_a2_off(g, j)));
-    z.cw[0] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols));
-    z.cw[1] = __ldg(reinterpret_cast<const uint32_t*>(binfo[b].cols) + 1);
-    z.rw[0] = z.nsal > 0 ? __ldg(reinterpret_cast<const uint32_t*>(z.rec + resid_code_off(0u, g))) : 0x55555555u;
-    z.rw[1] = z.nsal > 4 ? __ldg(reinterpret_cast<const uint32_t*>(z.rec + resid_code_off(1u, g))) : 0x55555555u;
-  };
-  Sal csal = {0, nullptr, 0u, {0, 0}, {0, 0}}, nsalv = {0, nullptr, 0u, {0, 0}, {0, 0}};
-  if (live && b0 < b1) { load_row_words<N>(rtbase + (size_t)b0 * tbytes, lane, j, cur); load_sal(b0, csal); }
+  if (live && b0 < b1) load_row_words<N>(rtbase + (size_t)b0 * tbytes, lane, j, cur);
   bool ok = true;
   for (int b = b0; b < b1 && ok; ++b) {
-    if (live && b + 1 < b1) { load_row_words<N>(rtbase + (size_t)(b + 1) * tbytes, lane, j, nxt); load_sal(b + 1, nsalv); }
-    // bf16 scale bytes of the row
+    if (live && b + 1 < b1) load_row_words<N>(rtbase + (size_t)(b + 1) * tbytes, lane, j, nxt);
+    // bf16 scale bytes of the row (a salient weight gets s1 bf16(a_sal1) here; its residual term comes with the residual stages)
     uint32_t A16 = 0, B16 = 0;
-    float a1f = 0.f, a2f = 0.f;
     if (live) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
@@ -182,29 +174,18 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
         const uint32_t v = bf16_bits(h16);
         A16 |= (v & 0xFFu) << (8 * c);
         B16 |= (v >> 8) << (8 * c);
-        if (c == 3) a1f = __half2float(__ushort_as_half((unsigned short)h16));
       }
-      a2f = __half2float(__ushort_as_half((unsigned short)csal.a2));
     }
     OneRow<N> row;
     row.init(cur, j, A16, B16);
-    const int nsal = live ? csal.nsal : 0;
     // position selectors of the row's slots of this block, looked up before the stage waits
     uint32_t P[4];
 #pragma unroll
     for (int sidx = 0; sidx < 4; ++sidx) P[sidx] = live ? ptab[(cur.mask >> (8 * sidx)) & 0xFFu] : 0u;
-    // Salient patches of this block: one per salient slot sq, dealt to the four lanes t of a lane
-    // group; the first one per lane is prepared here.
-    int pc0 = -1; uint32_t prc0 = 1u;          // column and residual code of patch t
-    if (t < nsal) {
-      const int sq = t;
-      pc0 = (int)((csal.cw[0] >> (8 * (sq & 3))) & 0xFFu);
-      prc0 = resid_code(csal.rw[0], j, sq & 3);
-    }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int it = 2 * (b - b0) + h, st = it % kStages;
-      // the verdict is made warp-uniform: nobody may be left alone at the __syncwarp()s below
+      // the verdict is made warp-uniform: nobody may be left alone at the __syncwarp() below
       if (!__all_sync(0xFFFFFFFFu, gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
       uint8_t* As = smem + kGemmA + st * kStageA;
       uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
@@ -217,40 +198,80 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
         const int chunk = 4 * sl + t;                      // 16-byte chunk of the 128-byte row
         *reinterpret_cast<uint4*>(rowp + ((chunk ^ g) << 4)) = make_uint4(f[0], f[1], f[2], f[3]);
       }
-      // salient columns: bf16( fl32( s1 a_sal1 + s2 a_sal2 ) ) replaces the value the main decode
-      // wrote (whose sign is s1); patch p = t + 4 i of the block's list belongs to lane t
-      if (nsal > 0) {
-        __syncwarp();
-        for (int p = t; p < nsal; p += 4) {
-          int c = pc0; uint32_t rc = prc0;
-          if (p >= 4) {
-            const int sq = p;
-            c = binfo[b].cols[sq];
-            const uint32_t word = sq < 8 ? csal.rw[1] :
-                __ldg(reinterpret_cast<const uint32_t*>(csal.rec + resid_code_off((uint32_t)(sq >> 2), g)));
-            rc = resid_code(word, j, sq & 3);
-          }
-          if ((c >> 6) != h || rc == 1u) continue;
-          const int c64 = c & 63;
-          unsigned short* pv = reinterpret_cast<unsigned short*>(rowp + (((c64 >> 3) ^ g) << 4) + (c64 & 7) * 2);
-          const bool neg1 = (*pv & 0x8000u) != 0;
-          const float v = __fadd_rn(neg1 ? -a1f : a1f, rc == 0u ? a2f : -a2f);
-          *pv = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-        }
-      }
       fence_async_smem();          // generic-proxy writes -> visible to the tensor core
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_full + 8 * st);
     }
     if (!ok) break;
-    if (live && b + 1 < b1) { cur = nxt; csal = nsalv; }
+    if (live && b + 1 < b1) cur = nxt;
+  }
+
+  // Residual stages: 64 residual slots (16 residual words) of K each.  The lane writes the same two 16-byte chunks
+  // of its row as above: chunk c holds the words 2 c and 2 c + 1 of the stage, four slots each, as +-bf16(a_sal2) or 0.
+  const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + rwtab_offset(nblk));
+  const uint32_t wfirst = da.rw0 & ~1u;
+  for (int rs = 0; rs < da.nres && ok; ++rs) {
+    const int it = 2 * (b1 - b0) + rs, st = it % kStages;
+    uint32_t f[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+#pragma unroll
+    for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const uint32_t w = wfirst + 16u * (uint32_t)rs + 2u * (uint32_t)(4 * sl + t) + (uint32_t)k;
+        if (live && w >= da.rw0 && w < da.rw1) {
+          const uint2 e = __ldg(reinterpret_cast<const uint2*>(rwt + w));
+          const uint8_t* rec = resid_rt + resid_block_off((int)(e.x >> 3), w - (e.x & 7u));
+          const uint32_t v = bf16_bits(__ldg(reinterpret_cast<const uint16_t*>(rec + resid_a2_off(g, j))));
+          const uint32_t word = __ldg(reinterpret_cast<const uint32_t*>(rec + resid_code_off(e.x & 7u, g)));
+          const uint32_t L2 = prmt(v, 0u, 0x4040u);                 // (lo, 0, lo, 0)
+          const uint32_t H2 = prmt(v, v ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
+          const uint32_t sel = resid_selector(word, j);
+          const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
+          f[sl][2 * k] = prmt(lo4, hi4, 0x5140u);
+          f[sl][2 * k + 1] = prmt(lo4, hi4, 0x7362u);
+        }
+      }
+    if (!__all_sync(0xFFFFFFFFu, gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
+    uint8_t* rowp = smem + kGemmA + st * kStageA + (size_t)(4 * q + j) * 1024 + g * 128;
+#pragma unroll
+    for (int sl = 0; sl < 2; ++sl)
+      *reinterpret_cast<uint4*>(rowp + (((4 * sl + t) ^ g) << 4)) = make_uint4(f[sl][0], f[sl][1], f[sl][2], f[sl][3]);
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_full + 8 * st);
+  }
+}
+
+// Gathers the activations of the residual slots: Xs[t][4 w + k] = X[t][128 block(w) + cols(w)[k]] for every residual
+// word w of the layer, and zeros in the 128 columns after the last word (a CTA's last residual stage may reach there).
+__global__ void gemm_gather_kernel(const uint8_t* __restrict__ packed, int n, int m, int N, const __nv_bfloat16* __restrict__ X, int T,
+                                   size_t ldx, __nv_bfloat16* __restrict__ Xs, int ldxs) {
+  const Header* hdr = reinterpret_cast<const Header*>(packed);
+  if (!header_matches(hdr, n, m, N)) return;
+  const int nblk = m / kBlock;
+  const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + rwtab_offset(nblk));
+  const uint32_t nrw = hdr->nrw;
+  uint32_t W = nrw + 32u;                                   // words written per token: the layer's and 32 of zeros
+  if (W > (uint32_t)ldxs / 4u) W = (uint32_t)ldxs / 4u;
+  const size_t total = (size_t)T * W;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t t = i / W;
+    const uint32_t w = (uint32_t)(i % W);
+    uint2 out = make_uint2(0u, 0u);
+    if (w < nrw) {
+      const uint2 e = __ldg(reinterpret_cast<const uint2*>(rwt + w));
+      const unsigned short* xr = reinterpret_cast<const unsigned short*>(X + t * ldx + (size_t)(e.x >> 3) * kBlock);
+      out.x = (uint32_t)xr[e.y & 0xFFu] | ((uint32_t)xr[(e.y >> 8) & 0xFFu] << 16);
+      out.y = (uint32_t)xr[(e.y >> 16) & 0xFFu] | ((uint32_t)xr[e.y >> 24] << 16);
+    }
+    *reinterpret_cast<uint2*>(Xs + t * (size_t)ldxs + 4u * w) = out;
   }
 }
 
 // ------------------------------------------------------------------------------------------
 template <int N>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict__ packed, int n, int m, int T,
+gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap xsmap, const uint8_t* __restrict__ packed, int n, int m, int T,
             void* __restrict__ Y, int y_bf16, size_t ldy, float* __restrict__ ws, int full_tiles, int ksplit, int bps,
             int ttiles, uint32_t box_bytes, int* dev_status) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -269,7 +290,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
   const int kz = split ? (cta - full_tiles) % ksplit : 0;
   const int tt = tile % ttiles, mt = tile / ttiles;
   const int b0 = split ? kz * bps : 0, b1 = split ? min(nblk, b0 + bps) : nblk;
-  const int nstage = 2 * max(b1 - b0, 0);              // 64-column stages of this CTA
+  // residual words of the CTA's blocks -> residual stages of 16 words, the first one starting at an even word
+  const BlockInfo* binfo_k = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+  uint32_t rw0 = 0, rw1 = 0;
+  if (b0 < b1) { rw0 = __ldg(&binfo_k[b0].rw_off); rw1 = b1 < nblk ? __ldg(&binfo_k[b1].rw_off) : hdr->nrw; }
+  const int nres = rw1 > rw0 ? (int)((rw1 - (rw0 & ~1u) + 15u) / 16u) : 0;
+  const int nmain = 2 * max(b1 - b0, 0);               // 64-column stages of the blocks
+  const int nstage = nmain + nres;
 
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar_full = sbase + kGemmBars, bar_empty = bar_full + 8 * kStages, bar_accum = bar_empty + 8 * kStages;
@@ -299,8 +326,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
         if (!gemm_wait<true>(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) break;
         mbar_expect_tx(bar_full + 8 * s, box_bytes * kAcc);
 #pragma unroll
-        for (int a = 0; a < kAcc; ++a)
-          tma_load_2d(sbase + kGemmB + s * kStageB + a * (kBN * kBK * 2), &xmap, (b0 * 2 + it) * kBK, tt * kTok + a * kBN, bar_full + 8 * s);
+        for (int a = 0; a < kAcc; ++a) {
+          const uint32_t dst = sbase + kGemmB + s * kStageB + a * (kBN * kBK * 2);
+          if (it < nmain) tma_load_2d(dst, &xmap, (b0 * 2 + it) * kBK, tt * kTok + a * kBN, bar_full + 8 * s);
+          else tma_load_2d(dst, &xsmap, (int)(4u * (rw0 & ~1u)) + (it - nmain) * kBK, tt * kTok + a * kBN, bar_full + 8 * s);
+        }
       }
       if (*abort_flag) {       // let copies in flight land before the CTA gives its shared memory up
         const long long t0 = clock64();
@@ -333,6 +363,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const uint8_t* __restrict_
     da.packed = packed; da.hdr = hdr; da.smem = smem; da.abort_flag = abort_flag;
     da.bar_full = bar_full; da.bar_empty = bar_empty;
     da.mt = mt; da.b0 = b0; da.b1 = b1; da.nblk = nblk; da.ntile = ntile; da.q = warp & 3; da.lane = lane;
+    da.rw0 = rw0; da.rw1 = rw1; da.nres = nres;
     decode_row<N>(da, gi);
 
     // ---------------- epilogue: TMEM -> registers -> Y ----------------
@@ -454,23 +485,42 @@ static EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+// Bytes of the gathered activations Xs[T][m / 4] (bf16) at the head of the workspace: room for the most residual
+// slots a layer can have (32 per block), so that the size depends on the shape alone.
+static size_t gemm_xs_bytes(int m, int T) { return (((size_t)T * (size_t)(m / 4) * 2u) + 255u) & ~(size_t)255u; }
+
 template <int N>
 static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T, size_t ldx, void* Y, int y_bf16,
                        size_t ldy, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t s) {
-  const GemmPlan plan = gemm_plan(n, m, T, ws_bytes, ws != nullptr);
-  if (plan.mandatory_bytes > 0 && (!ws || ws_bytes < plan.mandatory_bytes)) return STB_ERR_SIZE;
+  const size_t xs_bytes = gemm_xs_bytes(m, T);
+  if (ws && (reinterpret_cast<uintptr_t>(ws) & 255u)) return STB_ERR_ARG;
+  if (!ws || ws_bytes < xs_bytes) return STB_ERR_SIZE;
+  float* ws_split = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + xs_bytes);
+  const GemmPlan plan = gemm_plan(n, m, T, ws_bytes - xs_bytes, true);
+  if (plan.mandatory_bytes > ws_bytes - xs_bytes) return STB_ERR_SIZE;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return STB_ERR_CUDA;
-  CUtensorMap map;
-  const cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)T};
-  const cuuint64_t strides[1] = {(cuuint64_t)ldx * 2};
   const cuuint32_t box_rows = (cuuint32_t)(T < kBN ? T : kBN);
   const cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return STB_ERR_ARG;
+  CUtensorMap map, xsmap;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)T};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * 2};
+    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return STB_ERR_ARG;
+  }
+  const int ldxs = m / 4;                     // a multiple of 32 elements: rows of Xs start on 64-byte boundaries
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)ldxs, (cuuint64_t)T};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldxs * 2};
+    if (enc(&xsmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ws, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return STB_ERR_ARG;
+  }
   // the shared-memory limit of a kernel is a per-device setting
   static bool attr_done[64] = {};
   int dev = 0;
@@ -479,12 +529,15 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
     if (cudaFuncSetAttribute(gemm_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem) != cudaSuccess) return STB_ERR_CUDA;
     if (dev >= 0 && dev < 64) attr_done[dev] = true;
   }
+  gemm_gather_kernel<<<148 * 4, 256, 0, s>>>(packed, n, m, N, static_cast<const __nv_bfloat16*>(X), T, ldx,
+                                             static_cast<__nv_bfloat16*>(ws), ldxs);
+  if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   const unsigned grid = (unsigned)(plan.full_tiles + plan.split_tiles * plan.ksplit);
-  gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, packed, n, m, T, Y, y_bf16, ldy, static_cast<float*>(ws), plan.full_tiles,
+  gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, xsmap, packed, n, m, T, Y, y_bf16, ldy, ws_split, plan.full_tiles,
                                               plan.ksplit, plan.bps, plan.ttiles, box_rows * kBK * 2, dev_status);
   if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   if (plan.split_tiles > 0) {
-    gemm_reduce_kernel<<<148 * 4, 256, 0, s>>>(static_cast<const float*>(ws), plan.full_tiles, plan.split_tiles, plan.ksplit,
+    gemm_reduce_kernel<<<148 * 4, 256, 0, s>>>(ws_split, plan.full_tiles, plan.split_tiles, plan.ksplit,
                                                plan.ttiles, n, T, Y, y_bf16, ldy);
     if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   }
@@ -493,13 +546,17 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
 
 }  // namespace stb
 
-extern "C" int stb_gemm_workspace(int n, int m, int N, int T, size_t* bytes) {
+static int gemm_workspace_impl(int n, int m, int N, int T, size_t* bytes, bool minimum) {
   if (!bytes) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0 || T < 1) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
-  *bytes = stb::gemm_plan(n, m, T, 0, false).preferred_bytes;
+  const stb::GemmPlan plan = stb::gemm_plan(n, m, T, 0, false);
+  *bytes = stb::gemm_xs_bytes(m, T) + (minimum ? plan.mandatory_bytes : plan.preferred_bytes);
   return STB_OK;
 }
+
+extern "C" int stb_gemm_workspace(int n, int m, int N, int T, size_t* bytes) { return gemm_workspace_impl(n, m, N, T, bytes, false); }
+extern "C" int stb_gemm_workspace_min(int n, int m, int N, int T, size_t* bytes) { return gemm_workspace_impl(n, m, N, T, bytes, true); }
 
 extern "C" int stb_gemm(const void* packed, int n, int m, int N, const void* X, int T, size_t ldx,
                         void* Y, stb_dtype ydt, size_t ldy, void* ws, size_t ws_bytes,
@@ -521,8 +578,9 @@ extern "C" int stb_gemm(const void* packed, int n, int m, int N, const void* X, 
 }
 
 // ------------------------------------------------------------------------------------------
-// stb_gemm_noalloc: stb_gemm for callers that can hand over no workspace.  The split-K partial
-// sums live in a fixed array inside the library image instead of a caller's buffer.
+// stb_gemm_noalloc: stb_gemm for callers that can hand over no workspace.  The gathered residual
+// activations and the split-K partial sums live in a fixed array inside the library image instead of
+// a caller's buffer.
 namespace stb {
 constexpr size_t kNoAllocScratchBytes = 8u << 20;                       // 8 MiB per device, resident until exit
 static __device__ __align__(256) float g_noalloc_scratch[kNoAllocScratchBytes / sizeof(float)];
@@ -536,8 +594,8 @@ extern "C" int stb_gemm_noalloc(const void* packed, int n, int m, int N, const v
   if (N < 4 || N > 6) return STB_ERR_UNSUPPORTED;
   if (ydt != STB_F32 && ydt != STB_BF16) return STB_ERR_UNSUPPORTED;
   if (ldx < (size_t)m || ldy < (size_t)n || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u)) return STB_ERR_ARG;
-  // this shape needs the caller-workspace entry point if the partial sums it cannot do without do not fit
-  if (stb::gemm_plan(n, m, T, 0, false).mandatory_bytes > stb::kNoAllocScratchBytes) return STB_ERR_SIZE;
+  // this shape needs the caller-workspace entry point if the scratch it cannot do without does not fit
+  if (stb::gemm_xs_bytes(m, T) + stb::gemm_plan(n, m, T, 0, false).mandatory_bytes > stb::kNoAllocScratchBytes) return STB_ERR_SIZE;
   // The array's name is only a host-side handle: ask the runtime for its address on the current
   // device, once per device, and give the kernels that address.
   static float* scratch_of_device[64] = {nullptr};

@@ -353,8 +353,9 @@ def test_gemm_splits_the_tiles_of_a_small_last_wave(stb):
     d = si.logical_layer(n, m, N, 612)
     L = oracle.Logical(**d)
     layer = stb.pack_numpy(d)
-    need = stb.gemm_workspace(n, m, N, T)
-    assert need == 2 * 2 * 128 * 512 * 4                       # two tiles, two parts each, fp32 partial tiles
+    need, least = stb.gemm_workspace(n, m, N, T), stb.gemm_workspace(n, m, N, T, minimum=True)
+    assert need - least == 2 * 2 * 128 * 512 * 4               # two tiles, two parts each, fp32 partial tiles
+    assert least == (T * (m // 4) * 2 + 255) // 256 * 256      # the gathered activations of the residual slots
     g = np.random.default_rng(5)
     rows = np.unique(np.concatenate([[0, 148 * 128 - 1, 148 * 128, 149 * 128 + 7, n - 1], g.choice(n, 64, replace=False)])).astype(np.int32)
     toks = np.arange(T)
@@ -362,8 +363,9 @@ def test_gemm_splits_the_tiles_of_a_small_last_wave(stb):
     x = torch.from_numpy(si.activations(T, m, 31, "bf16")).cuda().to(torch.bfloat16)
     y_split = stb.gemm(layer, x)
     y_whole = torch.empty(T, n, device="cuda")
+    ws_least = torch.empty(least, dtype=torch.uint8, device="cuda")
     stb._check(stb._lib.stb_gemm(stb._ptr(layer.buf), n, m, N, stb._ptr(x), T, m, stb._ptr(y_whole), stb.STB_F32, n,
-                                 None, 0, stb._ptr(layer.dev_status), stb._stream()), "stb_gemm")
+                                 stb._ptr(ws_least), least, stb._ptr(layer.dev_status), stb._stream()), "stb_gemm")
     torch.cuda.synchronize()
     assert int(layer.dev_status.item()) == 0
     a, b = y_split.double().cpu().numpy(), y_whole.double().cpu().numpy()
