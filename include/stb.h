@@ -81,7 +81,14 @@ typedef struct stb_info {
                              columns (rounded up) of the block; rows padded to a multiple of 32 */
 } stb_info;
 
-/* One step of stb_layer_stack: out[batch][n] = layer(in[batch][m]).  HOST struct. */
+/* How a step forms its input.  STB_IN_PLAIN: x = in.  STB_IN_SILU_MUL: x = fp16(silu(in) * in2),
+ * silu(v) = v / (1 + exp(-v)), evaluated in fp32: the gated activation that sits between the gate / up and
+ * the down projection of a LLaMA MLP (every FFN linear is structured-binary, Section 3; the activation
+ * between them is not part of the layer), applied while the down projection stages its activations, so that
+ * no extra pass over them is needed.  Only stb_layer_stack_resident takes STB_IN_SILU_MUL. */
+typedef enum stb_input { STB_IN_PLAIN = 0, STB_IN_SILU_MUL = 1 } stb_input;
+
+/* One step of stb_layer_stack: out[batch][n] = layer(x[batch][m]).  HOST struct. */
 typedef struct stb_step {
   const void *packed;
   int n, m, N;
@@ -90,6 +97,8 @@ typedef struct stb_step {
   stb_dtype odt;    /* STB_F32 or STB_F16 (fp32 sum rounded to nearest even) */
   int batch;
   size_t ldin, ldout;
+  const void *in2;  /* fp16 [batch][ldin], 16-byte aligned: second input of STB_IN_SILU_MUL, else NULL */
+  stb_input input;
 } stb_step;
 
 /* Upper bound of the packed size of an n x m layer at N:8 (the packed size depends on the

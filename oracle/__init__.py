@@ -185,6 +185,15 @@ def layer_rows(L: Logical, rows, x, nthreads=0):
     return y
 
 
+def silu_mul(a, b):
+    """fp16 values (as float64) of silu(a) * b evaluated in float64: the gated MLP activation (not from the paper)."""
+    a = _c(a, np.float64); b = _c(b, np.float64)
+    assert a.shape == b.shape
+    out = np.empty(a.shape, np.uint16)
+    lib().stbo_silu_mul(_p(a), _p(b), C.c_int(a.size), _p(out))
+    return out.view(np.float16).astype(np.float64)
+
+
 def average_bits(N, r_salient):
     return float(lib().stbo_average_bits(C.c_int(N), C.c_double(r_salient)))
 

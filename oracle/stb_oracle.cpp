@@ -497,6 +497,14 @@ double stbo_recon_error(const double* W, const float* What, int n, int m, const 
   return e;
 }
 
+// ---------------------------------------------------------------------------
+// Not from the paper: the gated activation of the LLaMA MLP, whose three linears the paper binarizes
+// (Section 4.1 evaluates LLaMA-1/2/3).  out[i] = fp16( silu(a[i]) * b[i] ), silu(v) = v / (1 + exp(-v)), float64.
+// The CUDA path can form the input of the down projection this way (STB_IN_SILU_MUL).
+void stbo_silu_mul(const double* a, const double* b, int n, uint16_t* out) {
+  for (int i = 0; i < n; ++i) out[i] = double_to_half_bits(a[i] / (1.0 + std::exp(-a[i])) * b[i]);
+}
+
 int stbo_hardware_threads() { return (int)std::max(1u, std::thread::hardware_concurrency()); }
 
 }  // extern "C"

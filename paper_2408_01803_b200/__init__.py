@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libstb.so")
 STB_OK, STB_ERR_ARG, STB_ERR_SHAPE, STB_ERR_NM, STB_ERR_SIZE = 0, 1, 2, 3, 4
 STB_ERR_UNSUPPORTED, STB_ERR_CORRUPT, STB_ERR_TIMEOUT, STB_ERR_CUDA = 5, 6, 7, 8
 STB_F16, STB_BF16, STB_F32 = 0, 1, 2
+STB_IN_PLAIN, STB_IN_SILU_MUL = 0, 1
 
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
            "stb_gemm_workspace", "stb_gemm_workspace_min", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
@@ -46,7 +47,7 @@ class _Info(C.Structure):
 class _Step(C.Structure):
     _fields_ = [("packed", C.c_void_p), ("n", C.c_int), ("m", C.c_int), ("N", C.c_int),
                 ("inp", C.c_void_p), ("out", C.c_void_p), ("odt", C.c_int), ("batch", C.c_int),
-                ("ldin", C.c_size_t), ("ldout", C.c_size_t)]
+                ("ldin", C.c_size_t), ("ldout", C.c_size_t), ("in2", C.c_void_p), ("input", C.c_int)]
 
 
 def _load():
@@ -236,16 +237,25 @@ def gemm_noalloc(layer: PackedLayer, X, out, stream=None):
 
 
 def make_steps(steps):
-    """Marshal a list of (layer, x, out) into the C array stb_layer_stack takes."""
+    """Marshal a list of (layer, x, out) or (layer, (gate, up), out) into the C array stb_layer_stack takes; a pair
+    as input means x = silu(gate) * up (STB_IN_SILU_MUL, stb_layer_stack_resident only)."""
     import torch
     arr = (_Step * len(steps))()
     for k, (layer, x, out) in enumerate(steps):
+        second = None
+        if isinstance(x, (tuple, list)):
+            x, second = x
         x2 = x if x.dim() == 2 else x.unsqueeze(0)
         o2 = out if out.dim() == 2 else out.unsqueeze(0)
         assert x2.dtype == torch.float16 and x2.stride(1) == 1 and o2.stride(1) == 1
+        in2, mode = 0, STB_IN_PLAIN
+        if second is not None:
+            s2 = second if second.dim() == 2 else second.unsqueeze(0)
+            assert s2.dtype == torch.float16 and s2.stride(1) == 1 and s2.stride(0) == x2.stride(0) and s2.shape == x2.shape
+            in2, mode = s2.data_ptr(), STB_IN_SILU_MUL
         odt = {torch.float32: STB_F32, torch.float16: STB_F16}[o2.dtype]
         arr[k] = _Step(layer.buf.data_ptr(), layer.n, layer.m, layer.N, x2.data_ptr(), o2.data_ptr(), odt,
-                       x2.shape[0], x2.stride(0), o2.stride(0))
+                       x2.shape[0], x2.stride(0), o2.stride(0), in2, mode)
     return arr
 
 

@@ -759,6 +759,8 @@ static bool can_fuse(const stb_step& a, const stb_step& b) {
 
 extern "C" int stb_layer_stack(const stb_step* steps, int count, int* dev_status, void* stream) {
   if (!steps || count < 0) return STB_ERR_ARG;
+  for (int k = 0; k < count; ++k)
+    if (steps[k].input != STB_IN_PLAIN) return STB_ERR_UNSUPPORTED;      // only the resident kernel forms inputs
   int i = 0;
   while (i < count) {
     const stb_step& st = steps[i];

@@ -15,6 +15,9 @@
 //     mma.sp.m16n8k32 place them (activations from an image of x in operand order in shared memory, built once
 //     per phase and CTA); 4:8 and 5:8 (and 6:8 when the image does not fit or for more than two batch rows)
 //     decode to position order for mma.m16n8k16 with the activations read through L1.
+//   * A step may take x = silu(in) * in2 (the gated activation between gate / up and down of an MLP): the CTA forms
+//     it while it stages the activations in shared memory, in operand order (6:8, up to two batch rows) or as a
+//     plain fp16 copy (everything else), and the tiles and the residual term read it from there.
 //   * The residual term of the salient columns (Eq. 4) is applied per span of up to five blocks from the span's
 //     records of the residual stream, brought into shared memory by one bulk copy while the span's tiles run.
 //   * Partial sums: a warp that covers a whole row tile writes y itself; the others leave their head / tail
@@ -59,17 +62,19 @@ struct StackPhase {
   int32_t n[kMaxFusedSteps];
   int32_t tile_start[kMaxFusedSteps + 1];     // row tiles of the phase: step i owns [tile_start[i], tile_start[i + 1])
   const __half* x;
+  const __half* x2;                           // second input of STB_IN_SILU_MUL, else null
   uint32_t ldx;
   int32_t m;
   uint8_t N, batch, count, f16_mask;          // f16_mask bit i: step i writes fp16
-  uint8_t use_image, aligned, pad[2];         // aligned: CTA ranges are whole row tiles
+  uint8_t use_image, aligned, pad[2];         // use_image: 0 activations from global memory, 1 operand-order image (6:8),
+                                              // 2 plain fp16 copy in shared memory; aligned: CTA ranges are whole row tiles
   uint32_t done_before;                       // row tiles finished by all earlier phases of this launch
 };
 
 struct StackParams {
   StackPhase ph[kMaxPhases];
   int32_t nphase;
-  uint32_t image_bytes;                       // shared memory set aside for the 6:8 activation image
+  uint32_t image_bytes;                       // shared memory set aside for the staged activations
   uint32_t part_floats;                       // floats per partial slot: 32 rows x largest batch
   uint32_t max_share;                         // most CTAs that share one row tile
   uint32_t* sync;                             // [0] finished row tiles, [1] abort flag, [2] CTAs that left, [4..] per row tile arrivals
@@ -111,15 +116,39 @@ __device__ __forceinline__ uint32_t hmul2_bits(uint32_t a, uint32_t b) {
   asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
   return d;
 }
-__device__ __forceinline__ uint4 ld_v4(const void* p) {      // coherent load (the activations are written by this kernel)
+// Coherent loads of activations (written by this kernel, so never through the read-only path); the address may be
+// global or shared memory.
+__device__ __forceinline__ uint4 ld_v4(const void* p) {
   uint4 v;
-  asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  asm volatile("ld.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ uint32_t ld_u16(const void* p) {
   unsigned short v;
-  asm volatile("ld.global.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
+  asm volatile("ld.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
   return v;
+}
+// fp16 pair (bits) of silu(a) * b per half, in fp32, rounded to nearest even
+__device__ __forceinline__ uint32_t silu_mul_bits(uint32_t a, uint32_t b) {
+  const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&a)), fb = __half22float2(*reinterpret_cast<const __half2*>(&b));
+  const __half2 r = __floats2half2_rn(fa.x / (1.0f + __expf(-fa.x)) * fb.x, fa.y / (1.0f + __expf(-fa.y)) * fb.y);
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
+// the staged form of eight activations: as they are, or silu(in) * in2
+__device__ __forceinline__ uint4 staged_x(const __half* x, const __half* x2, size_t off) {
+  uint4 v = ld_v4(x + off);
+  if (x2) {
+    const uint4 w = ld_v4(x2 + off);
+    v.x = silu_mul_bits(v.x, w.x); v.y = silu_mul_bits(v.y, w.y); v.z = silu_mul_bits(v.z, w.z); v.w = silu_mul_bits(v.w, w.w);
+  }
+  return v;
+}
+// Activation of column c (0..127) of block blk from the operand-order image of one batch row (see the image build).
+__device__ __forceinline__ uint32_t image_x(const uint32_t* img_row, uint32_t blk, uint32_t c) {
+  const uint32_t Gp = c >> 3, pr = (c >> 1) & 3u;
+  const uint32_t* d = img_row + blk * kImgWordsPerBlock + (4u * (Gp & 1u) + ((Gp >> 2) & 1u)) * 12u + 2u * (Gp >> 3) + ((Gp >> 1) & 1u);
+  const uint32_t w = d[pr < 3u ? 4u * pr : 32u];
+  return (c & 1u) ? (w >> 16) : (w & 0xFFFFu);
 }
 
 // Dealing the T = R nb tiles of a phase (R row tiles of nb blocks) to G CTAs.
@@ -333,7 +362,9 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
   const int nb = q.m / kBlock, batch = q.batch;
   constexpr uint32_t tb = tile_bytes(N);
   const uint2* ptab = reinterpret_cast<const uint2*>(E.smem + SSmem::pos) + (N - 4) * kPosTableEntries;
-  const __half* xg = g < batch ? q.x + (size_t)g * q.ldx : nullptr;       // batch row of this lane group
+  // activations of batch row g (this lane group's): in global memory, or staged in shared memory as a plain copy
+  const __half* xg = nullptr;
+  if (g < batch) xg = q.use_image == 2 ? reinterpret_cast<const __half*>(ximg) + (size_t)g * q.m : q.x + (size_t)g * q.ldx;
   const uint32_t img_row_words = (uint32_t)nb * kImgWordsPerBlock;
   int R = lo / nb, b_first = lo - R * nb, left = hi - lo, nslot_used = 0;
   while (left > 0 && !W.failed) {
@@ -419,7 +450,13 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
             fa[j][1] = hmul2_bits(prmt(unit, 0u, 0x3424u), s2);
           }
           uint2 xr = make_uint2(0, 0);
-          if (xg) {
+          if constexpr (kImage) {
+            if (g < batch) {
+              const uint32_t* ir = ximg + (uint32_t)g * img_row_words;
+              xr.x = image_x(ir, block, cols & 0xFFu) | (image_x(ir, block, (cols >> 8) & 0xFFu) << 16);
+              xr.y = image_x(ir, block, (cols >> 16) & 0xFFu) | (image_x(ir, block, cols >> 24) << 16);
+            }
+          } else if (xg) {
             const __half* xq = xg + (size_t)block * kBlock;
             xr.x = ld_u16(xq + (cols & 0xFFu)) | (ld_u16(xq + ((cols >> 8) & 0xFFu)) << 16);
             xr.y = ld_u16(xq + ((cols >> 16) & 0xFFu)) | (ld_u16(xq + (cols >> 24)) << 16);
@@ -541,7 +578,7 @@ stack_kernel(const __grid_constant__ StackParams P) {
     }
     __syncthreads();
     if (ctl[0]) W.failed = true;
-    if (q.use_image && !ctl[0]) {
+    if (q.use_image == 1 && !ctl[0]) {
       // one item = the 8 activations of one group of one batch row: a 16-byte load, six 4-byte stores (see stb_gemv.cu)
       const uint32_t img_row_words = (uint32_t)nb * kImgWordsPerBlock;
       const int per_row = nb * 16, items = batch * per_row;
@@ -553,7 +590,7 @@ stack_kernel(const __grid_constant__ StackParams P) {
           v[k] = make_uint4(0, 0, 0, 0);
           if (it < items) {
             const int r = it >= per_row ? 1 : 0, qq = it - r * per_row;       // the image serves one or two batch rows
-            v[k] = ld_v4(q.x + (size_t)r * q.ldx + (size_t)qq * 8);
+            v[k] = staged_x(q.x, q.x2, (size_t)r * q.ldx + (size_t)qq * 8);
           }
         }
 #pragma unroll
@@ -568,13 +605,20 @@ stack_kernel(const __grid_constant__ StackParams P) {
           }
         }
       }
+    } else if (q.use_image == 2 && !ctl[0]) {
+      // plain fp16 copy [batch][m] of the (formed) activations
+      const int per_row = q.m / 8, items = batch * per_row;
+      for (int it = threadIdx.x; it < items; it += kSThreads) {
+        const int r = it / per_row, qq = it - r * per_row;
+        reinterpret_cast<uint4*>(ximg)[it] = staged_x(q.x, q.x2, (size_t)r * q.ldx + (size_t)qq * 8);
+      }
     }
     if (lane == 0) { pslot[2 * warp].R = -1; pslot[2 * warp + 1].R = -1; }
     __syncthreads();
 
     // ---- this warp's tiles ----
     if (!W.failed && wl < wh) {
-      if (q.N == 6 && q.use_image) run_tiles<6, true>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      if (q.N == 6 && q.use_image == 1) run_tiles<6, true>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
       else if (q.N == 6) run_tiles<6, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
       else if (q.N == 5) run_tiles<5, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
       else run_tiles<4, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
@@ -694,7 +738,8 @@ struct StackPlan {
 };
 
 static bool same_input(const stb_step& a, const stb_step& b) {
-  return a.in == b.in && a.ldin == b.ldin && a.batch == b.batch && a.m == b.m && a.N == b.N && b.out != a.in;
+  return a.in == b.in && a.in2 == b.in2 && a.input == b.input && a.ldin == b.ldin && a.batch == b.batch && a.m == b.m &&
+         a.N == b.N && b.out != a.in && b.out != a.in2;
 }
 
 static int check_step(const stb_step& s) {
@@ -707,6 +752,8 @@ static int check_step(const stb_step& s) {
   if (s.odt != STB_F32 && s.odt != STB_F16) return STB_ERR_UNSUPPORTED;
   if (s.ldin < (size_t)s.m || s.ldout < (size_t)s.n || (s.ldin % 8) != 0 || (reinterpret_cast<uintptr_t>(s.in) & 15u)) return STB_ERR_ARG;
   if (s.ldin > 0xFFFFFFFFull || s.ldout > 0xFFFFFFFFull) return STB_ERR_ARG;
+  if (s.input != STB_IN_PLAIN && s.input != STB_IN_SILU_MUL) return STB_ERR_ARG;
+  if (s.input == STB_IN_SILU_MUL && (!s.in2 || (reinterpret_cast<uintptr_t>(s.in2) & 15u))) return STB_ERR_ARG;
   return STB_OK;
 }
 
@@ -772,6 +819,7 @@ static int build_phases(const stb_step* steps, int count, int i0, int G, StackPa
     }
     for (int k = q.count; k < kMaxFusedSteps; ++k) q.tile_start[k + 1] = q.tile_start[q.count];
     q.x = static_cast<const __half*>(st.in);
+    q.x2 = st.input == STB_IN_SILU_MUL ? static_cast<const __half*>(st.in2) : nullptr;
     q.ldx = (uint32_t)st.ldin; q.m = st.m; q.N = (uint8_t)st.N; q.batch = (uint8_t)st.batch;
     q.use_image = 0; q.pad[0] = q.pad[1] = 0;
     q.done_before = done;
@@ -785,16 +833,20 @@ static int build_phases(const stb_step* steps, int count, int i0, int G, StackPa
     ++sp.nphase;
     i = j;
   }
-  // second pass: which 6:8 phases get the operand-order image of their activations in shared memory
+  // second pass: where each phase takes its activations from.  6:8 with up to two batch rows: the operand-order
+  // image in shared memory if it fits; a formed input (silu(in) * in2) must be staged: image or plain copy.
   const uint32_t fixed = SSmem::pdata + 32u * sp.part_floats * 4u;
   for (int p = 0; p < sp.nphase; ++p) {
     StackPhase& q = sp.ph[p];
-    if (q.N != 6 || q.batch > 2) continue;
-    const uint32_t need = (uint32_t)q.batch * (uint32_t)(q.m / kBlock) * kImgWordsPerBlock * 4u;
-    if (fixed + need <= kSmemLimit) {
-      q.use_image = 1;
-      if (need > sp.image_bytes) sp.image_bytes = need;
+    const uint32_t img = (uint32_t)q.batch * (uint32_t)(q.m / kBlock) * kImgWordsPerBlock * 4u;
+    const uint32_t plain = (uint32_t)q.batch * (uint32_t)q.m * 2u;
+    uint32_t need = 0;
+    if (q.N == 6 && q.batch <= 2 && fixed + img <= kSmemLimit) { q.use_image = 1; need = img; }
+    else if (q.x2) {
+      if (fixed + plain > kSmemLimit) return -1;          // the formed input does not fit shared memory
+      q.use_image = 2; need = plain;
     }
+    if (need > sp.image_bytes) sp.image_bytes = need;
   }
   const size_t s_need = (size_t)(4 + maxR) * sizeof(uint32_t);
   const size_t g_need = (size_t)maxR * sp.max_share * sp.part_floats * sizeof(float);
@@ -819,7 +871,10 @@ extern "C" int stb_layer_stack_resident_workspace(const stb_step* steps, int cou
   size_t sync_need = 0, gpart_need = 0;
   static thread_local stb::StackParams sp;
   int i = 0;
-  while (i < count) i = stb::build_phases(steps, count, i, G, sp, sync_need, gpart_need);
+  while (i < count) {
+    i = stb::build_phases(steps, count, i, G, sp, sync_need, gpart_need);
+    if (i < 0) return STB_ERR_UNSUPPORTED;
+  }
   *bytes = stb::align256(sync_need) + stb::align256(gpart_need);
   return STB_OK;
 }
@@ -840,7 +895,10 @@ static int stack_resident_impl(const stb_step* steps, int count, void* ws, size_
   static thread_local stb::StackParams sp;
   {
     int i = 0;
-    while (i < count) i = stb::build_phases(steps, count, i, G, sp, sync_need, gpart_need);
+    while (i < count) {
+      i = stb::build_phases(steps, count, i, G, sp, sync_need, gpart_need);
+      if (i < 0) return STB_ERR_UNSUPPORTED;
+    }
   }
   const size_t sync_bytes = stb::align256(sync_need);
   if (ws_bytes < sync_bytes + stb::align256(gpart_need)) return STB_ERR_SIZE;
@@ -856,6 +914,7 @@ static int stack_resident_impl(const stb_step* steps, int count, void* ws, size_
   while (i < count) {
     size_t a = 0, b = 0;
     i = stb::build_phases(steps, count, i, G, sp, a, b);
+    if (i < 0) return STB_ERR_UNSUPPORTED;
     sp.sync = static_cast<uint32_t*>(ws);
     sp.gpart = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + sync_bytes);
     sp.dev_status = dev_status;

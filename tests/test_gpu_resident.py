@@ -159,6 +159,57 @@ def test_unsupported_steps_are_refused_on_the_host(stb):
     assert stb._lib.stb_layer_stack_resident(steps, 1, stb._ptr(ws), 16, None, stb._stream()) == stb.STB_ERR_SIZE
 
 
+def _check_gated_mlp(stb, torch, dg, du, dd, batch, graph=False, rows_of=None):
+    """gate and up read x, down reads fp16(silu(gate) * up) formed while it stages its input (STB_IN_SILU_MUL): gate and
+    up against the oracle as usual, down against the oracle fed the oracle's own float64 evaluation of the gated
+    activation of the GPU's gate and up outputs."""
+    m, f = dg["m"], dg["n"]
+    lg, lu, ld = (stb.pack_numpy(d) for d in (dg, du, dd))
+    x = torch.from_numpy(si.activations(batch, m, 74)).cuda()
+    hg = torch.zeros(batch, f, dtype=torch.float16, device="cuda")
+    hu = torch.zeros(batch, f, dtype=torch.float16, device="cuda")
+    y = torch.zeros(batch, dd["n"], dtype=torch.float32, device="cuda")
+    triples = [(lg, x, hg), (lu, x, hu), (ld, (hg, hu), y)]
+    _run(stb, torch, triples, graph=graph)
+    as_l = wl.as_logical
+    _check_layers(triples[:2], [as_l(dg), as_l(du)], rows_of=rows_of)
+    act = oracle.silu_mul(hg.double().cpu().numpy(), hu.double().cpu().numpy())
+    got = y.double().cpu().numpy()
+    if rows_of is None:
+        ref = oracle.matmul(oracle.decode(as_l(dd)), act)
+    else:
+        rows = rows_of(dd["n"], 2)
+        ref = oracle.layer_rows(as_l(dd), rows, act)
+        got = got[:, rows]
+    assert np.abs(got - ref).max() <= TOL * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("N,batch", [(6, 1), (6, 2), (6, 3), (4, 1), (5, 8)])
+def test_gated_activation_is_formed_while_down_stages_its_input(stb, N, batch):
+    import torch
+    dg = si.logical_layer(384, 256, N, 171, max_salient=9)
+    du = si.logical_layer(384, 256, N, 172, max_salient=9)
+    dd = si.logical_layer(200, 384, N, 173, salient_counts=[3, 17, 0])
+    _check_gated_mlp(stb, torch, dg, du, dd, batch)
+
+
+def test_gated_mlp_full_size(stb):
+    """The LLaMA-2-7B MLP at 6:8 (quantizer-made) with the gated activation, in a CUDA graph as bench.py runs it."""
+    import torch
+    dg, du, dd = (wl.quantized_layer(*si.workload_layer(2, nm)) for nm in ("gate", "up", "down"))
+    _check_gated_mlp(stb, torch, dg, du, dd, 1, graph=True, rows_of=_rows_of)
+
+
+def test_per_layer_launches_refuse_formed_inputs(stb):
+    import torch
+    d = si.logical_layer(64, 128, 4, 97)
+    lay = stb.pack_numpy(d)
+    a = torch.zeros(1, 128, dtype=torch.float16, device="cuda")
+    y = torch.zeros(1, 64, device="cuda")
+    steps = stb.make_steps([(lay, (a, a), y)])
+    assert stb._lib.stb_layer_stack(steps, 1, None, stb._stream()) == stb.STB_ERR_UNSUPPORTED
+
+
 def _rows_of(n, k):
     g = np.random.default_rng(1000 + k)
     return np.unique(np.concatenate([[0, 31, 32, n - 1], g.choice(n, 60, replace=False)])).astype(np.int32)

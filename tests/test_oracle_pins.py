@@ -423,3 +423,21 @@ def test_degenerate_all_zero_and_all_equal_blocks():
     What = oracle.decode(L)
     assert (What[:, :128] == 0).all()
     assert np.array_equal(What[:, 128:][kb[:, 128:]], np.full(kb[:, 128:].sum(), 0.5, np.float32))
+
+
+def test_silu_mul_identities():
+    """The gated activation fp16(silu(a) * b): silu(v) - silu(-v) = v, silu(0) = 0, silu(ln 3) = 0.75 ln 3, silu(v) -> v for
+    large v, linear in b; results are fp16 values (checked against numpy's rounding of the closed forms)."""
+    import math
+    v = np.array([0.0, math.log(3.0), 30.0, -30.0, 2.5, -2.5, 0.125], np.float64)
+    one = np.ones_like(v)
+    s = oracle.silu_mul(v, one)
+    want = np.array([0.0, 0.75 * math.log(3.0), 30.0, 0.0, 0.0, 0.0, 0.0])
+    assert s[0] == 0.0 and s[1] == np.float64(np.float16(want[1])) and s[2] == 30.0 and abs(s[3]) < 1e-11
+    # silu(v) - silu(-v) = v: with b = 1 both terms are rounded to fp16, so compare within fp16 rounding of each
+    assert abs((s[4] - s[5]) - 2.5) <= 2.0 ** -10 * 2.5
+    # linear in b (exactly: scaling by a power of two commutes with the rounding)
+    assert np.array_equal(oracle.silu_mul(v, 4.0 * one), 4.0 * s)
+    assert np.array_equal(oracle.silu_mul(v, -one), -s)
+    # fp16 output: every value is representable
+    assert np.array_equal(s.astype(np.float16).astype(np.float64), s)
