@@ -636,6 +636,11 @@ def cuda_arm(args):
             dist.destroy_process_group()
         return
 
+    # the same list of passes walked by the checksum kernel: same dealing, rings and bulk copies, no arithmetic
+    sums = torch.zeros(len(wl._keep[0]), dtype=torch.int64, device="cuda")
+    g_sum = capture(torch, [lambda: stb.layer_stack_checksum(wl._keep[0], sums=sums, dev_status=wl.status)])
+    us_stream = time_graph(torch, g_sum, copies, min_calls=100 * copies)
+    del g_sum
     traffic, traffic_note = captured_traffic()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -664,7 +669,11 @@ def cuda_arm(args):
                      "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": traffic, "traffic_source": traffic_note,
                      "kernel": "stb::stack_kernel" if wl.resident else "stb::gemv_mma_kernel<6,1>", "peak_source": pk["_source"],
                      "bytes_per_launch": round(per_launch_bytes), "launch_us": round(launch_us, 3),
-                     "note": "launch_us = timed region / launches (includes the gaps between launches)"},
+                     "stream_only_frac": round(wl.bytes_step / us_stream / 1e3 / pk["hbm_gbs"], 4),
+                     "stream_only_us_per_pass": round(us_stream, 3),
+                     "note": "launch_us = timed region / launches (includes the gaps between launches); stream_only = the same "
+                             "passes through stb_layer_stack_checksum, which walks the layers as the resident kernel does (same "
+                             "dealing, rings and bulk copies) and XORs the words instead of decoding them"},
     }
     if world == 1 and not args.no_extras:
         # the same passes through the other entry point

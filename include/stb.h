@@ -223,6 +223,16 @@ int stb_layer_stack_resident_host(const stb_step *steps, int count, void *ws, si
 int stb_layer_stack_resident_wait_selftest(const stb_step *steps, int count, void *ws,
                                            size_t ws_bytes, int *dev_status, void *stream);
 
+/* Integrity check of packed layers (the paper has no counterpart): sums[i] (DEVICE, 64-bit, one per step)
+ * becomes the XOR of all 32-bit words of step i's tiles and residual streams, i.e. of the bytes
+ * [tiles offset, used_bytes) of its packed buffer -- everything a decode pass streams.  Only `packed`, n, m,
+ * N, batch and the pointers' validity of a step are looked at.  The layers are walked exactly as
+ * stb_layer_stack_resident walks them (same dealing to the SMs, same rings and bulk copies), without
+ * the arithmetic: its running time is what that way of streaming costs by itself.  One launch per 64
+ * groups of steps, plus a memset of sums. */
+int stb_layer_stack_checksum(const stb_step *steps, int count, unsigned long long *sums,
+                             int *dev_status, void *stream);
+
 /* stb_layer_stack for a caller whose activations live in HOST memory: copies in_bytes from
  * in_host (HOST, pinned for the copy to be asynchronous) into steps[0].in, runs the steps,
  * then copies out_bytes from steps[count-1].out to out_host (HOST).  The device buffers named

@@ -24,7 +24,7 @@ STB_IN_PLAIN, STB_IN_SILU_MUL = 0, 1
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
            "stb_gemm_workspace", "stb_gemm_workspace_min", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
            "stb_layer_stack_resident_workspace", "stb_layer_stack_resident", "stb_layer_stack_resident_host",
-           "stb_layer_stack_resident_wait_selftest", "stb_status_str"]
+           "stb_layer_stack_resident_wait_selftest", "stb_layer_stack_checksum", "stb_status_str"]
 
 
 class StbError(RuntimeError):
@@ -72,6 +72,7 @@ def _load():
     lib.stb_layer_stack_resident.argtypes = [p(_Step), i, v, z, v, v]
     lib.stb_layer_stack_resident_wait_selftest.argtypes = [p(_Step), i, v, z, v, v]
     lib.stb_layer_stack_resident_host.argtypes = [p(_Step), i, v, z, v, z, v, z, v, v]
+    lib.stb_layer_stack_checksum.argtypes = [p(_Step), i, v, v, v]
     lib.stb_status_str.argtypes = [i]
     lib.stb_status_str.restype = C.c_char_p
     for name in EXPORTS:
@@ -297,3 +298,13 @@ def layer_stack_resident_host(marshalled, ws, x_host, y_host, dev_status=None, s
                                               C.c_void_p(x_host.data_ptr()), x_host.numel() * x_host.element_size(),
                                               C.c_void_p(y_host.data_ptr()), y_host.numel() * y_host.element_size(),
                                               _ptr(dev_status), _stream(stream)), "stb_layer_stack_resident_host")
+
+
+def layer_stack_checksum(marshalled, sums=None, dev_status=None, stream=None):
+    """stb_layer_stack_checksum: XOR of the streamed words of every step's packed layer -> torch.int64[count]."""
+    import torch
+    if sums is None:
+        sums = torch.zeros(len(marshalled), dtype=torch.int64, device="cuda")
+    _check(_lib.stb_layer_stack_checksum(marshalled, len(marshalled), _ptr(sums), _ptr(dev_status), _stream(stream)),
+           "stb_layer_stack_checksum")
+    return sums

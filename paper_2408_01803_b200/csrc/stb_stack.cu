@@ -128,6 +128,11 @@ __device__ __forceinline__ uint32_t ld_u16(const void* p) {
   asm volatile("ld.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ uint4 ldg_v4_coherent(const void* p) {      // the same from global memory
+  uint4 v;
+  asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
 // fp16 pair (bits) of silu(a) * b per half, in fp32, rounded to nearest even
 __device__ __forceinline__ uint32_t silu_mul_bits(uint32_t a, uint32_t b) {
   const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&a)), fb = __half22float2(*reinterpret_cast<const __half2*>(&b));
@@ -136,9 +141,9 @@ __device__ __forceinline__ uint32_t silu_mul_bits(uint32_t a, uint32_t b) {
 }
 // the staged form of eight activations: as they are, or silu(in) * in2
 __device__ __forceinline__ uint4 staged_x(const __half* x, const __half* x2, size_t off) {
-  uint4 v = ld_v4(x + off);
+  uint4 v = ldg_v4_coherent(x + off);
   if (x2) {
-    const uint4 w = ld_v4(x2 + off);
+    const uint4 w = ldg_v4_coherent(x2 + off);
     v.x = silu_mul_bits(v.x, w.x); v.y = silu_mul_bits(v.y, w.y); v.z = silu_mul_bits(v.z, w.z); v.w = silu_mul_bits(v.w, w.w);
   }
   return v;
@@ -732,6 +737,94 @@ stack_kernel(const __grid_constant__ StackParams P) {
 }
 
 // ------------------------------------------------------------------------------------------
+// stb_layer_stack_checksum: XOR of all 32-bit words of the tiles and residual streams of every step's packed layer
+// (an integrity check for packed layers that were stored or moved).  It walks the layers exactly as stack_kernel
+// does -- same dealing, same per-warp rings and bulk copies, same residual-span copies -- and folds the words
+// instead of decoding them, so its rate is also the rate this way of streaming reaches with no arithmetic behind it.
+__global__ void __launch_bounds__(kSThreads, 1)
+checksum_kernel(const __grid_constant__ StackParams P, unsigned long long* __restrict__ sums, int first_step) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cta = (int)blockIdx.x, G = (int)gridDim.x;
+  WarpEnv E;
+  E.P = &P; E.smem = smem; E.cta = cta; E.G = G; E.warp = warp; E.lane = lane; E.g = lane >> 2; E.t = lane & 3;
+  E.bar0 = smem_u32(smem + SSmem::bars) + (uint32_t)warp * kSDepth * 8u;
+  E.bar_stage = smem_u32(smem + SSmem::bars) + (uint32_t)(kSWarps * kSDepth + warp) * 8u;
+  E.ring = smem + SSmem::ring + (size_t)warp * kSDepth * kSlotBytes;
+  E.stage = smem + SSmem::stage + (size_t)warp * kStageBytes;
+  if (lane == 0) {
+    for (int i = 0; i < kSDepth; ++i) mbar_init(E.bar0 + 8u * i, 1);
+    mbar_init(E.bar_stage, 1);
+    fence_async_smem();
+  }
+  __syncwarp();
+  WarpState W;
+  W.prod.enter(P, 0, cta, G, warp);
+  W.consumed = 0; W.cur_in = 0; W.stage_use = 0; W.failed = false;
+#pragma unroll
+  for (int i = 0; i < kSDepth; ++i) ring_issue(E, W, i);
+
+  int step_base = first_step;                    // index, in the caller's list, of the phase's first step
+  for (int ph = 0; ph < P.nphase && !W.failed; ++ph) {
+    const StackPhase& q = P.ph[ph];
+    const int nb = q.m / kBlock;
+    const uint32_t tb = tile_bytes(q.N);
+    int lo, hi;
+    warp_range(q, nb, cta, G, warp, lo, hi);
+    int R = lo / nb, b_first = lo - R * nb, left = hi - lo;
+    while (left > 0 && !W.failed) {
+      const int seg = left < nb - b_first ? left : nb - b_first, b_end = b_first + seg;
+      const int si = step_of(q, R), rt = R - q.tile_start[si];
+      const uint8_t* packed = q.packed[si];
+      const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
+      const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + rwtab_offset(nb));
+      const int ntile = (q.n[si] + kTileRows - 1) / kTileRows;
+      const uint32_t nrw_all = __ldg(&reinterpret_cast<const Header*>(packed)->nrw);
+      const uint8_t* resid_rt = packed + tiles_offset(nb) + (size_t)tb * nb * ntile + (size_t)rt * resid_rt_bytes(nb, nrw_all);
+      uint32_t fold = 0;
+      for (int bs = b_first; bs < b_end && !W.failed; bs += kSpan) {
+        const int be = bs + kSpan < b_end ? bs + kSpan : b_end;
+        const uint32_t rw0 = __ldg(&binfo[bs].rw_off), rw1 = __ldg(&binfo[be - 1].rw_off) + __ldg(&binfo[be - 1].nrw);
+        const uint32_t rec_bytes = (uint32_t)(be - bs) * kResidA2Bytes + (rw1 - rw0) * kResidWordBytes;
+        const uint32_t tab0 = rw0 & ~1u, tab_bytes = ((rw1 - tab0) * 8u + 15u) & ~15u;
+        __syncwarp();
+        if (lane == 0) {
+          fence_async_smem();
+          mbar_expect_tx(E.bar_stage, rec_bytes + (rw1 > rw0 ? tab_bytes : 0u));
+          bulk_g2s(smem_u32(E.stage), resid_rt + resid_block_off(bs, rw0), rec_bytes, E.bar_stage);
+          if (rw1 > rw0) bulk_g2s(smem_u32(E.stage + kStageTab), rwt + tab0, tab_bytes, E.bar_stage);
+        }
+        const uint32_t stage_parity = W.stage_use & 1u;
+        ++W.stage_use;
+        for (int b = bs; b < be; ++b) {
+          const int slot = (int)(W.consumed % kSDepth);
+          if (W.cur_in == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(E.bar0 + 8u * slot, (W.consumed / kSDepth) & 1u, P.wait_limit))) { W.failed = true; break; }
+          const uint8_t* tile = E.ring + (size_t)slot * kSlotBytes + (size_t)W.cur_in * tb;
+          const bool last_of_chunk = W.cur_in + 1 == (slot == 0 ? W.chunk_cnt0 : W.chunk_cnt1);
+          for (uint32_t o = (uint32_t)lane * 4u; o < tb; o += 128u) fold ^= *reinterpret_cast<const uint32_t*>(tile + o);
+          if (last_of_chunk) { __syncwarp(); ring_issue(E, W, slot); W.cur_in = 0; ++W.consumed; }
+          else ++W.cur_in;
+        }
+        if (W.failed) break;
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait(E.bar_stage, stage_parity, P.wait_limit))) { W.failed = true; break; }
+        for (uint32_t o = (uint32_t)lane * 4u; o < rec_bytes; o += 128u) fold ^= *reinterpret_cast<const uint32_t*>(E.stage + o);
+      }
+      // words of one step only ever meet words of the same step
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) fold ^= __shfl_xor_sync(0xFFFFFFFFu, fold, d);
+      if (lane == 0 && !W.failed) atomicXor(sums + step_base + si, (unsigned long long)fold);
+      left -= seg; ++R; b_first = 0;
+    }
+    step_base += q.count;
+  }
+  if (W.failed) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000) {}
+    if (lane == 0 && P.dev_status) *P.dev_status = STB_ERR_TIMEOUT;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Host side: steps -> phases -> launches.
 struct StackPlan {
   size_t sync_bytes, gpart_bytes;
@@ -957,5 +1050,40 @@ extern "C" int stb_layer_stack_resident_host(const stb_step* steps, int count, v
   if (rc != STB_OK) return rc;
   if (cudaMemcpyAsync(out_host, steps[count - 1].out, out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
     return STB_ERR_CUDA;
+  return STB_OK;
+}
+
+extern "C" int stb_layer_stack_checksum(const stb_step* steps, int count, unsigned long long* sums, int* dev_status, void* stream) {
+  if (!steps || count < 1 || !sums) return STB_ERR_ARG;
+  for (int i = 0; i < count; ++i) {
+    const int rc = stb::check_step(steps[i]);
+    if (rc != STB_OK) return rc;
+  }
+  int G = 0;
+  int rc = stb::stack_sm_count(&G);
+  if (rc != STB_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  static bool attr_done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return STB_ERR_CUDA;
+  if (!attr_done[dev]) {
+    if (cudaFuncSetAttribute(stb::checksum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stb::kSmemLimit) != cudaSuccess) return STB_ERR_CUDA;
+    attr_done[dev] = true;
+  }
+  if (cudaMemsetAsync(sums, 0, sizeof(unsigned long long) * (size_t)count, s) != cudaSuccess) return STB_ERR_CUDA;
+  static thread_local stb::StackParams sp;
+  int i = 0;
+  while (i < count) {
+    size_t a = 0, b = 0;
+    const int first = i;
+    i = stb::build_phases(steps, count, i, G, sp, a, b);
+    if (i < 0) return STB_ERR_UNSUPPORTED;
+    sp.sync = nullptr; sp.gpart = nullptr; sp.dev_status = dev_status;
+    sp.wait_limit = stb::kSWaitLimit; sp.copies_off = 0;
+    // the same shared-memory footprint as the arithmetic kernel would have for these steps
+    const uint32_t smem = stb::SSmem::pdata + 32u * sp.part_floats * 4u + sp.image_bytes;
+    stb::checksum_kernel<<<(unsigned)G, stb::kSThreads, smem, s>>>(sp, sums, first);
+    if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
+  }
   return STB_OK;
 }

@@ -210,6 +210,40 @@ def test_per_layer_launches_refuse_formed_inputs(stb):
     assert stb._lib.stb_layer_stack(steps, 1, None, stb._stream()) == stb.STB_ERR_UNSUPPORTED
 
 
+def test_checksum_of_the_streamed_bytes(stb):
+    """stb_layer_stack_checksum = XOR of the 32-bit words of [tiles offset, used_bytes) of every step's packed buffer;
+    a flipped bit in a tile or in a residual record changes it."""
+    import torch
+    ds = [si.logical_layer(200, 1024, 6, 301, salient_counts=[1, 9, 32, 0]), si.logical_layer(130, 1024, 6, 302, max_salient=5),
+          si.logical_layer(96, 256, 4, 303), si.logical_layer(4096, 1024, 5, 304, max_salient=20)]
+    layers = [stb.pack_numpy(d) for d in ds]
+    x = torch.zeros(1, 1024, dtype=torch.float16, device="cuda")
+    x2 = torch.zeros(1, 256, dtype=torch.float16, device="cuda")
+    outs = [torch.zeros(1, d["n"], device="cuda") for d in ds]
+    steps = stb.make_steps([(layers[0], x, outs[0]), (layers[1], x, outs[1]), (layers[2], x2, outs[2]), (layers[3], x, outs[3])])
+
+    def expected(lay):
+        info = lay.info()
+        nblk = lay.m // 128
+        t0 = (64 + 128 * nblk + 255) // 256 * 256
+        words = lay.buf[t0:info["used_bytes"]].cpu().numpy().view(np.uint32)
+        return int(np.bitwise_xor.reduce(words))
+
+    sums = stb.layer_stack_checksum(steps)
+    torch.cuda.synchronize()
+    got = [int(v) & 0xFFFFFFFFFFFFFFFF for v in sums.cpu().numpy()]
+    assert got == [expected(l) for l in layers]
+    # one flipped bit in the last byte a pass streams (a residual record), one in the first tile
+    for lay, off in ((layers[0], layers[0].info()["used_bytes"] - 1), (layers[3], (64 + 128 * 8 + 255) // 256 * 256 + 5)):
+        before = expected(lay)
+        lay.buf[off] ^= 0x10
+        after = stb.layer_stack_checksum(steps)
+        torch.cuda.synchronize()
+        k = layers.index(lay)
+        assert (int(after[k].item()) & 0xFFFFFFFFFFFFFFFF) == expected(lay) != before
+        lay.buf[off] ^= 0x10
+
+
 def _rows_of(n, k):
     g = np.random.default_rng(1000 + k)
     return np.unique(np.concatenate([[0, 31, 32, n - 1], g.choice(n, 60, replace=False)])).astype(np.int32)
