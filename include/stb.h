@@ -241,6 +241,15 @@ int stb_layer_stack_checksum(const stb_step *steps, int count, unsigned long lon
 int stb_layer_stack_host(const stb_step *steps, int count, const void *in_host, size_t in_bytes,
                          void *out_host, size_t out_bytes, int *dev_status, void *stream);
 
+/* Layer-wise N:M assignment (Section 3.3): more important layers, by the L2 norm of their weights, keep more of
+ * every 8.  stb_weight_sumsq adds the sum of squares of a dense fp16 matrix W[n][ldw] (DEVICE, 16-byte aligned, ldw a
+ * multiple of 8) to *sumsq (DEVICE float64, zeroed by the caller; one launch).  stb_allocate_nm is HOST arithmetic on
+ * the layers' sums of squares copied back: alpha_i = omega_i / sum_k omega_k with omega = sqrt(sum of squares),
+ * N_i = 8 (alpha_i + (1 - alpha_i) r_target) rounded to nearest (ties to even) and kept inside 1..8.  As printed in the
+ * paper the ratio never falls below r_target. */
+int stb_weight_sumsq(const void *W, int n, int m, size_t ldw, double *sumsq, void *stream);
+int stb_allocate_nm(const double *sumsq, int layers, double r_target, int *N_out);
+
 /* Static string for a status code. */
 const char *stb_status_str(int status);
 

@@ -45,7 +45,6 @@ def lib():
         _lib.stbo_average_bits.restype = C.c_double
         _lib.stbo_average_bits.argtypes = [C.c_int, C.c_double]
         _lib.stbo_counted_bits.restype = C.c_double
-        _lib.stbo_recon_error.restype = C.c_double
         _lib.stbo_salient_search.restype = C.c_int
         _lib.stbo_breakpoint_search.restype = C.c_int
         _lib.stbo_hardware_threads.restype = C.c_int
@@ -194,6 +193,14 @@ def silu_mul(a, b):
     return out.view(np.float16).astype(np.float64)
 
 
+def allocate_nm(l2norms, r_target):
+    """Layer-wise N:M assignment (Section 3.3): returns (N per layer, unrounded ratios)."""
+    w = _c(l2norms, np.float64)
+    N = np.empty(len(w), np.int32); ratio = np.empty(len(w), np.float64)
+    lib().stbo_allocate_nm(_p(w), C.c_int(len(w)), C.c_double(r_target), _p(N), _p(ratio))
+    return N, ratio
+
+
 def average_bits(N, r_salient):
     return float(lib().stbo_average_bits(C.c_int(N), C.c_double(r_salient)))
 
@@ -204,10 +211,3 @@ def counted_bits(L: Logical):
     v = lib().stbo_counted_bits(C.c_int(L.n), C.c_int(L.m), _p(L.keep), _p(L.salient),
                                 C.byref(r))
     return float(v), r.value
-
-
-def recon_error(W, What, keep, kept_only=True):
-    W = _c(W, np.float64); What = _c(What, np.float32); keep = _c(keep, np.uint8)
-    n, m = W.shape
-    return float(lib().stbo_recon_error(_p(W), _p(What), C.c_int(n), C.c_int(m), _p(keep),
-                                        C.c_int(1 if kept_only else 0)))

@@ -483,26 +483,28 @@ double stbo_counted_bits(int n, int m, const uint8_t* keep, const uint64_t* sali
   return (double)(nkept + nsalkept) / ((double)n * m);
 }
 
-// Squared error of the decoded layer against W (float64), for the invariants.
-double stbo_recon_error(const double* W, const float* What, int n, int m, const uint8_t* keep,
-                        int kept_only) {
-  Dims d = dims(n, m);
-  double e = 0.0;
-  for (int i = 0; i < n; ++i)
-    for (int j = 0; j < m; ++j) {
-      if (kept_only && !kept(keep, d, i, j)) continue;
-      double df = W[(size_t)i * m + j] - (double)What[(size_t)i * m + j];
-      e += df * df;
-    }
-  return e;
-}
-
 // ---------------------------------------------------------------------------
 // Not from the paper: the gated activation of the LLaMA MLP, whose three linears the paper binarizes
 // (Section 4.1 evaluates LLaMA-1/2/3).  out[i] = fp16( silu(a[i]) * b[i] ), silu(v) = v / (1 + exp(-v)), float64.
 // The CUDA path can form the input of the down projection this way (STB_IN_SILU_MUL).
 void stbo_silu_mul(const double* a, const double* b, int n, uint16_t* out) {
   for (int i = 0; i < n; ++i) out[i] = double_to_half_bits(a[i] / (1.0 + std::exp(-a[i])) * b[i]);
+}
+
+// ---------------------------------------------------------------------------
+// Section 3.3, Layer-wise N:M Assignment.  alpha_i = omega_i / sum_k omega_k with omega the L2 norm of layer i's
+// weights; N_i / M = alpha_i + (1 - alpha_i) R_target.  Reading: M = 8 and N_i is that ratio times 8 rounded to the
+// nearest integer (ties to even), kept inside 1..8.  ratio_out (may be null) receives the unrounded ratios.
+void stbo_allocate_nm(const double* l2norm, int layers, double r_target, int* N_out, double* ratio_out) {
+  double total = 0.0;
+  for (int i = 0; i < layers; ++i) total += l2norm[i];
+  for (int i = 0; i < layers; ++i) {
+    const double alpha = total > 0.0 ? l2norm[i] / total : 0.0;
+    const double ratio = alpha + (1.0 - alpha) * r_target;
+    if (ratio_out) ratio_out[i] = ratio;
+    int Ni = (int)std::nearbyint(ratio * (double)kM);
+    N_out[i] = std::min(kM, std::max(1, Ni));
+  }
 }
 
 int stbo_hardware_threads() { return (int)std::max(1u, std::thread::hardware_concurrency()); }

@@ -24,7 +24,8 @@ STB_IN_PLAIN, STB_IN_SILU_MUL = 0, 1
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
            "stb_gemm_workspace", "stb_gemm_workspace_min", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
            "stb_layer_stack_resident_workspace", "stb_layer_stack_resident", "stb_layer_stack_resident_host",
-           "stb_layer_stack_resident_wait_selftest", "stb_layer_stack_checksum", "stb_status_str"]
+           "stb_layer_stack_resident_wait_selftest", "stb_layer_stack_checksum", "stb_weight_sumsq",
+           "stb_allocate_nm", "stb_status_str"]
 
 
 class StbError(RuntimeError):
@@ -73,6 +74,8 @@ def _load():
     lib.stb_layer_stack_resident_wait_selftest.argtypes = [p(_Step), i, v, z, v, v]
     lib.stb_layer_stack_resident_host.argtypes = [p(_Step), i, v, z, v, z, v, z, v, v]
     lib.stb_layer_stack_checksum.argtypes = [p(_Step), i, v, v, v]
+    lib.stb_weight_sumsq.argtypes = [v, i, i, z, v, v]
+    lib.stb_allocate_nm.argtypes = [p(C.c_double), i, C.c_double, p(i)]
     lib.stb_status_str.argtypes = [i]
     lib.stb_status_str.restype = C.c_char_p
     for name in EXPORTS:
@@ -308,3 +311,19 @@ def layer_stack_checksum(marshalled, sums=None, dev_status=None, stream=None):
     _check(_lib.stb_layer_stack_checksum(marshalled, len(marshalled), _ptr(sums), _ptr(dev_status), _stream(stream)),
            "stb_layer_stack_checksum")
     return sums
+
+
+def allocate_nm(weights, r_target, stream=None):
+    """Layer-wise N:M assignment (stb_weight_sumsq per layer, then stb_allocate_nm): `weights` is a list of dense fp16
+    CUDA matrices; returns the list of N."""
+    import torch
+    sums = torch.zeros(len(weights), dtype=torch.float64, device=weights[0].device)
+    for k, W in enumerate(weights):
+        assert W.dtype == torch.float16 and W.dim() == 2 and W.stride(1) == 1
+        _check(_lib.stb_weight_sumsq(_ptr(W), W.shape[0], W.shape[1], W.stride(0), C.c_void_p(sums.data_ptr() + 8 * k),
+                                     _stream(stream)), "stb_weight_sumsq")
+    host = sums.cpu().numpy()
+    arr = (C.c_double * len(weights))(*[float(vv) for vv in host])
+    out = (C.c_int * len(weights))()
+    _check(_lib.stb_allocate_nm(arr, len(weights), float(r_target), out), "stb_allocate_nm")
+    return [int(vv) for vv in out], host

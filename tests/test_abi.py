@@ -81,3 +81,19 @@ def test_packed_layout_and_byte_permute_decode_on_the_host(tmp_path):
     out = subprocess.run([exe], capture_output=True, text=True)
     assert out.returncode == 0, out.stdout[-2000:]
     assert "OK: 0 errors" in out.stdout
+
+
+def test_layerwise_assignment_host_arithmetic_matches_the_oracle(stb):
+    """stb_allocate_nm (host arithmetic of the library) against the oracle's Section 3.3 assignment."""
+    import numpy as np
+    import oracle
+    g = np.random.default_rng(11)
+    for R in (0.5, 0.625, 0.75):
+        norms = g.random(37) * 10 + 0.05
+        want, _ = oracle.allocate_nm(norms, R)
+        arr = (C.c_double * 37)(*[float(v * v) for v in norms])
+        out = (C.c_int * 37)()
+        assert stb._lib.stb_allocate_nm(arr, 37, R, out) == stb.STB_OK
+        assert [int(v) for v in out] == [int(v) for v in want]
+    assert stb._lib.stb_allocate_nm(None, 3, 0.5, out) == stb.STB_ERR_ARG
+    assert stb._lib.stb_allocate_nm(arr, 3, 0.0, out) == stb.STB_ERR_ARG

@@ -463,3 +463,16 @@ def test_13b_decoder_block_chained(stb):
         ref = oracle.layer_rows(wl.as_logical(ds[i]), rows, io[i][0].double().cpu().numpy())
         got = io[i][1].double().cpu().numpy()[:, rows]
         assert np.abs(got - ref).max() <= TOL * np.abs(ref).max(), name
+
+
+def test_layerwise_nm_assignment_from_dense_weights(stb):
+    """Section 3.3: N per layer from the L2 norms of the dense weights, the norms summed on the GPU."""
+    import torch
+    shapes = [(256, 384), (100, 128), (512, 1024), (64, 136)]
+    Ws = [si.dense_weight(n, m, 1200 + k) * np.float16(1 + 3 * k) for k, (n, m) in enumerate(shapes)]
+    norms = [np.sqrt((W.astype(np.float64) ** 2).sum()) for W in Ws]
+    for R in (0.5, 0.75):
+        got, sums = stb.allocate_nm([torch.from_numpy(W).cuda() for W in Ws], R)
+        assert np.allclose(np.sqrt(sums), norms, rtol=1e-13, atol=0)
+        want, _ = oracle.allocate_nm(norms, R)
+        assert got == [int(v) for v in want]

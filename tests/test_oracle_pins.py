@@ -441,3 +441,22 @@ def test_silu_mul_identities():
     assert np.array_equal(oracle.silu_mul(v, -one), -s)
     # fp16 output: every value is representable
     assert np.array_equal(s.astype(np.float16).astype(np.float64), s)
+
+
+def test_layerwise_nm_assignment():
+    """Section 3.3: alpha_i = omega_i / sum omega, N_i / 8 = alpha_i + (1 - alpha_i) R.  Hand-worked: norms (3, 1), R = 1/2:
+    alpha = (3/4, 1/4), ratios (7/8, 5/8), N = (7, 5).  Equal norms give equal N; the ratio never falls below R and
+    reaches 1 only for a layer that holds all the norm; the mean ratio is R + (1 - R) / L."""
+    N, ratio = oracle.allocate_nm([3.0, 1.0], 0.5)
+    assert list(N) == [7, 5] and np.allclose(ratio, [0.875, 0.625], rtol=0, atol=1e-15)
+    N, ratio = oracle.allocate_nm([2.0] * 32, 0.5)
+    assert len(set(N)) == 1 and N[0] == 4 and np.allclose(ratio.mean(), 0.5 + 0.5 / 32)
+    g = np.random.default_rng(3)
+    w = g.random(40) + 0.1
+    for R in (0.375, 0.5, 0.625, 0.75):
+        N, ratio = oracle.allocate_nm(w, R)
+        assert (ratio >= R).all() and (ratio < 1).all() and np.isclose(ratio.mean(), R + (1 - R) / 40)
+        assert (np.argsort(ratio, kind="stable") == np.argsort(w, kind="stable")).all()      # monotone in the norm
+        assert ((N >= 1) & (N <= 8)).all() and (np.abs(N - 8 * ratio) <= 0.5).all()
+    N, ratio = oracle.allocate_nm([5.0, 0.0, 0.0], 0.5)
+    assert list(N) == [8, 4, 4] and ratio[0] == 1.0
