@@ -133,6 +133,11 @@ __device__ __forceinline__ uint4 ldg_v4_coherent(const void* p) {      // the sa
   asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ uint32_t ldg_u16_coherent(const void* p) {
+  unsigned short v;
+  asm volatile("ld.global.u16 %0, [%1];" : "=h"(v) : "l"(p) : "memory");
+  return v;
+}
 // fp16 pair (bits) of silu(a) * b per half, in fp32, rounded to nearest even
 __device__ __forceinline__ uint32_t silu_mul_bits(uint32_t a, uint32_t b) {
   const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&a)), fb = __half22float2(*reinterpret_cast<const __half2*>(&b));
@@ -370,6 +375,8 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
   // activations of batch row g (this lane group's): in global memory, or staged in shared memory as a plain copy
   const __half* xg = nullptr;
   if (g < batch) xg = q.use_image == 2 ? reinterpret_cast<const __half*>(ximg) + (size_t)g * q.m : q.x + (size_t)g * q.ldx;
+  // (with the operand-order image the tiles read the image; the residual term takes its few activations from global
+  // memory unless the input is a formed one)
   const uint32_t img_row_words = (uint32_t)nb * kImgWordsPerBlock;
   int R = lo / nb, b_first = lo - R * nb, left = hi - lo, nslot_used = 0;
   while (left > 0 && !W.failed) {
@@ -455,7 +462,8 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
             fa[j][1] = hmul2_bits(prmt(unit, 0u, 0x3424u), s2);
           }
           uint2 xr = make_uint2(0, 0);
-          if constexpr (kImage) {
+          if (kImage && q.x2 != nullptr) {
+            // a formed input exists only in the image: pick the four values out of its operand order
             if (g < batch) {
               const uint32_t* ir = ximg + (uint32_t)g * img_row_words;
               xr.x = image_x(ir, block, cols & 0xFFu) | (image_x(ir, block, (cols >> 8) & 0xFFu) << 16);
@@ -463,8 +471,13 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
             }
           } else if (xg) {
             const __half* xq = xg + (size_t)block * kBlock;
-            xr.x = ld_u16(xq + (cols & 0xFFu)) | (ld_u16(xq + ((cols >> 8) & 0xFFu)) << 16);
-            xr.y = ld_u16(xq + ((cols >> 16) & 0xFFu)) | (ld_u16(xq + (cols >> 24)) << 16);
+            if constexpr (kImage) {        // global memory for sure
+              xr.x = ldg_u16_coherent(xq + (cols & 0xFFu)) | (ldg_u16_coherent(xq + ((cols >> 8) & 0xFFu)) << 16);
+              xr.y = ldg_u16_coherent(xq + ((cols >> 16) & 0xFFu)) | (ldg_u16_coherent(xq + (cols >> 24)) << 16);
+            } else {                       // global memory or the plain copy in shared memory
+              xr.x = ld_u16(xq + (cols & 0xFFu)) | (ld_u16(xq + ((cols >> 8) & 0xFFu)) << 16);
+              xr.y = ld_u16(xq + ((cols >> 16) & 0xFFu)) | (ld_u16(xq + (cols >> 24)) << 16);
+            }
           }
           mma16816(acc[0], fa[0][0], fa[1][0], fa[0][1], fa[1][1], xr.x, xr.y);
           mma16816(acc[1], fa[2][0], fa[3][0], fa[2][1], fa[3][1], xr.x, xr.y);
