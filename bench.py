@@ -350,7 +350,7 @@ def gemv_table(stb, torch, wl, pk):
     return out, ctx
 
 
-def gemm_table(stb, torch, pk, real_ffn):
+def gemm_table(stb, torch, pk, real_ffn, only=None):
     """Prefill GEMM (stb_gemm, tcgen05) on the LLaMA-2-70B linear shapes at 4:8, 2048 bf16 tokens, with a
     dense bf16 cuBLAS GEMM (torch.matmul) of the same shape beside it.  q/o and k/v are quantizer-made.  The
     two tall / wide FFN layers take the CPU quantizer minutes, so by default they are built on the device by
@@ -389,6 +389,8 @@ def gemm_table(stb, torch, pk, real_ffn):
                   ("down 8192x28672", 8192, 28672, cols_x(b), "column blocks of the quantized q layer repeated 3.5 times", None)]
     out = []
     for name, n, m, t, how, hist in cases:
+        if only and not name.startswith(only):
+            continue
         lay = stb.pack(n, m, N, t["keep"], t["sign"], t["region"], t["sign2"], t["salient"], t["scale"])
         torch.cuda.synchronize()
         assert int(lay.dev_status.item()) == 0, name
@@ -556,6 +558,10 @@ def cuda_arm(args):
     import paper_2408_01803_b200 as stb
     pk = peaks()
 
+    if args.only_gemm:
+        # one prefill shape alone (for a profiler capture of stb::gemm_kernel)
+        print(json.dumps({"gemm_prefill": gemm_table(stb, torch, pk, False, only=args.only_gemm)}))
+        return
     copies = args.copies          # 12 distinct copies of the three layers per rotation: more than 6 x L2
     if world > 1 and rank != 0:
         dist.barrier()   # rank 0 quantizes (and caches) the layers first
@@ -739,6 +745,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--copies", type=int, default=12, help="distinct packed copies of the layers per rotation (cold L2 needs >= 3)")
     ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S, help="shortest timed region; 0 for a profiler capture")
+    ap.add_argument("--only-gemm", default=None, help="run only the prefill GEMM shape whose name starts with this (q/o, k/v, gate/up, down)")
     ap.add_argument("--per-layer-launches", action="store_true", help="headline through stb_layer_stack instead of stb_layer_stack_resident")
     ap.add_argument("--real-ffn", action="store_true", help="prefill GEMM: quantize the real 28672-wide FFN layers (CPU minutes)")
     args = ap.parse_args()

@@ -105,6 +105,9 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const void* p) {
   unsigned long long v;
   asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -296,7 +299,7 @@ __device__ __forceinline__ void tile_sp6(const LaneTile<6>& lt, const uint32_t (
 
 // One tile in position order (N = 4, 5, 6): byte-permute decode into m16n8k16 operands; activations of batch row g
 // through L1 (xrow = x + g ldx + 8 t + 128 b, or null for lanes beyond the batch).
-template <int N>
+template <int N, bool kStaged>
 __device__ __forceinline__ void tile_dense(const LaneTile<N>& lt, const uint2* ptab, const __half* xrow, float (&acc)[2][4]) {
   FastRows<N> fr;
   fr.init(lt, lt.A, lt.B);
@@ -312,7 +315,7 @@ __device__ __forceinline__ void tile_dense(const LaneTile<N>& lt, const uint2* p
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
     xf[s] = make_uint4(0, 0, 0, 0);
-    if (xrow) xf[s] = ld_v4(xrow + s * 32);
+    if (xrow) xf[s] = kStaged ? ld_v4(xrow + s * 32) : ldg_v4_coherent(xrow + s * 32);
   }
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
@@ -364,7 +367,8 @@ __device__ __forceinline__ void ring_issue(const WarpEnv& E, WarpState& W, int s
 }
 
 // The warp's tiles [lo, hi) of phase q: main stream, residual term per span, partial sums out.
-template <int N, bool kImage>
+// kImage: 6:8 from the operand-order image; kStaged: position order with the activations in a plain copy in shared memory
+template <int N, bool kImage, bool kStaged>
 __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const StackPhase& q, int lo, int hi,
                                           const uint32_t* ximg, PartSlot* pslot, float* pdata, volatile int* ctl) {
   const StackParams& P = *E.P;
@@ -428,7 +432,7 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
         if (last_of_chunk) { __syncwarp(); ring_issue(E, W, slot); W.cur_in = 0; ++W.consumed; }
         else ++W.cur_in;
         if constexpr (kImage) tile_sp6(lt, fld, E.smem, ximg + (uint32_t)g * img_row_words + (uint32_t)b * kImgWordsPerBlock + (uint32_t)(t * 24), g < batch, acc);
-        else tile_dense<N>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
+        else tile_dense<N, kStaged>(lt, ptab, xg ? xg + (size_t)b * kBlock + t * 8 : nullptr, acc);
       }
       if (W.failed) break;
 
@@ -471,7 +475,7 @@ __device__ __forceinline__ void run_tiles(const WarpEnv& E, WarpState& W, const 
             }
           } else if (xg) {
             const __half* xq = xg + (size_t)block * kBlock;
-            if constexpr (kImage) {        // global memory for sure
+            if constexpr (!kStaged) {      // global memory for sure
               xr.x = ldg_u16_coherent(xq + (cols & 0xFFu)) | (ldg_u16_coherent(xq + ((cols >> 8) & 0xFFu)) << 16);
               xr.y = ldg_u16_coherent(xq + ((cols >> 16) & 0xFFu)) | (ldg_u16_coherent(xq + (cols >> 24)) << 16);
             } else {                       // global memory or the plain copy in shared memory
@@ -636,10 +640,14 @@ stack_kernel(const __grid_constant__ StackParams P) {
 
     // ---- this warp's tiles ----
     if (!W.failed && wl < wh) {
-      if (q.N == 6 && q.use_image == 1) run_tiles<6, true>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
-      else if (q.N == 6) run_tiles<6, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
-      else if (q.N == 5) run_tiles<5, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
-      else run_tiles<4, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      if (q.N == 6 && q.use_image == 1) run_tiles<6, true, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      else if (q.use_image == 2) {
+        if (q.N == 6) run_tiles<6, false, true>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+        else if (q.N == 5) run_tiles<5, false, true>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+        else run_tiles<4, false, true>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      } else if (q.N == 6) run_tiles<6, false, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      else if (q.N == 5) run_tiles<5, false, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
+      else run_tiles<4, false, false>(E, W, q, wl, wh, ximg, pslot, pdata, ctl);
     }
     if (W.failed && lane == 0 && !ctl[0]) {
       // this warp's own wait ran out: tell the CTA and the grid
@@ -720,7 +728,9 @@ stack_kernel(const __grid_constant__ StackParams P) {
     if (threadIdx.x == 0) {
       const int fin = ctl[1];
       ctl[1] = 0;
-      if (fin > 0 && !ctl[0]) { __threadfence(); atomicAdd(P.sync, (uint32_t)fin); }
+      // release at GPU scope: the CTA's stores to y (ordered before this thread by the barrier) are visible to
+      // whoever sees the count
+      if (fin > 0 && !ctl[0]) red_release_add(P.sync, (uint32_t)fin);
     }
   }
 
