@@ -352,10 +352,9 @@ def gemv_table(stb, torch, wl, pk):
 
 def gemm_table(stb, torch, pk, real_ffn, only=None):
     """Prefill GEMM (stb_gemm, tcgen05) on the LLaMA-2-70B linear shapes at 4:8, 2048 bf16 tokens, with a
-    dense bf16 cuBLAS GEMM (torch.matmul) of the same shape beside it.  q/o and k/v are quantizer-made.  The
-    two tall / wide FFN layers take the CPU quantizer minutes, so by default they are built on the device by
-    repeating the rows / column blocks of the quantizer-made 8192 x 8192 layer (valid layers with the same
-    salient-column statistics; --real-ffn quantizes the real ones, as tests/ do)."""
+    dense bf16 cuBLAS GEMM (torch.matmul) of the same shape beside it.  q/o and k/v come from the oracle's
+    quantizer; the two tall / wide FFN layers (minutes on the CPU) from stb_quantize on the GPU, which the parity
+    tests hold equal to the oracle bit for bit (--tiled-ffn: repeat the quantized q layer instead)."""
     T, N = 2048, 4
     views = {"keep": np.uint8, "sign": np.uint8, "region": np.int16, "sign2": np.int32, "salient": np.int64, "scale": np.int16}
 
@@ -375,15 +374,29 @@ def gemm_table(stb, torch, pk, real_ffn, only=None):
                 out[k] = torch.cat([v] * 3 + [v[:, :half]], 1).contiguous()
         return out
 
+    def on_gpu(name):
+        # the workload's dense weights through stb_quantize (equal to the oracle's quantizer bit for bit in the parity tests)
+        n, m, NN, seed = si.workload_layer(4, name)
+        W = torch.from_numpy(si.dense_weight(n, m, seed)).cuda()
+        xn = torch.from_numpy(si.calib_norms(m, seed)).cuda()
+        t = stb.quantize(W, xn, NN)
+        torch.cuda.synchronize()
+        del W
+        sal = t["salient"].cpu().numpy().view(np.uint64)
+        return t, salient_histogram({"salient": sal})
+
     dq = quantized(4, "q")
     b = up(dq)
     cases = [("q/o 8192x8192", 8192, 8192, b, "oracle-quantized", salient_histogram(dq))]
     dk = quantized(4, "k")
     cases.append(("k/v 1024x8192", 1024, 8192, up(dk), "oracle-quantized", salient_histogram(dk)))
     if real_ffn:
-        dg, dd = quantized(4, "gate"), quantized(4, "down")
-        cases += [("gate/up 28672x8192", 28672, 8192, up(dg), "oracle-quantized", salient_histogram(dg)),
-                  ("down 8192x28672", 8192, 28672, up(dd), "oracle-quantized", salient_histogram(dd))]
+        tg, hg = on_gpu("gate")
+        cases.append(("gate/up 28672x8192", 28672, 8192, tg, "stb_quantize (GPU quantizer) of the workload's dense weights", hg))
+        del tg
+        td, hd = on_gpu("down")
+        cases.append(("down 8192x28672", 8192, 28672, td, "stb_quantize (GPU quantizer) of the workload's dense weights", hd))
+        del td
     else:
         cases += [("gate/up 28672x8192", 28672, 8192, rows_x(b), "rows of the quantized q layer repeated 3.5 times", None),
                   ("down 8192x28672", 8192, 28672, cols_x(b), "column blocks of the quantized q layer repeated 3.5 times", None)]
@@ -516,6 +529,25 @@ def stack_tables(stb, torch, pk):
     del l7
     torch.cuda.empty_cache()
     return out
+
+
+def quantizer_timing(stb, torch):
+    """stb_quantize on the dense gate layer of the workload (11008 x 4096, 6:8): milliseconds, with the oracle's time for
+    the same layer beside it when it was measured in this run."""
+    n, m, N, seed = si.workload_layer(2, "gate")
+    W = torch.from_numpy(si.dense_weight(n, m, seed)).cuda()
+    xn = torch.from_numpy(si.calib_norms(m, seed)).cuda()
+    stb.quantize(W, xn, N)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        stb.quantize(W, xn, N)
+    e1.record()
+    torch.cuda.synchronize()
+    return {"layer": "gate 11008x4096 6:8", "ms": round(e0.elapsed_time(e1) / 3, 2),
+            "note": "Eq. 3, N of 8, salient search (32 candidates), break-point search (160 grid points), residual + trisection, "
+                    "float64; equals the oracle's output bit for bit (parity tests)"}
 
 
 def pack_timing(stb, torch, wl):
@@ -697,9 +729,10 @@ def cuda_arm(args):
         iso = [r for r in tab if r["batch"] == 1 and r["N"] == 6]
         line["roofline"]["isolated_launch_frac"] = round(float(np.mean([r["frac_of_measured_hbm"] for r in iso])), 4)
         line["dense_context"] = ctx
-        line["gemm_prefill"] = gemm_table(stb, torch, pk, args.real_ffn)
+        line["gemm_prefill"] = gemm_table(stb, torch, pk, not args.tiled_ffn)
         line["gemm_prefill_note"] = "fractions of the MEASURED cuBLAS bf16 burst peak (%s TFLOP/s) decide the 50 %% target; fractions of the nominal 2250 TFLOP/s are printed beside them" % pk["bf16_tflops"]
         line["pack"] = pack_timing(stb, torch, wl)
+        line["quantizer"] = quantizer_timing(stb, torch)
         st = stack_tables(stb, torch, pk)
         line["decode_stacks"] = st
         big = [r for r in st if r.get("batch") == 1 and "roofline" in r][0]
@@ -747,7 +780,8 @@ def main():
     ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S, help="shortest timed region; 0 for a profiler capture")
     ap.add_argument("--only-gemm", default=None, help="run only the prefill GEMM shape whose name starts with this (q/o, k/v, gate/up, down)")
     ap.add_argument("--per-layer-launches", action="store_true", help="headline through stb_layer_stack instead of stb_layer_stack_resident")
-    ap.add_argument("--real-ffn", action="store_true", help="prefill GEMM: quantize the real 28672-wide FFN layers (CPU minutes)")
+    ap.add_argument("--tiled-ffn", action="store_true", help="prefill GEMM: build the 28672-wide FFN layers by repeating the quantized "
+                                                             "q layer instead of quantizing the real ones on the GPU")
     args = ap.parse_args()
     args.steps = args.steps or 20
     if args.impl == "reference":

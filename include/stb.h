@@ -241,6 +241,18 @@ int stb_layer_stack_checksum(const stb_step *steps, int count, unsigned long lon
 int stb_layer_stack_host(const stb_step *steps, int count, const void *in_host, size_t in_bytes,
                          void *out_host, size_t out_bytes, int *dev_status, void *stream);
 
+/* The quantizer on the GPU: Standardized Importance (Eq. 3), N of 8 per group (Section 3.3), the salient-column
+ * search and the break-point search of Algorithm 2 (32 candidate columns, 160 grid points, sigma = 2), residual
+ * binarization (Eq. 4) and trisection: the block loop of Algorithm 1 without its Hessian update (column score with
+ * the diagonal h_jj = 2 ||X_:,j||^2; lambda < 0 selects 0.01 mean_j h_jj).  W: dense fp16 [n][ldw]; xnorm: float64
+ * [m], the column norms of the calibration activations; out: a stb_logical whose n, m, N match and whose six DEVICE
+ * arrays (sizes as documented at stb_logical) are WRITTEN here, ready for stb_pack.  float64 throughout; sums that
+ * are not exact are taken in the order of the definition, so the result does not depend on the launch shape.
+ * ws: DEVICE workspace of stb_quantize_workspace bytes, 256-byte aligned.  About a dozen launches on `stream`. */
+int stb_quantize_workspace(int n, int m, size_t *bytes);
+int stb_quantize(const void *W, size_t ldw, const double *xnorm, int n, int m, int N, double lambda,
+                 const stb_logical *out, void *ws, size_t ws_bytes, void *stream);
+
 /* Layer-wise N:M assignment (Section 3.3): more important layers, by the L2 norm of their weights, keep more of
  * every 8.  stb_weight_sumsq adds the sum of squares of a dense fp16 matrix W[n][ldw] (DEVICE, 16-byte aligned, ldw a
  * multiple of 8) to *sumsq (DEVICE float64, zeroed by the caller; one launch).  stb_allocate_nm is HOST arithmetic on

@@ -24,7 +24,7 @@ STB_IN_PLAIN, STB_IN_SILU_MUL = 0, 1
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
            "stb_gemm_workspace", "stb_gemm_workspace_min", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
            "stb_layer_stack_resident_workspace", "stb_layer_stack_resident", "stb_layer_stack_resident_host",
-           "stb_layer_stack_resident_wait_selftest", "stb_layer_stack_checksum", "stb_weight_sumsq",
+           "stb_layer_stack_resident_wait_selftest", "stb_layer_stack_checksum", "stb_quantize_workspace", "stb_quantize", "stb_weight_sumsq",
            "stb_allocate_nm", "stb_status_str"]
 
 
@@ -74,6 +74,8 @@ def _load():
     lib.stb_layer_stack_resident_wait_selftest.argtypes = [p(_Step), i, v, z, v, v]
     lib.stb_layer_stack_resident_host.argtypes = [p(_Step), i, v, z, v, z, v, z, v, v]
     lib.stb_layer_stack_checksum.argtypes = [p(_Step), i, v, v, v]
+    lib.stb_quantize_workspace.argtypes = [i, i, p(z)]
+    lib.stb_quantize.argtypes = [v, z, v, i, i, i, C.c_double, p(_Logical), v, z, v]
     lib.stb_weight_sumsq.argtypes = [v, i, i, z, v, v]
     lib.stb_allocate_nm.argtypes = [p(C.c_double), i, C.c_double, p(i)]
     lib.stb_status_str.argtypes = [i]
@@ -327,3 +329,25 @@ def allocate_nm(weights, r_target, stream=None):
     out = (C.c_int * len(weights))()
     _check(_lib.stb_allocate_nm(arr, len(weights), float(r_target), out), "stb_allocate_nm")
     return [int(vv) for vv in out], host
+
+
+def quantize(W, xnorm, N, lam=-1.0, stream=None):
+    """stb_quantize: dense fp16 CUDA matrix W[n][m] + float64 CUDA column norms xnorm[m] -> dict of logical CUDA
+    tensors (keep, sign, region, sign2, salient, scale; the argument order of pack())."""
+    import torch
+    assert W.dtype == torch.float16 and W.is_cuda and W.dim() == 2 and W.stride(1) == 1
+    assert xnorm.dtype == torch.float64 and xnorm.is_cuda and xnorm.is_contiguous()
+    n, m = W.shape
+    dev = W.device
+    out = {"keep": torch.empty((n, m // 8), dtype=torch.uint8, device=dev), "sign": torch.empty((n, m // 8), dtype=torch.uint8, device=dev),
+           "region": torch.empty((n, m // 8), dtype=torch.int16, device=dev), "sign2": torch.empty((n, m // 128), dtype=torch.int32, device=dev),
+           "salient": torch.empty((m // 128, 2), dtype=torch.int64, device=dev), "scale": torch.empty((n, m // 128, 5), dtype=torch.int16, device=dev)}
+    need = C.c_size_t()
+    _check(_lib.stb_quantize_workspace(n, m, C.byref(need)), "stb_quantize_workspace")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=dev)
+    L = _Logical(n, m, N, out["keep"].data_ptr(), out["sign"].data_ptr(), out["region"].data_ptr(), out["sign2"].data_ptr(),
+                 out["salient"].data_ptr(), out["scale"].data_ptr())
+    _check(_lib.stb_quantize(_ptr(W), W.stride(0), _ptr(xnorm), n, m, N, float(lam), C.byref(L), _ptr(ws), ws.numel(), _stream(stream)),
+           "stb_quantize")
+    out.update(n=n, m=m, N=N)
+    return out

@@ -155,7 +155,6 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
   const int rtile = mt * 4 + q;                 // packed row tile
   const bool live = rtile < ntile;
   const uint32_t* ptab = reinterpret_cast<const uint32_t*>(smem + kGemmTab);     // low half: columns 0..3, high half: 4..7
-  const BlockInfo* binfo = reinterpret_cast<const BlockInfo*>(packed + sizeof(Header));
   const uint8_t* rtbase = packed + hdr->tiles_offset + (size_t)rtile * hdr->rt_stride;
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
                             (size_t)rtile * resid_rt_bytes(nblk, hdr->nrw);

@@ -476,3 +476,40 @@ def test_layerwise_nm_assignment_from_dense_weights(stb):
         assert np.allclose(np.sqrt(sums), norms, rtol=1e-13, atol=0)
         want, _ = oracle.allocate_nm(norms, R)
         assert got == [int(v) for v in want]
+
+
+def _gpu_quantize(stb, torch, n, m, N, seed):
+    W = si.dense_weight(n, m, seed)
+    xn = si.calib_norms(m, seed)
+    return stb.quantize(torch.from_numpy(W).cuda(), torch.from_numpy(xn).cuda(), N), W, xn
+
+
+def _same_logical(got, L):
+    views = {"keep": np.uint8, "sign": np.uint8, "region": np.uint16, "sign2": np.uint32, "salient": np.uint64, "scale": np.uint16}
+    for k, v in views.items():
+        g = got[k].cpu().numpy().view(v)
+        assert np.array_equal(g, getattr(L, k)), k
+
+
+@pytest.mark.parametrize("N", [1, 3, 4, 5, 6, 8])
+@pytest.mark.parametrize("n,m", [(40, 256), (300, 384)])
+def test_gpu_quantizer_matches_the_oracle_bit_for_bit(stb, N, n, m):
+    """stb_quantize against the oracle's quantizer on the same dense weights and calibration norms: keep masks, signs,
+    region codes, residual signs, salient masks and fp16 scales, all equal."""
+    import torch
+    got, W, xn = _gpu_quantize(stb, torch, n, m, N, 3000 + 10 * N + n)
+    L, _, _ = oracle.quantize(W.astype(np.float64), xn, N)
+    _same_logical(got, L)
+    layer = stb.pack(n, m, N, got["keep"], got["sign"], got["region"], got["sign2"], got["salient"], got["scale"])
+    torch.cuda.synchronize()
+    assert int(layer.dev_status.item()) == 0
+    assert np.array_equal(stb.dequant(layer).cpu().numpy(), oracle.decode(L))
+
+
+def test_gpu_quantizer_full_size_layer(stb):
+    """The 7B down projection (4096 x 11008 at 6:8): the GPU quantizer's logical arrays equal the oracle's."""
+    import torch
+    n, m, N, seed = si.workload_layer(2, "down")
+    got, W, xn = _gpu_quantize(stb, torch, n, m, N, seed)
+    torch.cuda.synchronize()
+    _same_logical(got, wl.as_logical(wl.quantized_layer(n, m, N, seed)))
