@@ -8,7 +8,7 @@
 //   B = kAcc slices of 256 x 64 bf16 of X, brought in by TMA with the same swizzle; every decoded
 //       A stage is multiplied with all of them (kAcc accumulators of 256 TMEM columns), which
 //       divides the decode work per flop by kAcc,
-// in a ring of kStages stages over K.  Warp roles:
+// in rings over K (kStagesA decoded A stages, kStagesB X stages: the decode warps run ahead of the tensor core).  Warp roles:
 //   warp 0      TMA producer (one lane): X slices
 //   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage and accumulator,
 //               tcgen05.commit frees the stage; also allocates / frees TMEM
@@ -47,16 +47,20 @@ constexpr int kBN = 256;          // tokens per accumulator (UMMA N)
 constexpr int kAcc = 2;                         // accumulators per CTA: a decoded A stage is used kAcc times
 constexpr int kTok = kBN * kAcc;                // tokens per CTA
 constexpr int kBK = 64;           // K per stage: one 128-byte swizzle row of bf16
-constexpr int kStages = 2;
+constexpr int kStagesA = 4;        // ring of decoded A stages (16 KB each)
+constexpr int kStagesB = 5;        // ring of X boxes (256 tokens x 64 of K = 32 KB each; a stage of K takes kAcc of them): what
+                                   // is in flight from L2 is what hides its latency, so the ring is deep and its slots small
 constexpr int kGroups = 4;                              // decode warps per 32-row quarter: one per row of a lane
 constexpr int kGemmThreads = 64 + 128 * kGroups;
 constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
-constexpr uint32_t kStageB = kTok * kBK * 2;     // 32 KB per accumulator
+constexpr uint32_t kStageB = kBN * kBK * 2;      // 32 KB: one box
 constexpr uint32_t kGemmTab = 0;                                   // position table (576 B)
-constexpr uint32_t kGemmBars = 1024;                               // full[4], empty[4], accum, tmem slot, abort
+constexpr uint32_t kGemmBars = 1024;                               // fullA, emptyA, fullB, emptyB, accum, tmem slot, abort
 constexpr uint32_t kGemmA = 2048;                                  // 1024-byte aligned stages
-constexpr uint32_t kGemmB = kGemmA + kStages * kStageA;
-constexpr uint32_t kGemmSmem = kGemmB + kStages * kStageB;         // 198656 B
+constexpr uint32_t kGemmB = kGemmA + kStagesA * kStageA;
+constexpr uint32_t kGemmSmem = kGemmB + kStagesB * kStageB;        // 231424 B
+static_assert(kGemmSmem <= 232448, "one CTA's shared memory");
+static_assert(8 * (2 * kStagesA + 2 * kStagesB + 1) + 16 <= 1024, "barrier area");
 constexpr long long kGemmWaitLimit = 2000000000ll;
 
 // ---- tcgen05 / TMA wrappers ---------------------------------------------------------------
@@ -129,7 +133,7 @@ __device__ __forceinline__ uint32_t bf16_bits(uint32_t h16) {
 // What a decode warp needs to know.
 struct DecodeArgs {
   const uint8_t* packed; const Header* hdr; uint8_t* smem; volatile int* abort_flag;
-  uint32_t bar_full, bar_empty;
+  uint32_t bar_full, bar_empty;      // of the A ring
   int mt, b0, b1, nblk, ntile, q, lane;
   uint32_t rw0, rw1;        // residual words of the blocks [b0, b1)
   int nres;                 // residual stages (64 slots = 16 words each, the first one starts at word rw0 & ~1)
@@ -159,11 +163,13 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
   const uint8_t* resid_rt = packed + hdr->tiles_offset + hdr->rt_stride * (size_t)ntile +
                             (size_t)rtile * resid_rt_bytes(nblk, hdr->nrw);
   constexpr uint32_t tbytes = tile_bytes(N);
-  RowWords cur = {}, nxt = {};
-  if (live && b0 < b1) load_row_words<N>(rtbase + (size_t)b0 * tbytes, lane, j, cur);
-  bool ok = true;
-  for (int b = b0; b < b1 && ok; ++b) {
-    if (live && b + 1 < b1) load_row_words<N>(rtbase + (size_t)(b + 1) * tbytes, lane, j, nxt);
+  // The row's words are loaded three blocks ahead of their use (three sets of registers in rotation): the loads
+  // come straight from HBM, and one block of decode is shorter than their latency.
+  RowWords w0 = {}, w1 = {}, w2 = {};
+  auto fetch = [&](int b, RowWords& w) {
+    if (live && b < b1) load_row_words<N>(rtbase + (size_t)b * tbytes, lane, j, w);
+  };
+  auto block = [&](int b, const RowWords& cur) -> bool {
     // bf16 scale bytes of the row (a salient weight gets s1 bf16(a_sal1) here; its residual term comes with the residual stages)
     uint32_t A16 = 0, B16 = 0;
     if (live) {
@@ -183,9 +189,9 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
     for (int sidx = 0; sidx < 4; ++sidx) P[sidx] = live ? ptab[(cur.mask >> (8 * sidx)) & 0xFFu] : 0u;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const int it = 2 * (b - b0) + h, st = it % kStages;
+      const int it = 2 * (b - b0) + h, st = it % kStagesA;
       // the verdict is made warp-uniform: nobody may be left alone at the __syncwarp() below
-      if (!__all_sync(0xFFFFFFFFu, gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
+      if (!__all_sync(0xFFFFFFFFu, gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStagesA) & 1u) ^ 1u, abort_flag))) return false;
       uint8_t* As = smem + kGemmA + st * kStageA;
       uint8_t* rowp = As + (size_t)(4 * q + j) * 1024 + g * 128;
       if (N == 6 && live) row.high(h);
@@ -201,36 +207,51 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_full + 8 * st);
     }
-    if (!ok) break;
-    if (live && b + 1 < b1) cur = nxt;
-  }
-
-  // Residual stages: 64 residual slots (16 residual words) of K each.  The lane writes the same two 16-byte chunks
-  // of its row as above: chunk c holds the words 2 c and 2 c + 1 of the stage, four slots each, as +-bf16(a_sal2) or 0.
+    return true;
+  };
+  // Residual stages (after the blocks): 64 residual slots (16 residual words) of K each.  The lane writes the same
+  // two 16-byte chunks of its row as above: chunk c holds the words 2 c and 2 c + 1 of the stage, four slots each,
+  // as +-bf16(a_sal2) or 0.  What a stage needs sits behind two dependent loads from global memory (the word's table
+  // entry, then a_sal2 and the codes from the block's record), so both are taken ahead: the entries two stages, the
+  // records one stage before their use, the first ones before the blocks.
   const ResidWord* rwt = reinterpret_cast<const ResidWord*>(packed + rwtab_offset(nblk));
   const uint32_t wfirst = da.rw0 & ~1u;
-  for (int rs = 0; rs < da.nres && ok; ++rs) {
-    const int it = 2 * (b1 - b0) + rs, st = it % kStages;
+  auto res_word = [&](int rs, int idx) { return wfirst + 16u * (uint32_t)rs + 2u * (uint32_t)(4 * (idx >> 1) + t) + (uint32_t)(idx & 1); };
+  auto res_entries = [&](int rs, uint2 (&e)[4], uint32_t& valid) {
+    valid = 0;
+#pragma unroll
+    for (int idx = 0; idx < 4; ++idx) {
+      const uint32_t w = res_word(rs, idx);
+      e[idx] = make_uint2(0u, 0u);
+      if (live && rs < da.nres && w >= da.rw0 && w < da.rw1) { e[idx] = __ldg(reinterpret_cast<const uint2*>(rwt + w)); valid |= 1u << idx; }
+    }
+  };
+  auto res_records = [&](int rs, const uint2 (&e)[4], uint32_t valid, uint32_t (&a2)[4], uint32_t (&word)[4]) {
+#pragma unroll
+    for (int idx = 0; idx < 4; ++idx) {
+      a2[idx] = 0; word[idx] = 0;
+      if ((valid >> idx) & 1u) {
+        const uint8_t* rec = resid_rt + resid_block_off((int)(e[idx].x >> 3), res_word(rs, idx) - (e[idx].x & 7u));
+        a2[idx] = __ldg(reinterpret_cast<const uint16_t*>(rec + resid_a2_off(g, j)));
+        word[idx] = __ldg(reinterpret_cast<const uint32_t*>(rec + resid_code_off(e[idx].x & 7u, g)));
+      }
+    }
+  };
+  auto res_stage = [&](int rs, uint32_t valid, const uint32_t (&a2)[4], const uint32_t (&word)[4]) -> bool {
+    const int it = 2 * (b1 - b0) + rs, st = it % kStagesA;
     uint32_t f[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
 #pragma unroll
-    for (int sl = 0; sl < 2; ++sl)
-#pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const uint32_t w = wfirst + 16u * (uint32_t)rs + 2u * (uint32_t)(4 * sl + t) + (uint32_t)k;
-        if (live && w >= da.rw0 && w < da.rw1) {
-          const uint2 e = __ldg(reinterpret_cast<const uint2*>(rwt + w));
-          const uint8_t* rec = resid_rt + resid_block_off((int)(e.x >> 3), w - (e.x & 7u));
-          const uint32_t v = bf16_bits(__ldg(reinterpret_cast<const uint16_t*>(rec + resid_a2_off(g, j))));
-          const uint32_t word = __ldg(reinterpret_cast<const uint32_t*>(rec + resid_code_off(e.x & 7u, g)));
-          const uint32_t L2 = prmt(v, 0u, 0x4040u);                 // (lo, 0, lo, 0)
-          const uint32_t H2 = prmt(v, v ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
-          const uint32_t sel = resid_selector(word, j);
-          const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
-          f[sl][2 * k] = prmt(lo4, hi4, 0x5140u);
-          f[sl][2 * k + 1] = prmt(lo4, hi4, 0x7362u);
-        }
+    for (int idx = 0; idx < 4; ++idx)
+      if ((valid >> idx) & 1u) {
+        const uint32_t v = bf16_bits(a2[idx]);
+        const uint32_t L2 = prmt(v, 0u, 0x4040u);                 // (lo, 0, lo, 0)
+        const uint32_t H2 = prmt(v, v ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
+        const uint32_t sel = resid_selector(word[idx], j);
+        const uint32_t lo4 = prmt(L2, L2, sel), hi4 = prmt(H2, H2, sel);
+        f[idx >> 1][2 * (idx & 1)] = prmt(lo4, hi4, 0x5140u);
+        f[idx >> 1][2 * (idx & 1) + 1] = prmt(lo4, hi4, 0x7362u);
       }
-    if (!__all_sync(0xFFFFFFFFu, gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
+    if (!__all_sync(0xFFFFFFFFu, gemm_wait(bar_empty + 8 * st, ((uint32_t)(it / kStagesA) & 1u) ^ 1u, abort_flag))) return false;
     uint8_t* rowp = smem + kGemmA + st * kStageA + (size_t)(4 * q + j) * 1024 + g * 128;
 #pragma unroll
     for (int sl = 0; sl < 2; ++sl)
@@ -238,6 +259,31 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
     fence_async_smem();
     __syncwarp();
     if (lane == 0) mbar_arrive(bar_full + 8 * st);
+    return true;
+  };
+  uint2 eX[4], eY[4];
+  uint32_t veX = 0, veY = 0, vrX = 0, vrY = 0, a2X[4], a2Y[4], wdX[4], wdY[4];
+  res_entries(0, eX, veX);
+  fetch(b0, w0);
+  fetch(b0 + 1, w1);
+  res_records(0, eX, veX, a2X, wdX); vrX = veX;
+  res_entries(1, eY, veY);
+  bool ok = true;
+  for (int b = b0; b < b1 && ok; b += 3) {
+    fetch(b + 2, w2);
+    ok = block(b, w0);
+    if (ok && b + 1 < b1) { fetch(b + 3, w0); ok = block(b + 1, w1); }
+    if (ok && b + 2 < b1) { fetch(b + 4, w1); ok = block(b + 2, w2); }
+  }
+  for (int rs = 0; rs < da.nres && ok; rs += 2) {
+    res_records(rs + 1, eY, veY, a2Y, wdY); vrY = veY;
+    res_entries(rs + 2, eX, veX);
+    ok = res_stage(rs, vrX, a2X, wdX);
+    if (ok && rs + 1 < da.nres) {
+      res_records(rs + 2, eX, veX, a2X, wdX); vrX = veX;
+      res_entries(rs + 3, eY, veY);
+      ok = res_stage(rs + 1, vrY, a2Y, wdY);
+    }
   }
 }
 
@@ -298,12 +344,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
   const int nstage = nmain + nres;
 
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar_full = sbase + kGemmBars, bar_empty = bar_full + 8 * kStages, bar_accum = bar_empty + 8 * kStages;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kGemmBars + 8 * (2 * kStages + 1));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kGemmBars + 8 * (2 * kStages + 1) + 8);
+  // A ring: full = the 16 decode warps have written the stage, empty = the tensor core has read it;
+  // B ring: full = the X boxes have landed, empty = the tensor core has read them
+  const uint32_t bar_fullA = sbase + kGemmBars, bar_emptyA = bar_fullA + 8 * kStagesA;
+  const uint32_t bar_fullB = bar_emptyA + 8 * kStagesA, bar_emptyB = bar_fullB + 8 * kStagesB, bar_accum = bar_emptyB + 8 * kStagesB;
+  constexpr uint32_t kBarBytes = 8 * (2 * kStagesA + 2 * kStagesB + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kGemmBars + kBarBytes);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kGemmBars + kBarBytes + 8);
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 1 + 4 * kGroups); mbar_init(bar_empty + 8 * i, 1); }
+    for (int i = 0; i < kStagesA; ++i) { mbar_init(bar_fullA + 8 * i, 4 * kGroups); mbar_init(bar_emptyA + 8 * i, 1); }
+    for (int i = 0; i < kStagesB; ++i) { mbar_init(bar_fullB + 8 * i, 1); mbar_init(bar_emptyB + 8 * i, 1); }
     mbar_init(bar_accum, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -320,16 +371,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      for (int it = 0; it < nstage; ++it) {
-        const int s = it % kStages;
-        if (!gemm_wait<true>(bar_empty + 8 * s, ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag)) break;
-        mbar_expect_tx(bar_full + 8 * s, box_bytes * kAcc);
-#pragma unroll
-        for (int a = 0; a < kAcc; ++a) {
-          const uint32_t dst = sbase + kGemmB + s * kStageB + a * (kBN * kBK * 2);
-          if (it < nmain) tma_load_2d(dst, &xmap, (b0 * 2 + it) * kBK, tt * kTok + a * kBN, bar_full + 8 * s);
-          else tma_load_2d(dst, &xsmap, (int)(4u * (rw0 & ~1u)) + (it - nmain) * kBK, tt * kTok + a * kBN, bar_full + 8 * s);
-        }
+      for (int hb = 0; hb < nstage * kAcc; ++hb) {
+        const int it = hb / kAcc, a = hb % kAcc, s = hb % kStagesB;
+        if (!gemm_wait<true>(bar_emptyB + 8 * s, ((uint32_t)(hb / kStagesB) & 1u) ^ 1u, abort_flag)) break;
+        mbar_expect_tx(bar_fullB + 8 * s, box_bytes);
+        const uint32_t dst = sbase + kGemmB + s * kStageB;
+        if (it < nmain) tma_load_2d(dst, &xmap, (b0 * 2 + it) * kBK, tt * kTok + a * kBN, bar_fullB + 8 * s);
+        else tma_load_2d(dst, &xsmap, (int)(4u * (rw0 & ~1u)) + (it - nmain) * kBK, tt * kTok + a * kBN, bar_fullB + 8 * s);
       }
       if (*abort_flag) {       // let copies in flight land before the CTA gives its shared memory up
         const long long t0 = clock64();
@@ -339,19 +387,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      for (int it = 0; it < nstage; ++it) {
-        const int s = it % kStages;
-        if (!gemm_wait<true>(bar_full + 8 * s, (uint32_t)(it / kStages) & 1u, abort_flag)) break;
-        tc_fence_after();
-        const uint64_t ad = umma_desc(sbase + kGemmA + s * kStageA);
+      bool go = true;
+      for (int it = 0; it < nstage && go; ++it) {
+        const int sa = it % kStagesA;
+        if (!gemm_wait<true>(bar_fullA + 8 * sa, (uint32_t)(it / kStagesA) & 1u, abort_flag)) break;
+        const uint64_t ad = umma_desc(sbase + kGemmA + sa * kStageA);
 #pragma unroll
         for (int a = 0; a < kAcc; ++a) {
-          const uint64_t bd = umma_desc(sbase + kGemmB + s * kStageB + a * (kBN * kBK * 2));
+          const int hb = it * kAcc + a, sb = hb % kStagesB;
+          if (!gemm_wait<true>(bar_fullB + 8 * sb, (uint32_t)(hb / kStagesB) & 1u, abort_flag)) { go = false; break; }
+          tc_fence_after();
+          const uint64_t bd = umma_desc(sbase + kGemmB + sb * kStageB);
 #pragma unroll
           for (int kk = 0; kk < kBK / 16; ++kk)
             umma_bf16(tmem_d + (uint32_t)(a * kBN), ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(bar_emptyB + 8 * sb);      // the box is free once these MMAs have read it
         }
-        umma_commit(bar_empty + 8 * s);          // the stage is free once these MMAs have read it
+        if (go) umma_commit(bar_emptyA + 8 * sa);
       }
       umma_commit(bar_accum);                    // all MMAs issued so far have completed
     }
@@ -360,7 +412,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
     const int gi = (warp - 2) >> 2;               // decode group: which of the lane's four rows this warp takes
     DecodeArgs da;
     da.packed = packed; da.hdr = hdr; da.smem = smem; da.abort_flag = abort_flag;
-    da.bar_full = bar_full; da.bar_empty = bar_empty;
+    da.bar_full = bar_fullA; da.bar_empty = bar_emptyA;
     da.mt = mt; da.b0 = b0; da.b1 = b1; da.nblk = nblk; da.ntile = ntile; da.q = warp & 3; da.lane = lane;
     da.rw0 = rw0; da.rw1 = rw1; da.nres = nres;
     decode_row<N>(da, gi);
