@@ -167,6 +167,18 @@ int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size
              stb_dtype ydt, size_t ldy, void *ws, size_t ws_bytes, int *dev_status,
              void *stream);
 
+/* The same product for fp16 activations: X fp16 [T][ldx], Y fp32 or fp16 (ydt = STB_F32 / STB_F16); W^ is decoded to
+ * fp16 with its scales as stored (no rounding: a kept weight is s a_region exactly, a salient one s1 a_sal1 + s2 a_sal2 as
+ * two terms of the sum), so the result is the one stb_gemv defines.  Meant for decode batches beyond what the GEMV
+ * kernels do well (Appendix C.2 between its two stages: tens of tokens): for T <= 64 the CTA tile is 128 rows x 64 tokens
+ * (one accumulator of 64 TMEM columns), K is split into as many parts as fill the 148 SMs best and the kernel runs at the
+ * speed of its decode warps; for T > 64 it is stb_gemm's tiling.  The workspace (stb_gemm_f16_workspace bytes, 256-byte
+ * aligned; the gathered residual activations and the fp32 partial tiles) is required.  Errors as stb_gemm. */
+int stb_gemm_f16_workspace(int n, int m, int N, int T, size_t *bytes);
+int stb_gemm_f16(const void *packed, int n, int m, int N, const void *X, int T, size_t ldx, void *Y,
+                 stb_dtype ydt, size_t ldy, void *ws, size_t ws_bytes, int *dev_status,
+                 void *stream);
+
 /* stb_gemm without a workspace argument (the paper has no counterpart: this entry point exists
  * for the integration, not for the method).  Some hosts of this library may not allocate device
  * memory while they run: a serving process that gave its whole memory budget to one arena at

@@ -22,7 +22,7 @@ STB_F16, STB_BF16, STB_F32 = 0, 1, 2
 STB_IN_PLAIN, STB_IN_SILU_MUL = 0, 1
 
 EXPORTS = ["stb_pack_size", "stb_pack", "stb_packed_info", "stb_dequant", "stb_gemv", "stb_gemv_wait_selftest",
-           "stb_gemm_workspace", "stb_gemm_workspace_min", "stb_gemm", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
+           "stb_gemm_workspace", "stb_gemm_workspace_min", "stb_gemm", "stb_gemm_f16_workspace", "stb_gemm_f16", "stb_gemm_noalloc", "stb_layer_stack", "stb_layer_stack_host",
            "stb_layer_stack_resident_workspace", "stb_layer_stack_resident", "stb_layer_stack_resident_host",
            "stb_layer_stack_resident_wait_selftest", "stb_layer_stack_checksum", "stb_quantize_workspace", "stb_quantize", "stb_weight_sumsq",
            "stb_allocate_nm", "stb_status_str"]
@@ -66,6 +66,8 @@ def _load():
     lib.stb_gemm_workspace.argtypes = [i, i, i, i, p(z)]
     lib.stb_gemm_workspace_min.argtypes = [i, i, i, i, p(z)]
     lib.stb_gemm.argtypes = [v, i, i, i, v, i, z, v, i, z, v, z, v, v]
+    lib.stb_gemm_f16_workspace.argtypes = [i, i, i, i, p(z)]
+    lib.stb_gemm_f16.argtypes = [v, i, i, i, v, i, z, v, i, z, v, z, v, v]
     lib.stb_gemm_noalloc.argtypes = [v, i, i, i, v, i, z, v, i, z, v, v]
     lib.stb_layer_stack.argtypes = [p(_Step), i, v, v]
     lib.stb_layer_stack_host.argtypes = [p(_Step), i, v, z, v, z, v, v]
@@ -225,6 +227,29 @@ def gemm(layer: PackedLayer, X, out=None, out_dtype=None, ws=None, stream=None):
     _check(_lib.stb_gemm(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(X), T, X.stride(0), _ptr(out),
                          ydt, out.stride(0), _ptr(ws), (ws.numel() * ws.element_size()) if ws is not None else 0,
                          _ptr(layer.dev_status), _stream(stream)), "stb_gemm")
+    return out
+
+
+def gemm_f16_workspace(n, m, N, T) -> int:
+    out = C.c_size_t()
+    _check(_lib.stb_gemm_f16_workspace(n, m, N, T, C.byref(out)), "stb_gemm_f16_workspace")
+    return out.value
+
+
+def gemm_f16(layer: PackedLayer, X, out=None, out_dtype=None, ws=None, stream=None):
+    """stb_gemm_f16: X fp16 [T][m] -> Y [T][n] fp32 (or fp16); exact fp16 scales, the small token tile for T <= 64."""
+    import torch
+    assert X.dtype == torch.float16 and X.is_cuda and X.dim() == 2 and X.stride(1) == 1
+    T = X.shape[0]
+    if out is None:
+        out = torch.empty((T, layer.n), dtype=out_dtype or torch.float32, device=X.device)
+    ydt = {torch.float32: STB_F32, torch.float16: STB_F16}[out.dtype]
+    need = gemm_f16_workspace(layer.n, layer.m, layer.N, T)
+    if ws is None or ws.numel() * ws.element_size() < need:
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=X.device)
+    _check(_lib.stb_gemm_f16(_ptr(layer.buf), layer.n, layer.m, layer.N, _ptr(X), T, X.stride(0), _ptr(out),
+                             ydt, out.stride(0), _ptr(ws), ws.numel() * ws.element_size(),
+                             _ptr(layer.dev_status), _stream(stream)), "stb_gemm_f16")
     return out
 
 

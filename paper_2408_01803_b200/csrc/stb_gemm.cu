@@ -43,24 +43,29 @@
 namespace stb {
 
 constexpr int kBM = 128;          // rows of W^ per CTA (UMMA M)
-constexpr int kBN = 256;          // tokens per accumulator (UMMA N)
-constexpr int kAcc = 2;                         // accumulators per CTA: a decoded A stage is used kAcc times
-constexpr int kTok = kBN * kAcc;                // tokens per CTA
+// Token side of the CTA tile: kAcc accumulators of kBN tokens (UMMA N).  Prefill: 2 x 256 (all 512 TMEM columns; a
+// decoded A stage is used twice).  Up to 64 tokens (a decode batch): 1 x 64, the tensor core then takes an eighth
+// of the time per stage and the kernel runs at the speed of the decode warps.
+template <int kAcc_, int kBN_>
+struct TokCfg {
+  static constexpr int kAcc = kAcc_, kBN = kBN_, kTok = kAcc_ * kBN_;
+  static constexpr uint32_t kStageB = (uint32_t)kBN_ * 64u * 2u;                 // one X box: kBN tokens x 64 of K
+  static constexpr int kStagesB = kBN_ >= 256 ? 5 : 8;                            // ring of X boxes
+};
 constexpr int kBK = 64;           // K per stage: one 128-byte swizzle row of bf16
 constexpr int kStagesA = 4;        // ring of decoded A stages (16 KB each)
-constexpr int kStagesB = 5;        // ring of X boxes (256 tokens x 64 of K = 32 KB each; a stage of K takes kAcc of them): what
-                                   // is in flight from L2 is what hides its latency, so the ring is deep and its slots small
+// (the ring of X boxes, TokCfg::kStagesB: 256 tokens x 64 of K = 32 KB each in prefill; a stage of K takes kAcc of them:
+// what is in flight from L2 is what hides its latency, so the ring is deep and its slots small)
 constexpr int kGroups = 4;                              // decode warps per 32-row quarter: one per row of a lane
 constexpr int kGemmThreads = 64 + 128 * kGroups;
 constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
-constexpr uint32_t kStageB = kBN * kBK * 2;      // 32 KB: one box
 constexpr uint32_t kGemmTab = 0;                                   // position table (576 B)
 constexpr uint32_t kGemmBars = 1024;                               // fullA, emptyA, fullB, emptyB, accum, tmem slot, abort
 constexpr uint32_t kGemmA = 2048;                                  // 1024-byte aligned stages
 constexpr uint32_t kGemmB = kGemmA + kStagesA * kStageA;
-constexpr uint32_t kGemmSmem = kGemmB + kStagesB * kStageB;        // 231424 B
-static_assert(kGemmSmem <= 232448, "one CTA's shared memory");
-static_assert(8 * (2 * kStagesA + 2 * kStagesB + 1) + 16 <= 1024, "barrier area");
+template <class Cfg> constexpr uint32_t gemm_smem_bytes() { return kGemmB + (uint32_t)Cfg::kStagesB * Cfg::kStageB; }   // prefill: 231424 B
+static_assert(gemm_smem_bytes<TokCfg<2, 256>>() <= 232448 && gemm_smem_bytes<TokCfg<1, 64>>() <= 232448, "one CTA's shared memory");
+static_assert(8 * (2 * kStagesA + 2 * 8 + 1) + 16 <= 1024, "barrier area");
 constexpr long long kGemmWaitLimit = 2000000000ll;
 
 // ---- tcgen05 / TMA wrappers ---------------------------------------------------------------
@@ -108,8 +113,11 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                  // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+// Instruction descriptor: D = f32, A and B both bf16 (format 1) or both fp16 (format 0), both K-major, N = kBN, M = 128.
+template <int kBN, bool kF16>
+struct GemmIdesc {
+  static constexpr uint32_t value = (1u << 4) | ((kF16 ? 0u : 1u) << 7) | ((kF16 ? 0u : 1u) << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+};
 
 // Bounded mbarrier wait with a CTA-wide abort flag (a volatile int in shared memory).  The two
 // single-lane roles back off between polls so that their spinning does not take issue slots from
@@ -142,7 +150,8 @@ struct DecodeArgs {
 // Decode role of one warp: row j (of the four rows g + 8 j each lane owns) of packed row tile 4 mt + q, for
 // every block of the CTA's K range, written into the A stages.  j is a run-time value: the four warps of a
 // row tile run the same code.
-template <int N>
+// kF16: the stages hold fp16 (the scales as stored); otherwise bf16 (the scales rounded to nearest even).
+template <int N, bool kF16>
 __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
   const uint8_t* packed = da.packed;
   const Header* hdr = da.hdr;
@@ -176,7 +185,7 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const uint32_t h16 = ((cur.A >> (8 * c)) & 0xFFu) | (((cur.B >> (8 * c)) & 0xFFu) << 8);
-        const uint32_t v = bf16_bits(h16);
+        const uint32_t v = kF16 ? h16 : bf16_bits(h16);
         A16 |= (v & 0xFFu) << (8 * c);
         B16 |= (v >> 8) << (8 * c);
       }
@@ -243,7 +252,7 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
 #pragma unroll
     for (int idx = 0; idx < 4; ++idx)
       if ((valid >> idx) & 1u) {
-        const uint32_t v = bf16_bits(a2[idx]);
+        const uint32_t v = kF16 ? a2[idx] : bf16_bits(a2[idx]);
         const uint32_t L2 = prmt(v, 0u, 0x4040u);                 // (lo, 0, lo, 0)
         const uint32_t H2 = prmt(v, v ^ 0x8000u, 0x2521u);        // (hi, 0, hi ^ 0x80, 0)
         const uint32_t sel = resid_selector(word[idx], j);
@@ -314,11 +323,13 @@ __global__ void gemm_gather_kernel(const uint8_t* __restrict__ packed, int n, in
 }
 
 // ------------------------------------------------------------------------------------------
-template <int N>
+template <int N, class Cfg, bool kF16>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap xsmap, const uint8_t* __restrict__ packed, int n, int m, int T,
-            void* __restrict__ Y, int y_bf16, size_t ldy, float* __restrict__ ws, int full_tiles, int ksplit, int bps,
+            void* __restrict__ Y, int y_16, size_t ldy, float* __restrict__ ws, int full_tiles, int ksplit, int bps,
             int ttiles, uint32_t box_bytes, int* dev_status) {
+  constexpr int kAcc = Cfg::kAcc, kBN = Cfg::kBN, kTok = Cfg::kTok, kStagesB = Cfg::kStagesB;
+  constexpr uint32_t kStageB = Cfg::kStageB, kIdesc = GemmIdesc<kBN, kF16>::value;
   extern __shared__ __align__(1024) uint8_t smem[];
   const Header* hdr = reinterpret_cast<const Header*>(packed);
   if (!header_matches(hdr, n, m, N)) {
@@ -415,7 +426,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
     da.bar_full = bar_fullA; da.bar_empty = bar_emptyA;
     da.mt = mt; da.b0 = b0; da.b1 = b1; da.nblk = nblk; da.ntile = ntile; da.q = warp & 3; da.lane = lane;
     da.rw0 = rw0; da.rw1 = rw1; da.nres = nres;
-    decode_row<N>(da, gi);
+    decode_row<N, kF16>(da, gi);
 
     // ---------------- epilogue: TMEM -> registers -> Y ----------------
     const int q = warp & 3;                        // TMEM lane quarter of this warp
@@ -434,7 +445,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
             if (tok < T) {
               const float v = __uint_as_float(r[i]);
               if (wsz) wsz[(size_t)(32 * cc + i) * kBM + 32 * q + lane] = v;
-              else if (y_bf16) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(v);
+              else if (y_16 && kF16) static_cast<__half*>(Y)[(size_t)tok * ldy + row] = __float2half_rn(v);
+              else if (y_16) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(v);
               else static_cast<float*>(Y)[(size_t)tok * ldy + row] = v;
             }
           }
@@ -454,30 +466,42 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
 }
 
 // Split-K reduction of the tiles that were computed in parts: partial tile z of split tile u is
-// ws[(u ksplit + z)][token 0..kTok-1][row 0..kBM-1]; summed in z order.
-__global__ void gemm_reduce_kernel(const float* __restrict__ ws, int first_tile, int split_tiles, int ksplit, int ttiles,
-                                   int n, int T, void* __restrict__ Y, int y_bf16, size_t ldy) {
-  const size_t per = (size_t)kBM * kTok, total = (size_t)split_tiles * per;
+// ws[(u ksplit + z)][token 0..ktok-1][row 0..kBM-1]; summed in z order.  y_16: 1 = bf16, 2 = fp16 output.
+__global__ void gemm_reduce_kernel(const float* __restrict__ ws, int first_tile, int split_tiles, int ksplit, int ttiles, int ktok,
+                                   int n, int T, void* __restrict__ Y, int y_16, size_t ldy) {
+  const size_t per = (size_t)kBM * ktok, total = (size_t)split_tiles * per;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t u = i / per, r = i % per;
     const int tile = first_tile + (int)u, tt = tile % ttiles, mt = tile / ttiles;
-    const int tok = tt * kTok + (int)(r / kBM), row = mt * kBM + (int)(r % kBM);
+    const int tok = tt * ktok + (int)(r / kBM), row = mt * kBM + (int)(r % kBM);
     if (tok >= T || row >= n) continue;
     float acc = 0.0f;
     for (int z = 0; z < ksplit; ++z) acc += ws[(u * ksplit + z) * per + r];
-    if (y_bf16) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(acc);
+    if (y_16 == 2) static_cast<__half*>(Y)[(size_t)tok * ldy + row] = __float2half_rn(acc);
+    else if (y_16 == 1) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(acc);
     else static_cast<float*>(Y)[(size_t)tok * ldy + row] = acc;
   }
 }
 
 // K split: only when the output tiles alone cannot fill the 148 SMs
-static int gemm_ksplit(int n, int m, int T) {
-  const int tiles = ((n + kBM - 1) / kBM) * ((T + kTok - 1) / kTok), nblk = m / kBlock;
+static int gemm_ksplit(int n, int m, int T, int ktok) {
+  const int tiles = ((n + kBM - 1) / kBM) * ((T + ktok - 1) / ktok), nblk = m / kBlock;
   int ks = 1;
-  if (tiles < 100) ks = 148 / tiles;
-  if (ks > 16) ks = 16;
-  while (ks > 1 && nblk / ks < 4) --ks;
-  if (ks < 1) ks = 1;
+  if (ktok < 512) {
+    // decode batch: a CTA's time is the decode of its blocks, so any number of parts with at least four blocks each
+    // will do; take the one that fills the waves of 148 CTAs best (the fewest parts among equals)
+    double best = 0.0;
+    for (int k = 1; k <= 16 && nblk / k >= 4; ++k) {
+      const long long ctas = (long long)tiles * k, waves = (ctas + 147) / 148;
+      const double fill = (double)ctas / (double)(waves * 148);
+      if (fill > best + 1e-9) { best = fill; ks = k; }
+    }
+  } else {
+    if (tiles < 100) ks = 148 / tiles;
+    if (ks > 16) ks = 16;
+    while (ks > 1 && nblk / ks < 4) --ks;
+    if (ks < 1) ks = 1;
+  }
   const int bps = (nblk + ks - 1) / ks;          // blocks per split; every split gets at least one
   return (nblk + bps - 1) / bps;
 }
@@ -491,13 +515,13 @@ struct GemmPlan {
   int ttiles, tiles, full_tiles, split_tiles, ksplit, bps;
   size_t mandatory_bytes, preferred_bytes;
 };
-static GemmPlan gemm_plan(int n, int m, int T, size_t ws_bytes, bool have_ws) {
+static GemmPlan gemm_plan(int n, int m, int T, int ktok, size_t ws_bytes, bool have_ws) {
   GemmPlan p;
   const int nblk = m / kBlock;
-  p.ttiles = (T + kTok - 1) / kTok;
+  p.ttiles = (T + ktok - 1) / ktok;
   p.tiles = ((n + kBM - 1) / kBM) * p.ttiles;
-  const size_t per = (size_t)kBM * kTok * sizeof(float);
-  const int ks = gemm_ksplit(n, m, T);
+  const size_t per = (size_t)kBM * ktok * sizeof(float);
+  const int ks = gemm_ksplit(n, m, T, ktok);
   p.full_tiles = p.tiles; p.split_tiles = 0; p.ksplit = 1; p.bps = nblk;
   p.mandatory_bytes = 0; p.preferred_bytes = 0;
   if (ks > 1) {
@@ -540,17 +564,21 @@ static EncodeTiledFn encode_tiled_fn() {
 // slots a layer can have (32 per block), so that the size depends on the shape alone.
 static size_t gemm_xs_bytes(int m, int T) { return (((size_t)T * (size_t)(m / 4) * 2u) + 255u) & ~(size_t)255u; }
 
-template <int N>
-static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T, size_t ldx, void* Y, int y_bf16,
+// y_16: 0 = fp32 output, 1 = the 16-bit type of the activations (bf16, or fp16 with kF16)
+template <int N, class Cfg, bool kF16>
+static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T, size_t ldx, void* Y, int y_16,
                        size_t ldy, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t s) {
+  constexpr int kBN = Cfg::kBN, kTok = Cfg::kTok;
+  constexpr uint32_t kSmem = gemm_smem_bytes<Cfg>();
   const size_t xs_bytes = gemm_xs_bytes(m, T);
   if (ws && (reinterpret_cast<uintptr_t>(ws) & 255u)) return STB_ERR_ARG;
   if (!ws || ws_bytes < xs_bytes) return STB_ERR_SIZE;
   float* ws_split = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + xs_bytes);
-  const GemmPlan plan = gemm_plan(n, m, T, ws_bytes - xs_bytes, true);
+  const GemmPlan plan = gemm_plan(n, m, T, kTok, ws_bytes - xs_bytes, true);
   if (plan.mandatory_bytes > ws_bytes - xs_bytes) return STB_ERR_SIZE;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return STB_ERR_CUDA;
+  const CUtensorMapDataType dt = kF16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
   const cuuint32_t box_rows = (cuuint32_t)(T < kBN ? T : kBN);
   const cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
   const cuuint32_t estr[2] = {1, 1};
@@ -558,7 +586,7 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
   {
     const cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)T};
     const cuuint64_t strides[1] = {(cuuint64_t)ldx * 2};
-    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+    if (enc(&map, dt, 2, const_cast<void*>(X), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return STB_ERR_ARG;
@@ -567,7 +595,7 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
   {
     const cuuint64_t dims[2] = {(cuuint64_t)ldxs, (cuuint64_t)T};
     const cuuint64_t strides[1] = {(cuuint64_t)ldxs * 2};
-    if (enc(&xsmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ws, dims, strides, box, estr,
+    if (enc(&xsmap, dt, 2, ws, dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return STB_ERR_ARG;
@@ -577,55 +605,89 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return STB_ERR_CUDA;
   if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-    if (cudaFuncSetAttribute(gemm_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem) != cudaSuccess) return STB_ERR_CUDA;
+    if (cudaFuncSetAttribute(gemm_kernel<N, Cfg, kF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem) != cudaSuccess) return STB_ERR_CUDA;
     if (dev >= 0 && dev < 64) attr_done[dev] = true;
   }
+  // the gather moves 16-bit values: the same kernel serves bf16 and fp16
   gemm_gather_kernel<<<148 * 4, 256, 0, s>>>(packed, n, m, N, static_cast<const __nv_bfloat16*>(X), T, ldx,
                                              static_cast<__nv_bfloat16*>(ws), ldxs);
   if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   const unsigned grid = (unsigned)(plan.full_tiles + plan.split_tiles * plan.ksplit);
-  gemm_kernel<N><<<grid, kGemmThreads, kGemmSmem, s>>>(map, xsmap, packed, n, m, T, Y, y_bf16, ldy, ws_split, plan.full_tiles,
-                                              plan.ksplit, plan.bps, plan.ttiles, box_rows * kBK * 2, dev_status);
+  gemm_kernel<N, Cfg, kF16><<<grid, kGemmThreads, kSmem, s>>>(map, xsmap, packed, n, m, T, Y, y_16, ldy, ws_split, plan.full_tiles,
+                                                              plan.ksplit, plan.bps, plan.ttiles, box_rows * kBK * 2, dev_status);
   if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   if (plan.split_tiles > 0) {
     gemm_reduce_kernel<<<148 * 4, 256, 0, s>>>(ws_split, plan.full_tiles, plan.split_tiles, plan.ksplit,
-                                               plan.ttiles, n, T, Y, y_bf16, ldy);
+                                               plan.ttiles, kTok, n, T, Y, y_16 ? (kF16 ? 2 : 1) : 0, ldy);
     if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
   }
   return STB_OK;
 }
 
+using PrefillCfg = TokCfg<2, 256>;
+using BatchCfg = TokCfg<1, 64>;
+// fp16 activations: up to 64 tokens take the small token tile
+static int ktok_f16(int T) { return T <= BatchCfg::kTok ? BatchCfg::kTok : PrefillCfg::kTok; }
+
+template <bool kF16>
+static int launch_gemm_n(int N, const uint8_t* packed, int n, int m, const void* X, int T, size_t ldx, void* Y, int y_16,
+                         size_t ldy, void* ws, size_t ws_bytes, int* dev_status, cudaStream_t s) {
+  if (kF16 && T <= BatchCfg::kTok) {
+    switch (N) {
+      case 4: return launch_gemm<4, BatchCfg, kF16>(packed, n, m, X, T, ldx, Y, y_16, ldy, ws, ws_bytes, dev_status, s);
+      case 5: return launch_gemm<5, BatchCfg, kF16>(packed, n, m, X, T, ldx, Y, y_16, ldy, ws, ws_bytes, dev_status, s);
+      default: return launch_gemm<6, BatchCfg, kF16>(packed, n, m, X, T, ldx, Y, y_16, ldy, ws, ws_bytes, dev_status, s);
+    }
+  }
+  switch (N) {
+    case 4: return launch_gemm<4, PrefillCfg, kF16>(packed, n, m, X, T, ldx, Y, y_16, ldy, ws, ws_bytes, dev_status, s);
+    case 5: return launch_gemm<5, PrefillCfg, kF16>(packed, n, m, X, T, ldx, Y, y_16, ldy, ws, ws_bytes, dev_status, s);
+    default: return launch_gemm<6, PrefillCfg, kF16>(packed, n, m, X, T, ldx, Y, y_16, ldy, ws, ws_bytes, dev_status, s);
+  }
+}
+
 }  // namespace stb
 
-static int gemm_workspace_impl(int n, int m, int N, int T, size_t* bytes, bool minimum) {
+static int gemm_workspace_impl(int n, int m, int N, int T, int ktok, size_t* bytes, bool minimum) {
   if (!bytes) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0 || T < 1) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
-  const stb::GemmPlan plan = stb::gemm_plan(n, m, T, 0, false);
+  const stb::GemmPlan plan = stb::gemm_plan(n, m, T, ktok, 0, false);
   *bytes = stb::gemm_xs_bytes(m, T) + (minimum ? plan.mandatory_bytes : plan.preferred_bytes);
   return STB_OK;
 }
 
-extern "C" int stb_gemm_workspace(int n, int m, int N, int T, size_t* bytes) { return gemm_workspace_impl(n, m, N, T, bytes, false); }
-extern "C" int stb_gemm_workspace_min(int n, int m, int N, int T, size_t* bytes) { return gemm_workspace_impl(n, m, N, T, bytes, true); }
+extern "C" int stb_gemm_workspace(int n, int m, int N, int T, size_t* bytes) { return gemm_workspace_impl(n, m, N, T, stb::PrefillCfg::kTok, bytes, false); }
+extern "C" int stb_gemm_workspace_min(int n, int m, int N, int T, size_t* bytes) { return gemm_workspace_impl(n, m, N, T, stb::PrefillCfg::kTok, bytes, true); }
+extern "C" int stb_gemm_f16_workspace(int n, int m, int N, int T, size_t* bytes) { return gemm_workspace_impl(n, m, N, T, stb::ktok_f16(T), bytes, false); }
 
-extern "C" int stb_gemm(const void* packed, int n, int m, int N, const void* X, int T, size_t ldx,
-                        void* Y, stb_dtype ydt, size_t ldy, void* ws, size_t ws_bytes,
-                        int* dev_status, void* stream) {
+static int gemm_check_args(const void* packed, int n, int m, int N, const void* X, int T, size_t ldx, void* Y, size_t ldy) {
   if (!packed || !X || !Y) return STB_ERR_ARG;
   if (n < 1 || m < stb::kBlock || m % stb::kBlock != 0 || T < 1) return STB_ERR_SHAPE;
   if (N < 1 || N > 8) return STB_ERR_NM;
   if (N < 4 || N > 6) return STB_ERR_UNSUPPORTED;          // the tensor-core decode covers N = 4, 5, 6
-  if (ydt != STB_F32 && ydt != STB_BF16) return STB_ERR_UNSUPPORTED;
   if (ldx < (size_t)m || ldy < (size_t)n || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u)) return STB_ERR_ARG;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const uint8_t* p = static_cast<const uint8_t*>(packed);
-  const int y_bf16 = ydt == STB_BF16;
-  switch (N) {
-    case 4: return stb::launch_gemm<4>(p, n, m, X, T, ldx, Y, y_bf16, ldy, ws, ws_bytes, dev_status, s);
-    case 5: return stb::launch_gemm<5>(p, n, m, X, T, ldx, Y, y_bf16, ldy, ws, ws_bytes, dev_status, s);
-    default: return stb::launch_gemm<6>(p, n, m, X, T, ldx, Y, y_bf16, ldy, ws, ws_bytes, dev_status, s);
-  }
+  return STB_OK;
+}
+
+extern "C" int stb_gemm(const void* packed, int n, int m, int N, const void* X, int T, size_t ldx,
+                        void* Y, stb_dtype ydt, size_t ldy, void* ws, size_t ws_bytes,
+                        int* dev_status, void* stream) {
+  const int rc = gemm_check_args(packed, n, m, N, X, T, ldx, Y, ldy);
+  if (rc != STB_OK) return rc;
+  if (ydt != STB_F32 && ydt != STB_BF16) return STB_ERR_UNSUPPORTED;
+  return stb::launch_gemm_n<false>(N, static_cast<const uint8_t*>(packed), n, m, X, T, ldx, Y, ydt == STB_BF16, ldy, ws, ws_bytes,
+                                   dev_status, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int stb_gemm_f16(const void* packed, int n, int m, int N, const void* X, int T, size_t ldx,
+                            void* Y, stb_dtype ydt, size_t ldy, void* ws, size_t ws_bytes,
+                            int* dev_status, void* stream) {
+  const int rc = gemm_check_args(packed, n, m, N, X, T, ldx, Y, ldy);
+  if (rc != STB_OK) return rc;
+  if (ydt != STB_F32 && ydt != STB_F16) return STB_ERR_UNSUPPORTED;
+  return stb::launch_gemm_n<true>(N, static_cast<const uint8_t*>(packed), n, m, X, T, ldx, Y, ydt == STB_F16, ldy, ws, ws_bytes,
+                                  dev_status, static_cast<cudaStream_t>(stream));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -646,7 +708,7 @@ extern "C" int stb_gemm_noalloc(const void* packed, int n, int m, int N, const v
   if (ydt != STB_F32 && ydt != STB_BF16) return STB_ERR_UNSUPPORTED;
   if (ldx < (size_t)m || ldy < (size_t)n || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15u)) return STB_ERR_ARG;
   // this shape needs the caller-workspace entry point if the scratch it cannot do without does not fit
-  if (stb::gemm_xs_bytes(m, T) + stb::gemm_plan(n, m, T, 0, false).mandatory_bytes > stb::kNoAllocScratchBytes) return STB_ERR_SIZE;
+  if (stb::gemm_xs_bytes(m, T) + stb::gemm_plan(n, m, T, stb::PrefillCfg::kTok, 0, false).mandatory_bytes > stb::kNoAllocScratchBytes) return STB_ERR_SIZE;
   // The array's name is only a host-side handle: ask the runtime for its address on the current
   // device, once per device, and give the kernels that address.
   static float* scratch_of_device[64] = {nullptr};
@@ -657,13 +719,6 @@ extern "C" int stb_gemm_noalloc(const void* packed, int n, int m, int N, const v
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), stb::g_noalloc_scratch) != cudaSuccess || !p) return STB_ERR_CUDA;
     scratch_of_device[dev] = p;
   }
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const uint8_t* pk = static_cast<const uint8_t*>(packed);
-  const int y_bf16 = ydt == STB_BF16;
-  float* ws = scratch_of_device[dev];
-  switch (N) {
-    case 4: return stb::launch_gemm<4>(pk, n, m, X, T, ldx, Y, y_bf16, ldy, ws, stb::kNoAllocScratchBytes, dev_status, s);
-    case 5: return stb::launch_gemm<5>(pk, n, m, X, T, ldx, Y, y_bf16, ldy, ws, stb::kNoAllocScratchBytes, dev_status, s);
-    default: return stb::launch_gemm<6>(pk, n, m, X, T, ldx, Y, y_bf16, ldy, ws, stb::kNoAllocScratchBytes, dev_status, s);
-  }
+  return stb::launch_gemm_n<false>(N, static_cast<const uint8_t*>(packed), n, m, X, T, ldx, Y, ydt == STB_BF16, ldy,
+                                   scratch_of_device[dev], stb::kNoAllocScratchBytes, dev_status, static_cast<cudaStream_t>(stream));
 }

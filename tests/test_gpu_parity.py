@@ -328,6 +328,74 @@ def test_gemm_many_salient_columns(stb, N, max_salient):
     _check_gemm(stb, layer, L, 70, 9)
 
 
+def _check_gemm_f16(stb, layer, L, T, seed, out_dtype=None, rows=None):
+    """stb_gemm_f16 against the float64 dequantise-then-matmul on fp16 activations."""
+    import torch
+    x = si.activations(T, L.m, seed)                                # fp16
+    xd = torch.from_numpy(x).cuda()
+    y = stb.gemm_f16(layer, xd, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    assert int(layer.dev_status.item()) == 0
+    if rows is None:
+        y_ref = oracle.matmul(oracle.decode(L), x.astype(np.float64))
+        got = y.double().cpu().numpy()
+    else:
+        y_ref = oracle.layer_rows(L, rows, x.astype(np.float64))
+        got = y.double().cpu().numpy()[:, rows]
+    scale = np.abs(y_ref).max()
+    err = np.abs(got - y_ref).max()
+    assert err <= TOL * scale, (err, TOL * scale)
+    if out_dtype is not None and out_dtype != torch.float32:
+        y32 = stb.gemm_f16(layer, xd)
+        torch.cuda.synchronize()
+        assert torch.equal(y32.to(out_dtype), y)                     # the fp16 output is the fp32 one rounded, bit for bit
+    return y
+
+
+@pytest.mark.parametrize("N", [4, 5, 6])
+@pytest.mark.parametrize("n,m,T", [(40, 256, 1), (100, 384, 37), (300, 1024, 64), (257, 2048, 33), (200, 512, 65), (130, 640, 200)])
+def test_gemm_f16_quantized_layers(stb, N, n, m, T):
+    """The fp16 product on quantizer output: the 64-token tile (T <= 64: one to several row tiles, K split in parts,
+    ragged rows and tokens) and the prefill tile beyond; fp32 and fp16 outputs."""
+    import torch
+    L = _quantized(n, m, N, 2100 + 10 * N + n)
+    layer = stb.pack_numpy(_fields(L))
+    y = _check_gemm_f16(stb, layer, L, T, 60 + T)
+    _check_gemm_f16(stb, layer, L, T, 61 + T, out_dtype=torch.float16)
+    if T <= 64:
+        # the same operation as the decode GEMV: both within the tolerance of the oracle, hence of each other
+        xd = torch.from_numpy(si.activations(T, m, 60 + T)).cuda()
+        yv = stb.gemv(layer, xd)
+        torch.cuda.synchronize()
+        assert (y - yv).abs().max().item() <= 2 * TOL * yv.abs().max().item()
+
+
+@pytest.mark.parametrize("max_salient", [0, 30])
+def test_gemm_f16_salient_extremes(stb, max_salient):
+    d = si.logical_layer(200, 1024, 6, 520 + max_salient, max_salient=max_salient)
+    L = oracle.Logical(**d)
+    layer = stb.pack_numpy(d)
+    _check_gemm_f16(stb, layer, L, 48, 19)
+
+
+@pytest.mark.parametrize("name", ["gate", "down"])
+def test_gemm_f16_full_size_decode_batch(stb, name):
+    """A decode batch of 64 on the LLaMA-2-7B MLP layers at 6:8 from the oracle's quantizer, sampled rows."""
+    n, m, N, seed = si.workload_layer(2, name)
+    d = wl.quantized_layer(n, m, N, seed)
+    L = wl.as_logical(d)
+    layer = stb.pack_numpy(d)
+    g = np.random.default_rng(n + 3 * m)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, n - 129, n - 1], g.choice(n, 64, replace=False)])).astype(np.int32)
+    _check_gemm_f16(stb, layer, L, 64, si.seed_for(2, 12), rows=rows)
+    with pytest.raises(stb.StbError) as e:                      # no workspace: refused on the host
+        import torch
+        x = torch.zeros(64, m, dtype=torch.float16, device="cuda")
+        stb._check(stb._lib.stb_gemm_f16(stb._ptr(layer.buf), n, m, N, stb._ptr(x), 64, m, stb._ptr(torch.empty(64, n, device="cuda")),
+                                         stb.STB_F32, n, None, 0, stb._ptr(layer.dev_status), stb._stream()), "stb_gemm_f16")
+    assert e.value.status == stb.STB_ERR_SIZE
+
+
 def test_gemm_split_k_uses_the_workspace(stb):
     """Few output tiles and a long K: the launch splits K, partial sums go through the caller's workspace."""
     import torch
