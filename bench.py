@@ -442,7 +442,8 @@ def gemm_table(stb, torch, pk, real_ffn, only=None):
     return out
 
 
-CALL = {True: "stb_layer_stack_resident (one resident kernel)", False: "stb_layer_stack (per-layer launches)"}
+CALL = {True: "stb_layer_stack_resident (one resident kernel)", False: "stb_layer_stack (per-layer launches)",
+        "tc": "stb_gemm_f16 per linear (tcgen05, 64-token tile; gather + GEMM + sum of K parts = 3 launches each)"}
 
 
 def decoder(h, f):
@@ -478,14 +479,24 @@ def run_stack(stb, torch, layers, h, f, batch, nl, min_calls, resident):
         cur = hb[4]      # (the data flow of attention / activation functions is not part of this path)
     arr = stb.make_steps(steps)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    if resident:
+    if resident == "tc":
+        need = max(stb.gemm_f16_workspace(lay.n, lay.m, lay.N, batch) for lay, _, _ in steps)
+        wsb = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+        def fn():
+            for lay, xin, yout in steps:
+                stb.gemm_f16(lay, xin, out=yout, ws=wsb)
+        status = None
+    elif resident:
         ws = stb.resident_workspace(arr)
         fn = lambda: stb.layer_stack_resident(None, ws, dev_status=status, marshalled=arr)
     else:
         fn = lambda: stb.layer_stack(None, dev_status=status, marshalled=arr)
     g = capture(torch, [fn])
     us = time_graph(torch, g, 1, min_calls=min_calls)
-    assert int(status.item()) == 0
+    if status is None:
+        assert all(int(t.item()) == 0 for t in {id(lay.dev_status): lay.dev_status for lay, _, _ in steps}.values())
+    else:
+        assert int(status.item()) == 0
     return us
 
 
@@ -511,16 +522,16 @@ def stack_tables(stb, torch, pk):
     names_N = [(nm, Nl[l]) for l in range(32) for nm, _, _ in decoder(4096, 11008)]
     l7 = build_stack(stb, 5, names_N)
     b7 = sum(b for _, _, b in l7)
-    for batch, resident in ((1, True), (1, False), (8, True), (8, False), (64, False)):
+    for batch, resident in ((1, True), (1, False), (8, True), (8, False), (64, False), (64, "tc")):
         # resident: 128 groups of same-input linears = two launches of 64 groups; per-layer launches: q/k/v as one grid,
         # o, gate/up as one grid, down = 128 launches
-        launches = 2 if resident else 32 * 4
+        launches = 2 if resident is True else 32 * 4
         us = run_stack(stb, torch, l7, 4096, 11008, batch, 32, 20, resident)
         row = {"stack": "LLaMA-2-7B, 32 decoder layers x 7 linears, N per layer from {4,5,6} (%d/%d/%d layers)" % (
                    Nl.count(4), Nl.count(5), Nl.count(6)), "call": CALL[resident], "batch": batch, "us": round(us, 1),
                "packed_GB": round(b7 / 1e9, 3), "GBps": round(b7 / us / 1e3, 1),
                "frac_of_measured_hbm": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "us_per_linear": round(us / 224, 2)}
-        if batch == 1 and resident:
+        if batch == 1 and resident is True:
             row["roofline"] = {"bound": "hbm", "achieved": round(b7 / us / 1e3, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                                "frac": round(b7 / us / 1e3 / pk["hbm_gbs"], 4), "traffic": None,
                                "kernel": "stb::stack_kernel", "bytes_per_launch": round(b7 / launches),
