@@ -272,6 +272,15 @@ __device__ __forceinline__ void tile_sp6(const LaneTile<6>& lt, const uint32_t (
     E[bb][1] = ((en[3].y * 16u + en[2].y) * 16u + en[1].y) * 16u + en[0].y;
     E[bb][2] = ((en[3].z * 16u + en[2].z) * 16u + en[1].z) * 16u + en[0].z;
   }
+  // the activations of the tile's six chunk positions, once for both halves of the rows
+  uint4 bxs[2][3];
+#pragma unroll
+  for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      bxs[sl][i] = make_uint4(0, 0, 0, 0);
+      if (xlive) bxs[sl][i] = *reinterpret_cast<const uint4*>(xi0 + sl * 12 + 4 * i);
+    }
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt) {
     uint32_t XLh[2][2], XHh[2][2];
@@ -288,8 +297,7 @@ __device__ __forceinline__ void tile_sp6(const LaneTile<6>& lt, const uint32_t (
         for (int h = 0; h < 2; ++h) fr.pairs(2 * mt + jj, 2 * h + sl, XLh[jj][h], XHh[jj][h], R[jj][h]);
 #pragma unroll
       for (int i = 0; i < 3; ++i) {
-        uint4 bx = make_uint4(0, 0, 0, 0);
-        if (xlive) bx = *reinterpret_cast<const uint4*>(xi0 + sl * 12 + 4 * i);
+        const uint4 bx = bxs[sl][i];
         if (mt == 0) mma_sp16832<0>(acc[0], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
         else mma_sp16832<1>(acc[1], R[0][0][i], R[1][0][i], R[0][1][i], R[1][1][i], bx.x, bx.y, bx.z, bx.w, E[sl][i]);
       }
