@@ -10,8 +10,9 @@
 //       divides the decode work per flop by kAcc,
 // in rings over K (kStagesA decoded A stages, kStagesB X stages: the decode warps run ahead of the tensor core).  Warp roles:
 //   warp 0      TMA producer (one lane): X slices
-//   warp 1      MMA issuer (one lane): 4 x tcgen05.mma (K = 16) per stage and accumulator,
-//               tcgen05.commit frees the stage; also allocates / frees TMEM
+//   warp 1, 18  MMA issuers (one lane each, on two schedulers): with two accumulators each takes one (4 x tcgen05.mma,
+//               K = 16, per stage); with one, each takes half of a stage's K into an accumulator of its own and the
+//               epilogue adds the two.  tcgen05.commit frees the boxes and stages; warp 1 allocates / frees TMEM
 //   warps 2..   decode: warp w works on rows 32 (w % 4) .. +31 of the tile = one packed row tile;
 //               four warps share a row tile, each taking one of the four rows a lane owns (the row
 //               index is a run-time value: one copy of the code; one warp alone per scheduler
@@ -57,7 +58,9 @@ constexpr int kStagesA = 4;        // ring of decoded A stages (16 KB each)
 // (the ring of X boxes, TokCfg::kStagesB: 256 tokens x 64 of K = 32 KB each in prefill; a stage of K takes kAcc of them:
 // what is in flight from L2 is what hides its latency, so the ring is deep and its slots small)
 constexpr int kGroups = 4;                              // decode warps per 32-row quarter: one per row of a lane
-constexpr int kGemmThreads = 64 + 128 * kGroups;
+constexpr int kIssuers = 2;                             // MMA-issuing lanes (in two warps, on two schedulers)
+constexpr int kIssuerWarpB = 2 + 4 * kGroups;           // the second one's warp: after the decode warps
+constexpr int kGemmThreads = 64 + 128 * kGroups + 32;
 constexpr uint32_t kStageA = kBM * kBK * 2;      // 16 KB
 constexpr uint32_t kGemmTab = 0;                                   // position table (576 B)
 constexpr uint32_t kGemmBars = 1024;                               // fullA, emptyA, fullB, emptyB, accum, tmem slot, abort
@@ -82,10 +85,20 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+// The descriptors come as their low words (start address / 16; the high word is the same for every operand tile of
+// this kernel) and the accumulate flag as a template argument: an issuing lane is ONE thread whose instructions go
+// out one dependent step at a time, and what it runs per stage of K (waits, descriptors, MMAs, commits) was longer
+// than the tensor core needs for the stage.
+template <bool kAccumulate>
+__device__ __forceinline__ void umma_16(uint32_t d_tmem, uint32_t adesc_lo, uint32_t bdesc_lo, uint32_t desc_hi, uint32_t idesc) {
+  if (kAccumulate)
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.eq.b32 p, 0, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(desc_hi), "r"(idesc) : "memory");
+  else
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, 0, 0;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+                 ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(desc_hi), "r"(idesc) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -364,16 +377,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kGemmBars + kBarBytes + 8);
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kStagesA; ++i) { mbar_init(bar_fullA + 8 * i, 4 * kGroups); mbar_init(bar_emptyA + 8 * i, 1); }
-    for (int i = 0; i < kStagesB; ++i) { mbar_init(bar_fullB + 8 * i, 1); mbar_init(bar_emptyB + 8 * i, 1); }
-    mbar_init(bar_accum, 1);
+    // a stage of A is read by both issuers; an X box by the issuer of its accumulator (by both when there is one box per stage)
+    for (int i = 0; i < kStagesA; ++i) { mbar_init(bar_fullA + 8 * i, 4 * kGroups); mbar_init(bar_emptyA + 8 * i, kIssuers); }
+    for (int i = 0; i < kStagesB; ++i) { mbar_init(bar_fullB + 8 * i, 1); mbar_init(bar_emptyB + 8 * i, kAcc == 1 ? kIssuers : 1); }
+    mbar_init(bar_accum, kIssuers);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
   for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x)     // 4-byte entries: fewer bank conflicts than 8-byte ones
     reinterpret_cast<uint32_t*>(smem + kGemmTab)[i] = g_pos_table.v[N][i].x | (g_pos_table.v[N][i].y << 16);
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTok);
+  constexpr uint32_t kTmemCols = kAcc == 1 ? 2 * kTok : kTok;      // one accumulator: a second one for the other half of K
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -395,28 +410,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
         while (clock64() - t0 < 200000) {}
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+  } else if (warp == 1 || warp == kIssuerWarpB) {
+    // ---------------- MMA issuers ----------------
     if (lane == 0) {
-      bool go = true;
-      for (int it = 0; it < nstage && go; ++it) {
-        const int sa = it % kStagesA;
-        if (!gemm_wait<true>(bar_fullA + 8 * sa, (uint32_t)(it / kStagesA) & 1u, abort_flag)) break;
-        const uint64_t ad = umma_desc(sbase + kGemmA + sa * kStageA);
+      const int w = warp == 1 ? 0 : 1;
+      // two accumulators: issuer w takes accumulator w (box w of every stage, all of K);
+      // one accumulator:  issuer w takes the K steps 2 w, 2 w + 1 of every stage into accumulator w
+      const uint32_t desc_hi = (uint32_t)(umma_desc(0u) >> 32);
+      const uint32_t a_lo0 = (uint32_t)umma_desc(sbase + kGemmA) + (kAcc == 1 ? 4u * (uint32_t)w : 0u);
+      const uint32_t b_lo0 = (uint32_t)umma_desc(sbase + kGemmB) + (kAcc == 1 ? 4u * (uint32_t)w : 0u);
+      const uint32_t dt = tmem_d + (uint32_t)(w * (kAcc == 1 ? kTok : kBN));
+      constexpr int kSteps = kAcc == 1 ? kBK / 32 : kBK / 16;           // MMAs per stage and issuer
+      int sa = 0, sb = kAcc == 1 ? 0 : w;                               // ring slots, advanced without divisions
+      uint32_t pa = 0, pb = 0;                                          // their phase parities
+      for (int it = 0; it < nstage; ++it) {
+        if (!gemm_wait<true>(bar_fullA + 8 * sa, pa, abort_flag)) break;
+        if (!gemm_wait<true>(bar_fullB + 8 * sb, pb, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t a_lo = a_lo0 + (uint32_t)sa * (kStageA >> 4), b_lo = b_lo0 + (uint32_t)sb * (kStageB >> 4);
+        if (it > 0) umma_16<true>(dt, a_lo, b_lo, desc_hi, kIdesc);
+        else umma_16<false>(dt, a_lo, b_lo, desc_hi, kIdesc);
 #pragma unroll
-        for (int a = 0; a < kAcc; ++a) {
-          const int hb = it * kAcc + a, sb = hb % kStagesB;
-          if (!gemm_wait<true>(bar_fullB + 8 * sb, (uint32_t)(hb / kStagesB) & 1u, abort_flag)) { go = false; break; }
-          tc_fence_after();
-          const uint64_t bd = umma_desc(sbase + kGemmB + sb * kStageB);
-#pragma unroll
-          for (int kk = 0; kk < kBK / 16; ++kk)
-            umma_bf16(tmem_d + (uint32_t)(a * kBN), ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
-          umma_commit(bar_emptyB + 8 * sb);      // the box is free once these MMAs have read it
-        }
-        if (go) umma_commit(bar_emptyA + 8 * sa);
+        for (int kk = 1; kk < kSteps; ++kk) umma_16<true>(dt, a_lo + 2u * kk, b_lo + 2u * kk, desc_hi, kIdesc);
+        umma_commit(bar_emptyB + 8 * sb);        // the box is free once the MMAs that read it have completed
+        umma_commit(bar_emptyA + 8 * sa);
+        if (++sa == kStagesA) { sa = 0; pa ^= 1u; }
+        sb += kAcc == 1 ? 1 : kAcc;
+        if (sb >= kStagesB) { sb -= kStagesB; pb ^= 1u; }
       }
-      umma_commit(bar_accum);                    // all MMAs issued so far have completed
+      umma_commit(bar_accum);                    // all MMAs this lane issued have completed
     }
   } else {
     // ---------------- decode warps ----------------
@@ -438,6 +460,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
       for (int cc = gi; cc < kTok / 32; cc += kGroups) {       // the groups share the column chunks
         uint32_t r[32];
         tmem_ld32(tmem_d + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * cc), r);
+        if (kAcc == 1) {
+          // the other half of K sits in the second accumulator
+          uint32_t r2[32];
+          tmem_ld32(tmem_d + ((uint32_t)(32 * q) << 16) + (uint32_t)(kTok + 32 * cc), r2);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+        }
         if (row < n) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
@@ -461,7 +490,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
   if (warp == 1 && lane == 0) mbar_wait(bar_accum, 0u, kGemmWaitLimit);
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_d, kTok);
+  if (warp == 1) tmem_dealloc(tmem_d, kTmemCols);
   if (threadIdx.x == 0 && *abort_flag && dev_status) *dev_status = STB_ERR_TIMEOUT;
 }
 
