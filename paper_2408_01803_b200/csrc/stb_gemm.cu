@@ -452,7 +452,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
 
     // ---------------- epilogue: TMEM -> registers -> Y ----------------
     const int q = warp & 3;                        // TMEM lane quarter of this warp
-    if (__all_sync(0xFFFFFFFFu, gemm_wait(bar_accum, 0u, abort_flag)) && nstage > 0) {
+    // A 16-bit output tile goes through shared memory (the X ring: every box has been consumed by then) so that it
+    // leaves in 16-byte pieces along the rows: straight from the registers a warp's store is 32 rows x 2 bytes of
+    // one token, and the epilogue took a ninth of the CTA's time.  The same for every thread of the CTA:
+    const bool staged = y_16 != 0 && !split && (ldy % 8) == 0 && (reinterpret_cast<uintptr_t>(Y) & 15u) == 0 &&
+                        (uint32_t)kTok * kBM * 2u <= (uint32_t)kStagesB * kStageB;
+    uint16_t* stage = reinterpret_cast<uint16_t*>(smem + kGemmB);           // [token of the tile][row of the tile]
+    const bool have = __all_sync(0xFFFFFFFFu, gemm_wait(bar_accum, 0u, abort_flag)) && nstage > 0;
+    if (have) {
       tc_fence_after();
       const int row = mt * kBM + 32 * q + lane;                // output feature (row of W^)
       float* wsz = split ? ws + ((size_t)(tile - full_tiles) * ksplit + kz) * (size_t)(kBM * kTok) : nullptr;
@@ -467,7 +474,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
         }
-        if (row < n) {
+        if (staged) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float v = __uint_as_float(r[i]);
+            stage[(32 * cc + i) * kBM + 32 * q + lane] = kF16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+          }
+        } else if (row < n) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const int tok = tt * kTok + 32 * cc + i;
@@ -478,6 +491,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
               else if (y_16) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(v);
               else static_cast<float*>(Y)[(size_t)tok * ldy + row] = v;
             }
+          }
+        }
+      }
+    }
+    if (staged) {
+      // every decode warp takes the barrier, whatever its wait said
+      asm volatile("bar.sync 1, %0;" ::"n"(128 * kGroups) : "memory");
+      if (have) {
+        const int d = (warp - 2) * 32 + lane;                  // 0 .. 511: 16 threads per token, 8 rows each
+        const int piece = d & 15, row0 = mt * kBM + 8 * piece;
+        uint16_t* Y16 = static_cast<uint16_t*>(Y);
+#pragma unroll 4
+        for (int tl = d >> 4; tl < kTok; tl += (128 * kGroups) / 16) {
+          const int tok = tt * kTok + tl;
+          if (tok >= T) break;
+          const uint4 v = *reinterpret_cast<const uint4*>(stage + tl * kBM + 8 * piece);
+          uint16_t* dst = Y16 + (size_t)tok * ldy + row0;
+          if (row0 + 8 <= n) *reinterpret_cast<uint4*>(dst) = v;
+          else {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              if (row0 + e < n) dst[e] = (uint16_t)(w[e >> 1] >> (16 * (e & 1)));
           }
         }
       }
