@@ -313,6 +313,7 @@ __device__ __forceinline__ void decode_row(const DecodeArgs& da, const int j) {
 // word w of the layer, and zeros in the 128 columns after the last word (a CTA's last residual stage may reach there).
 __global__ void gemm_gather_kernel(const uint8_t* __restrict__ packed, int n, int m, int N, const __nv_bfloat16* __restrict__ X, int T,
                                    size_t ldx, __nv_bfloat16* __restrict__ Xs, int ldxs) {
+  grid_launch_dependents();        // the GEMM may start; it waits for this grid before it reads Xs
   const Header* hdr = reinterpret_cast<const Header*>(packed);
   if (!header_matches(hdr, n, m, N)) return;
   const int nblk = m / kBlock;
@@ -400,11 +401,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
       for (int hb = 0; hb < nstage * kAcc; ++hb) {
         const int it = hb / kAcc, a = hb % kAcc, s = hb % kStagesB;
         if (!gemm_wait<true>(bar_emptyB + 8 * s, ((uint32_t)(hb / kStagesB) & 1u) ^ 1u, abort_flag)) break;
+        // Xs comes from the gather kernel, which this grid may have overtaken (programmatic dependent launch)
+        if (it == nmain && a == 0) grid_dependency_wait();
         mbar_expect_tx(bar_fullB + 8 * s, box_bytes);
         const uint32_t dst = sbase + kGemmB + s * kStageB;
         if (it < nmain) tma_load_2d(dst, &xmap, (b0 * 2 + it) * kBK, tt * kTok + a * kBN, bar_fullB + 8 * s);
         else tma_load_2d(dst, &xsmap, (int)(4u * (rw0 & ~1u)) + (it - nmain) * kBK, tt * kTok + a * kBN, bar_fullB + 8 * s);
       }
+      grid_dependency_wait();  // (every CTA, whether or not it had residual stages)
       if (*abort_flag) {       // let copies in flight land before the CTA gives its shared memory up
         const long long t0 = clock64();
         while (clock64() - t0 < 200000) {}
@@ -677,10 +681,20 @@ static int launch_gemm(const uint8_t* packed, int n, int m, const void* X, int T
   gemm_gather_kernel<<<148 * 4, 256, 0, s>>>(packed, n, m, N, static_cast<const __nv_bfloat16*>(X), T, ldx,
                                              static_cast<__nv_bfloat16*>(ws), ldxs);
   if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
-  const unsigned grid = (unsigned)(plan.full_tiles + plan.split_tiles * plan.ksplit);
-  gemm_kernel<N, Cfg, kF16><<<grid, kGemmThreads, kSmem, s>>>(map, xsmap, packed, n, m, T, Y, y_16, ldy, ws_split, plan.full_tiles,
-                                                              plan.ksplit, plan.bps, plan.ttiles, box_rows * kBK * 2, dev_status);
-  if (cudaGetLastError() != cudaSuccess) return STB_ERR_CUDA;
+  // The GEMM is a programmatic dependent of the gather: its CTAs may be scheduled while the gather runs (they need
+  // Xs only for the residual stages at the end of their K range) and wait (griddepcontrol.wait) before they read it.
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(plan.full_tiles + plan.split_tiles * plan.ksplit));
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = kSmem;
+  cfg.stream = s;
+  cfg.attrs = pdl; cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, gemm_kernel<N, Cfg, kF16>, map, xsmap, packed, n, m, T, Y, y_16, ldy, ws_split, plan.full_tiles,
+                         plan.ksplit, plan.bps, plan.ttiles, (uint32_t)(box_rows * kBK * 2), dev_status) != cudaSuccess)
+    return STB_ERR_CUDA;
   if (plan.split_tiles > 0) {
     gemm_reduce_kernel<<<148 * 4, 256, 0, s>>>(ws_split, plan.full_tiles, plan.split_tiles, plan.ksplit,
                                                plan.ttiles, kTok, n, T, Y, y_16 ? (kF16 ? 2 : 1) : 0, ldy);
