@@ -538,17 +538,38 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
 // ws[(u ksplit + z)][token 0..ktok-1][row 0..kBM-1]; summed in z order.  y_16: 1 = bf16, 2 = fp16 output.
 __global__ void gemm_reduce_kernel(const float* __restrict__ ws, int first_tile, int split_tiles, int ksplit, int ttiles, int ktok,
                                    int n, int T, void* __restrict__ Y, int y_16, size_t ldy) {
-  const size_t per = (size_t)kBM * ktok, total = (size_t)split_tiles * per;
+  // four consecutive rows of one token per thread: 16-byte loads of the parts, one 8- or 16-byte store
+  const size_t per = (size_t)kBM * ktok, per4 = per / 4, total = (size_t)split_tiles * per4;
+  const bool vec = (ldy % 4) == 0 && (reinterpret_cast<uintptr_t>(Y) & 15u) == 0;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    const size_t u = i / per, r = i % per;
+    const size_t u = i / per4, r = (i % per4) * 4;
     const int tile = first_tile + (int)u, tt = tile % ttiles, mt = tile / ttiles;
     const int tok = tt * ktok + (int)(r / kBM), row = mt * kBM + (int)(r % kBM);
     if (tok >= T || row >= n) continue;
-    float acc = 0.0f;
-    for (int z = 0; z < ksplit; ++z) acc += ws[(u * ksplit + z) * per + r];
-    if (y_16 == 2) static_cast<__half*>(Y)[(size_t)tok * ldy + row] = __float2half_rn(acc);
-    else if (y_16 == 1) static_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(acc);
-    else static_cast<float*>(Y)[(size_t)tok * ldy + row] = acc;
+    float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    for (int z = 0; z < ksplit; ++z) {
+      const float4 v = __ldcs(reinterpret_cast<const float4*>(ws + (u * ksplit + z) * per + r));
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    const size_t o = (size_t)tok * ldy + row;
+    if (vec && row + 4 <= n) {
+      if (y_16 == 2) {
+        const __half2 lo = __floats2half2_rn(acc.x, acc.y), hi = __floats2half2_rn(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(static_cast<__half*>(Y) + o) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+      } else if (y_16 == 1) {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(Y) + o) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+      } else {
+        *reinterpret_cast<float4*>(static_cast<float*>(Y) + o) = acc;
+      }
+    } else {
+      const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+      for (int e = 0; e < 4 && row + e < n; ++e) {
+        if (y_16 == 2) static_cast<__half*>(Y)[o + e] = __float2half_rn(a4[e]);
+        else if (y_16 == 1) static_cast<__nv_bfloat16*>(Y)[o + e] = __float2bfloat16_rn(a4[e]);
+        else static_cast<float*>(Y)[o + e] = a4[e];
+      }
+    }
   }
 }
 
