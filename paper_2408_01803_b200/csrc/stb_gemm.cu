@@ -578,13 +578,14 @@ static int gemm_ksplit(int n, int m, int T, int ktok) {
   const int tiles = ((n + kBM - 1) / kBM) * ((T + ktok - 1) / ktok), nblk = m / kBlock;
   int ks = 1;
   if (ktok < 512) {
-    // decode batch: a CTA's time is the decode of its blocks, so any number of parts with at least four blocks each
-    // will do; take the one that fills the waves of 148 CTAs best (the fewest parts among equals)
+    // decode batch: a CTA's time is a fixed part (prologue, first loads, epilogue: measured about as long as the decode
+    // of seven blocks) plus the decode of its blocks, and the call takes as many such times as it has waves of 148
+    // CTAs: take the number of parts (at least four blocks each) with the smallest product
     double best = 0.0;
-    for (int k = 1; k <= 16 && nblk / k >= 4; ++k) {
+    for (int k = 1; k <= 16 && (k == 1 || nblk / k >= 4); ++k) {
       const long long ctas = (long long)tiles * k, waves = (ctas + 147) / 148;
-      const double fill = (double)ctas / (double)(waves * 148);
-      if (fill > best + 1e-9) { best = fill; ks = k; }
+      const double cost = (double)waves * (7.0 + (double)((nblk + k - 1) / k));
+      if (k == 1 || cost < best - 1e-9) { best = cost; ks = k; }
     }
   } else {
     if (tiles < 100) ks = 148 / tiles;
