@@ -345,6 +345,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
   constexpr int kAcc = Cfg::kAcc, kBN = Cfg::kBN, kTok = Cfg::kTok, kStagesB = Cfg::kStagesB;
   constexpr uint32_t kStageB = Cfg::kStageB, kIdesc = GemmIdesc<kBN, kF16>::value;
   extern __shared__ __align__(1024) uint8_t smem[];
+  // (the position table's entry of this thread is asked for before the header: two global-memory latencies side by
+  // side instead of one after the other in every CTA's prologue)
+  uint32_t tab_entry = 0;
+  if (threadIdx.x < kPosTableEntries) tab_entry = g_pos_table.v[N][threadIdx.x].x | (g_pos_table.v[N][threadIdx.x].y << 16);
   const Header* hdr = reinterpret_cast<const Header*>(packed);
   if (!header_matches(hdr, n, m, N)) {
     if (threadIdx.x == 0 && dev_status) *dev_status = STB_ERR_CORRUPT;
@@ -386,8 +390,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CU
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  for (int i = threadIdx.x; i < kPosTableEntries; i += blockDim.x)     // 4-byte entries: fewer bank conflicts than 8-byte ones
-    reinterpret_cast<uint32_t*>(smem + kGemmTab)[i] = g_pos_table.v[N][i].x | (g_pos_table.v[N][i].y << 16);
+  static_assert(kPosTableEntries <= kGemmThreads, "one table entry per thread");
+  if (threadIdx.x < kPosTableEntries) reinterpret_cast<uint32_t*>(smem + kGemmTab)[threadIdx.x] = tab_entry;   // 4-byte entries: fewer bank conflicts than 8-byte ones
   constexpr uint32_t kTmemCols = kAcc == 1 ? 2 * kTok : kTok;      // one accumulator: a second one for the other half of K
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   tc_fence_before();
