@@ -396,6 +396,33 @@ def test_gemm_f16_full_size_decode_batch(stb, name):
     assert e.value.status == stb.STB_ERR_SIZE
 
 
+@pytest.mark.parametrize("n,ldy,shift", [(100, 104, 0), (200, 208, 0), (136, 136, 8), (136, 144, 2)])
+def test_gemm_16_bit_output_layouts(stb, n, ldy, shift):
+    """16-bit outputs leave through shared memory in 16-byte pieces when the output allows it (row stride a multiple of
+    8, base 16-byte aligned) and element by element otherwise; a last piece of rows that crosses n is cut.  Every
+    layout must give the fp32 result rounded, and must not touch what lies beside the output."""
+    import torch
+    m, N = 512, 5
+    L = _quantized(n, m, N, 2300 + n)
+    layer = stb.pack_numpy(_fields(L))
+    for dt, act, T in ((torch.bfloat16, "bf16", 70), (torch.float16, None, 70), (torch.float16, None, 40)):
+        x = si.activations(T, m, 77, act) if act else si.activations(T, m, 77)
+        xd = torch.from_numpy(x).cuda().to(dt)
+        fn = stb.gemm if act else stb.gemm_f16
+        y32 = fn(layer, xd)
+        buf = torch.full((T * ldy + 16,), 7.0, dtype=dt, device="cuda")
+        out = buf[shift:shift + T * ldy].view(T, ldy)[:, :n]
+        fn(layer, xd, out=out)
+        torch.cuda.synchronize()
+        assert int(layer.dev_status.item()) == 0
+        assert torch.equal(out, y32.to(dt))
+        mask = torch.ones(T * ldy + 16, dtype=torch.bool, device="cuda")
+        mask[shift:shift + T * ldy].view(T, ldy)[:, :n] = False
+        assert bool((buf[mask] == 7.0).all()), "wrote outside the output"
+        ref = oracle.matmul(oracle.decode(L), x.astype(np.float64))
+        assert np.abs(y32.double().cpu().numpy() - ref).max() <= TOL * np.abs(ref).max()
+
+
 def test_gemm_split_k_uses_the_workspace(stb):
     """Few output tiles and a long K: the launch splits K, partial sums go through the caller's workspace."""
     import torch
