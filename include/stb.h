@@ -171,8 +171,8 @@ int stb_gemm(const void *packed, int n, int m, int N, const void *X, int T, size
  * fp16 with its scales as stored (no rounding: a kept weight is s a_region exactly, a salient one s1 a_sal1 + s2 a_sal2 as
  * two terms of the sum), so the result is the one stb_gemv defines.  Meant for decode batches beyond what the GEMV
  * kernels do well (Appendix C.2 between its two stages: tens of tokens): for T <= 64 the CTA tile is 128 rows x 64 tokens
- * (one accumulator of 64 TMEM columns), K is split into as many parts as fill the 148 SMs best and the kernel runs at the
- * speed of its decode warps; for T > 64 it is stb_gemm's tiling.  The workspace (stb_gemm_f16_workspace bytes, 256-byte
+ * (one accumulator of 64 TMEM columns per MMA-issuing lane), K is split into the number of parts that makes waves of
+ * 148 CTAs x (a CTA's fixed cost + its blocks) smallest, and the kernel runs at the speed of its decode warps; for T > 64 it is stb_gemm's tiling.  The workspace (stb_gemm_f16_workspace bytes, 256-byte
  * aligned; the gathered residual activations and the fp32 partial tiles) is required.  Errors as stb_gemm. */
 int stb_gemm_f16_workspace(int n, int m, int N, int T, size_t *bytes);
 int stb_gemm_f16(const void *packed, int n, int m, int N, const void *X, int T, size_t ldx, void *Y,
