@@ -434,6 +434,11 @@ def gemm_table(stb, torch, pk, real_ffn, only=None):
                "frac_of_measured_bf16_sustained": round(fl / us / 1e6 / pk["bf16_tflops_sustained"], 4),
                "useful_TFLOPs": round(fl * N / 8 / us / 1e6, 1), "split_k_workspace_MB": round(need / 1e6, 1),
                "cublas_bf16_us": round(usd, 1), "cublas_bf16_TFLOPs": round(fl / usd / 1e6, 1)}
+        # the same in the form of the headline's roofline object: a dense contraction against the measured cuBLAS burst peak
+        # (the kernel is timed alone); the whole call (gather, GEMM, sum of K parts) counts as the kernel's time
+        row["roofline"] = {"bound": "tensor", "achieved": round(fl / us / 1e6, 1), "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                           "frac": round(fl / us / 1e6 / pk["bf16_tflops"], 4), "traffic": None, "kernel": "stb::gemm_kernel",
+                           "peak_source": pk["_source"]}
         if hist:
             row["salient_columns_per_block"] = hist
         out.append(row)
